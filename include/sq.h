@@ -1,0 +1,229 @@
+/*
+ * sq.h -- C ABI of libsq: the SmoothQuant W8A8 hot path on NVIDIA B200 (sm_100a).
+ *
+ * Notation follows the paper: an activation X has T tokens (rows, "M") and C_i input
+ * channels (columns, "K"); a linear layer has C_o output channels ("N").  Weights are
+ * STORED as W[C_o, C_i] row-major, i.e. the transpose of the paper's W in R^{C_i x C_o},
+ * so both GEMM operands have the reduction dimension contiguous.  "A" below is the
+ * activation dtype, SQ_F16 or SQ_BF16.
+ *
+ * Conventions shared by every call
+ * --------------------------------
+ *  - Every pointer is a DEVICE pointer owned by the caller (unless it says "host"),
+ *    valid until the work queued on `stream` has finished.  The library never allocates
+ *    or frees device memory in these calls and keeps no state between them.
+ *  - Tensors are row-major with the innermost dimension contiguous.  Base pointers and
+ *    row strides of INT8 operands of the GEMM/BMM must be multiples of 16 bytes
+ *    (they are read by TMA); otherwise SQ_ERR_ALIGN.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *    Calls only enqueue work: they never synchronise and never change the current device.
+ *  - The return code reports argument validation and launch errors.  Device-side waits
+ *    are bounded; if one expires the kernel records a non-zero word at workspace[0]
+ *    (see sq_w8a8_gemm) and returns instead of hanging.
+ *  - Rounding is round-to-nearest-even everywhere; INT8 codes lie in [-127, 127].
+ *  - Inputs must be finite; NaN/Inf give unspecified codes (never a fault).
+ *  - A zero-sized problem (M == 0 or N == 0 ...) is a no-op that returns SQ_OK.
+ */
+#ifndef SQ_H_
+#define SQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SQ_OK = 0,
+    SQ_ERR_INVALID_ARG = 1, /* null pointer, bad enum, alpha outside [0,1] ...          */
+    SQ_ERR_SHAPE = 2,       /* negative size, stride smaller than the row                */
+    SQ_ERR_ALIGN = 3,       /* pointer or stride not aligned as the call requires        */
+    SQ_ERR_UNSUPPORTED = 4, /* e.g. K > 133144 (INT32 accumulator could overflow)        */
+    SQ_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed (launch, tensor map)    */
+    SQ_ERR_TIMEOUT = 6,     /* value stored at workspace[0] by a kernel whose wait ran out */
+    SQ_ERR_WORKSPACE = 7    /* workspace missing or smaller than sq_workspace_bytes()    */
+} sq_status;
+
+typedef enum { SQ_F16 = 0, SQ_BF16 = 1, SQ_I8 = 2, SQ_I32 = 3 } sq_dtype;
+
+/* Activation quantisation granularity (Table 2): O3, O2, O1. */
+typedef enum {
+    SQ_PER_TENSOR_STATIC = 0,
+    SQ_PER_TENSOR_DYNAMIC = 1,
+    SQ_PER_TOKEN_DYNAMIC = 2
+} sq_act_gran;
+
+/* Weight quantisation granularity (Fig. 3): one step size, or one per output channel. */
+typedef enum { SQ_W_PER_TENSOR = 0, SQ_W_PER_CHANNEL = 1 } sq_w_gran;
+
+typedef enum { SQ_EPI_NONE = 0, SQ_EPI_RELU = 1 } sq_epilogue_act;
+
+/* Operation ids for sq_workspace_bytes(). */
+typedef enum {
+    SQ_OP_QUANT_ACT = 0,
+    SQ_OP_LN_QUANT = 1,
+    SQ_OP_QUANT_WEIGHT = 2,
+    SQ_OP_GEMM = 3,
+    SQ_OP_BMM = 4
+} sq_op;
+
+/* Largest reduction length for which |sum| <= 127*127*K stays inside INT32. */
+#define SQ_MAX_K 133144
+
+/* Human-readable name of a status code (host pointer to a static string). */
+const char* sq_status_str(sq_status s);
+
+/* Bytes of caller-provided workspace `op` needs for the given sizes (host call, no CUDA
+ * work).  The workspace must be 256-byte aligned and ZERO-FILLED ONCE by the caller before
+ * its first use; every call leaves it zero-filled again except for workspace[0..3], the
+ * sticky device status word (0 = no device-side error).  M is the token count, N/K as in
+ * the call; pass 0 for sizes the op does not have. */
+size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K);
+
+/*
+ * Calibration statistic of Section 4 ("s_j = max(|X_j|)", estimated on calibration
+ * samples): running per-channel absolute maximum
+ *     absmax[j] = max(absmax[j], max_t |X[t, j]|).
+ * X: [rows, cols] of dtype `dt` (F16/BF16) with row stride `ld` elements (ld >= cols).
+ * absmax_inout: [cols] fp32, updated in place; the caller zero-initialises it before the
+ * first batch and may call once per calibration batch.  Applied to the stored weight
+ * W[C_o, C_i] it yields max(|W_j|) of Eq. 4 (one value per INPUT channel).
+ * The fast path needs X 16-byte aligned with cols and ld multiples of 8; other shapes run
+ * a slower element-wise kernel.
+ */
+sq_status sq_calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld,
+                          float* absmax_inout, void* stream);
+
+/*
+ * Smoothing factor, Eq. 4:  s_j = max|X_j|^alpha / max|W_j|^(1-alpha),  j < C.
+ * act_absmax, w_absmax: [C] fp32 (both floored at 1e-5 so that s_j is finite and
+ * non-zero); alpha in [0, 1] else SQ_ERR_INVALID_ARG; s_out: [C] fp32.  The powers are
+ * evaluated in double precision and rounded once to fp32.  s_inv_out: optional [C] fp32,
+ * receives 1/s_j (fp32 division) -- the explicit activation-side multiplier of Eq. 3 for a
+ * producer whose parameters cannot absorb it (see col_mul of sq_quant_act).
+ */
+sq_status sq_smooth_scales(const float* act_absmax, const float* w_absmax, int64_t C, float alpha,
+                           float* s_out, float* s_inv_out, void* stream);
+
+/*
+ * Eq. 3, activation side, folded offline into the preceding LayerNorm (Section 4: the
+ * smoothing factor is fused into the previous layer's parameters, so no scaling runs at
+ * inference):  gamma_out = gamma / s,  beta_out = beta / s  (fp32 division, result rounded
+ * to `dt`).  gamma, beta, gamma_out, beta_out: [C] of dtype dt; beta and beta_out may both
+ * be NULL.  In-place (gamma_out == gamma) is allowed.
+ */
+sq_status sq_fold_ln_weight(const void* gamma, const void* beta, sq_dtype dt, const float* s,
+                            int64_t C, void* gamma_out, void* beta_out, void* stream);
+
+/*
+ * Eq. 3 weight side and Eq. 1:  W_hat[o, j] = W[o, j] * s_j (fp32, s == NULL means s_j = 1),
+ * Delta_w = max|W_hat| / 127 per output channel (row) or per tensor,
+ * Wq = clamp(round(W_hat / Delta_w), -127, 127).
+ * W: [N, K] dtype dt, contiguous.  Wq: [N, K] int8.  w_scale: [N] (per channel) or [1]
+ * fp32, receives Delta_w.  workspace: sq_workspace_bytes(SQ_OP_QUANT_WEIGHT, ...) bytes
+ * (only the per-tensor mode uses it).  K must be a multiple of 8 and W 16-byte aligned.
+ */
+sq_status sq_quant_weight(const void* W, sq_dtype dt, int64_t N, int64_t K, const float* s,
+                          sq_w_gran g, int8_t* Wq, float* w_scale, void* workspace,
+                          size_t ws_bytes, void* stream);
+
+/*
+ * Eq. 1 on an activation tensor, at the three granularities of Table 2.
+ *   per-token dynamic : Delta_t = max_j |x[t, j]| / 127, written to x_scale[t]   ([M])
+ *   per-tensor dynamic: one Delta from the whole [M, C] of this call -> x_scale[0]
+ *   per-tensor static : Delta = x_scale[0] is an INPUT (from calibration); larger values
+ *                       saturate at +-127
+ * Xq = clamp(round(x * (1/Delta)), -127, 127); maxima are floored at 1e-5.
+ * X: [M, C] dtype dt, contiguous, 16-byte aligned, C a multiple of 8.  col_mul: optional
+ * [C] fp32 multiplier applied first in fp32 (an explicit 1/s when the producer is not a
+ * LayerNorm); NULL for none.  Xq: [M, C] int8.  workspace: used by the per-tensor dynamic
+ * mode only.
+ */
+sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_gran g,
+                       const float* col_mul, int8_t* Xq, float* x_scale, void* workspace,
+                       size_t ws_bytes, void* stream);
+
+/*
+ * Fused LayerNorm (with the smoothing factor already folded into gamma_hat, beta_hat by
+ * sq_fold_ln_weight) + Eq. 1, one pass over X:
+ *     mu_t, var_t = mean and biased variance of row t (fp32, two-pass),
+ *     y = fma((x - mu_t) * rstd_t, gamma_hat_j, beta_hat_j),  rstd_t = 1/sqrt(var_t + eps),
+ * then y is quantised exactly as in sq_quant_act WITHOUT being rounded to A first.
+ * X: [M, C] dtype dt; gamma_hat, beta_hat: [C] dtype dt (beta_hat may be NULL).
+ * dbg_mean_rstd: optional [2*M] fp32, receives mu_t at [2t] and rstd_t at [2t+1] so that a
+ * checker can reproduce the element-wise part bit for bit.  Other arguments as sq_quant_act.
+ */
+sq_status sq_ln_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma_hat,
+                      const void* beta_hat, float eps, sq_act_gran g, int8_t* Xq, float* x_scale,
+                      float* dbg_mean_rstd, void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * The W8A8 linear layer, Eq. 2:
+ *     acc[t, o] = sum_j Xq[t, j] * Wq[o, j]                         (INT32, exact)
+ *     y[t, o]   = fma((float)acc, x_scale[t] * w_scale[o], bias[o]) (fp32), optional ReLU
+ * and then ONE of
+ *     Y = round_to(out_dt)(y)                         out_dt = SQ_F16 / SQ_BF16
+ *     Y = clamp(round(y * requant_mul[o or 0]))       out_dt = SQ_I8 (requant_mul != NULL)
+ *     Y = acc                                         out_dt = SQ_I32 (raw accumulators;
+ *                                                     scales, bias, ReLU ignored)
+ * Xq: [M, K] int8, row stride K.  Wq: [N, K] int8, row stride K.  K a multiple of 16,
+ * K <= SQ_MAX_K.  x_scale: [M] if x_scale_is_per_token else [1]; w_scale: [N] if
+ * w_scale_is_per_channel else [1].  bias: [N] of dtype bias_dt (F16/BF16) or NULL.
+ * requant_mul: [N] if requant_is_per_channel else [1]; required iff out_dt == SQ_I8.
+ * row_absmax_out: optional [M] fp32, caller-zeroed; receives max_o |y[t, o]| (after ReLU,
+ * before output rounding) via atomic max, so that the next layer's per-token step size
+ * needs no extra pass.  Y: [M, N] with row stride ldy elements.
+ * workspace: sq_workspace_bytes(SQ_OP_GEMM, M, N, K) bytes; word 0 is the device status.
+ */
+sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
+                       const float* x_scale, int x_scale_is_per_token, const float* w_scale,
+                       int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt,
+                       sq_epilogue_act act, const float* requant_mul, int requant_is_per_channel,
+                       float* row_absmax_out, void* Y, sq_dtype out_dt, int64_t ldy,
+                       void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * INT8 batched matmul for attention (Fig. 6: the BMMs run in INT8):
+ * for every b < batch, h < heads
+ *     acc = A[b,h] * B[b,h]^T   (B stored [N, K], K contiguous;  b_is_kn == 0)   e.g. Q.K^T
+ *     acc = A[b,h] * B[b,h]     (B stored [K, N], N contiguous;  b_is_kn != 0)   e.g. P.V
+ *     C[b,h] = round_to(out_dt)((float)acc * alpha)          out_dt = SQ_F16 / SQ_BF16
+ *     C[b,h] = clamp(round(((float)acc * alpha) * *requant_mul))   out_dt = SQ_I8
+ *     C[b,h] = acc                                           out_dt = SQ_I32
+ * A[b,h]: [M, K] int8.  strideX[3] = {batch stride, head stride, row stride} in ELEMENTS
+ * (HOST arrays); the innermost dimension is contiguous.  All strides of A and B must be
+ * multiples of 16; K a multiple of 16; with b_is_kn, N must be a multiple of 16 and at
+ * most 128 (the head dimension).  alpha carries the operands' static step sizes (and
+ * 1/sqrt(d) for Q.K^T).  requant_mul: device pointer to one fp32, required iff out_dt == SQ_I8.
+ * Strided views let Q, K, V be read in place from the fused QKV GEMM output [T, 3*H*d].
+ */
+sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M,
+                      int64_t N, int64_t K, const int64_t strideA[3], const int64_t strideB[3],
+                      int b_is_kn, float alpha, const float* requant_mul, void* C, sq_dtype out_dt,
+                      const int64_t strideC[3], void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Attention plumbing between the two BMMs (Fig. 6 keeps Softmax in floating point):
+ * causal softmax over each [S, S] score matrix followed by quantisation of the
+ * probabilities with the fixed step 1/127 (softmax output lies in [0, 1]):
+ *     p[i, j] = exp(s[i, j] - max_i) / sum_{j' <= i} exp(s[i, j'] - max_i),  0 for j > i
+ *     Pq[i, j] = round(127 * p[i, j])
+ * scores: [n_mat, S, S] dtype dt (F16/BF16), contiguous; Pq: [n_mat, S, S] int8.
+ * S a multiple of 8.  Computed in fp32; exp and the row sum are not bit-reproducible
+ * against another implementation, so codes may differ by one at rounding ties.
+ */
+sq_status sq_softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_t S, int8_t* Pq,
+                             void* stream);
+
+/*
+ * Residual add around a sub-layer (pre-LayerNorm block): out = a + b in fp32, rounded to dt.
+ * a, b, out: [n] dtype dt, n a multiple of 8, 16-byte aligned; out may alias a.
+ */
+sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out,
+                          void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQ_H_ */

@@ -104,6 +104,15 @@ def smooth_scales(act_absmax, w_absmax, alpha: float):
     return s
 
 
+def smooth_scales_inv(s):
+    """The explicit activation-side factor of Eq. 3, 1/s_j, as one fp32 division."""
+    s = _f32(s)
+    o = np.empty_like(s)
+    one = np.ones_like(s)
+    _lib.sqo_div_by_s(_p(one, _f32p), _p(s, _f32p), _i64(s.size), _p(o, _f32p))
+    return o
+
+
 def fold_ln_weight(gamma, beta, s, dtype: str):
     """Eq. 3 folded offline into the preceding LayerNorm: gamma/s, beta/s, stored in `dtype`."""
     s = _f32(s)

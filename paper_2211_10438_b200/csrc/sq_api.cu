@@ -1,0 +1,238 @@
+// extern "C" entry points of libsq: argument validation and kernel dispatch only.
+#include "sq_common.cuh"
+#include "sq_kernels.h"
+
+using namespace sq;
+
+namespace {
+
+inline bool is_act_dtype(sq_dtype dt) { return dt == SQ_F16 || dt == SQ_BF16; }
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+inline float* ws_absmax(void* ws) { return reinterpret_cast<float*>(static_cast<char*>(ws) + kWsAbsmaxOff); }
+inline float* ws_stats(void* ws) { return reinterpret_cast<float*>(static_cast<char*>(ws) + kWsHeader); }
+inline bool ws_ok(const void* ws, size_t have, size_t need) {
+    return ws != nullptr && have >= need && (reinterpret_cast<uintptr_t>(ws) & 255) == 0;
+}
+
+// shared body of sq_quant_act / sq_ln_quant / sq_quant_weight
+sq_status quant_rows_common(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul,
+                            const void* gamma, const void* beta, float eps, bool ln, int gran /*sq_act_gran*/,
+                            int8_t* Xq, float* scale, float* dbg_stats, void* workspace, size_t ws_bytes,
+                            size_t ws_need, cudaStream_t st) {
+    if (gran == SQ_PER_TOKEN_DYNAMIC)
+        return row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_DYNAMIC, Xq, scale, nullptr,
+                         dbg_stats, 0, st);
+    if (gran == SQ_PER_TENSOR_STATIC)
+        return row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_GIVEN_SCALE, Xq, scale, nullptr,
+                         dbg_stats, 0, st);
+    // per-tensor dynamic: pass 1 folds every row's maximum into one word (and keeps the
+    // LayerNorm statistics), pass 2 quantises with the step derived from it
+    if (!ws_ok(workspace, ws_bytes, ws_need)) return SQ_ERR_WORKSPACE;
+    float* word = ws_absmax(workspace);
+    float* stats = ln ? (dbg_stats ? dbg_stats : ws_stats(workspace)) : nullptr;
+    sq_status s = row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_ABSMAX_ONLY, nullptr, nullptr,
+                            word, stats, 0, st);
+    if (s != SQ_OK) return s;
+    s = row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_FROM_ABSMAX_WORD, Xq, scale, word, stats,
+                  ln ? 1 : 0, st);
+    if (s != SQ_OK) return s;
+    SQ_CUDA_OK(cudaMemsetAsync(word, 0, sizeof(float), st));  // leave the workspace zero-filled
+    if (ln && !dbg_stats) SQ_CUDA_OK(cudaMemsetAsync(stats, 0, (size_t)M * 2 * sizeof(float), st));
+    return SQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* sq_status_str(sq_status s) {
+    switch (s) {
+        case SQ_OK: return "SQ_OK";
+        case SQ_ERR_INVALID_ARG: return "SQ_ERR_INVALID_ARG";
+        case SQ_ERR_SHAPE: return "SQ_ERR_SHAPE";
+        case SQ_ERR_ALIGN: return "SQ_ERR_ALIGN";
+        case SQ_ERR_UNSUPPORTED: return "SQ_ERR_UNSUPPORTED";
+        case SQ_ERR_CUDA: return "SQ_ERR_CUDA";
+        case SQ_ERR_TIMEOUT: return "SQ_ERR_TIMEOUT";
+        case SQ_ERR_WORKSPACE: return "SQ_ERR_WORKSPACE";
+    }
+    return "SQ_ERR_UNKNOWN";
+}
+
+size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K) {
+    (void)N; (void)K;
+    switch (op) {
+        case SQ_OP_LN_QUANT: return kWsHeader + (size_t)(M > 0 ? M : 0) * 2 * sizeof(float);
+        case SQ_OP_QUANT_ACT:
+        case SQ_OP_QUANT_WEIGHT:
+        case SQ_OP_GEMM:
+        case SQ_OP_BMM: return kWsHeader;
+    }
+    return kWsHeader;
+}
+
+sq_status sq_calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld,
+                          float* absmax_inout, void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (rows < 0 || cols < 0 || ld < cols) return SQ_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return SQ_OK;
+    if (!X || !absmax_inout) return SQ_ERR_INVALID_ARG;
+    return calib_absmax(X, dt, rows, cols, ld, absmax_inout, as_stream(stream));
+}
+
+sq_status sq_smooth_scales(const float* act_absmax, const float* w_absmax, int64_t C, float alpha,
+                           float* s_out, float* s_inv_out, void* stream) {
+    if (!(alpha >= 0.0f && alpha <= 1.0f)) return SQ_ERR_INVALID_ARG;
+    if (C < 0) return SQ_ERR_SHAPE;
+    if (C == 0) return SQ_OK;
+    if (!act_absmax || !w_absmax || !s_out) return SQ_ERR_INVALID_ARG;
+    return smooth_scales(act_absmax, w_absmax, C, alpha, s_out, s_inv_out, as_stream(stream));
+}
+
+sq_status sq_fold_ln_weight(const void* gamma, const void* beta, sq_dtype dt, const float* s, int64_t C,
+                            void* gamma_out, void* beta_out, void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (C < 0) return SQ_ERR_SHAPE;
+    if (C == 0) return SQ_OK;
+    if (!gamma || !gamma_out || !s) return SQ_ERR_INVALID_ARG;
+    if ((beta == nullptr) != (beta_out == nullptr)) return SQ_ERR_INVALID_ARG;
+    return fold_ln_weight(gamma, beta, dt, s, C, gamma_out, beta_out, as_stream(stream));
+}
+
+sq_status sq_quant_weight(const void* W, sq_dtype dt, int64_t N, int64_t K, const float* s, sq_w_gran g,
+                          int8_t* Wq, float* w_scale, void* workspace, size_t ws_bytes, void* stream) {
+    if (!is_act_dtype(dt) || (g != SQ_W_PER_TENSOR && g != SQ_W_PER_CHANNEL)) return SQ_ERR_INVALID_ARG;
+    if (N < 0 || K < 0) return SQ_ERR_SHAPE;
+    if (N == 0 || K == 0) return SQ_OK;
+    if (!W || !Wq || !w_scale) return SQ_ERR_INVALID_ARG;
+    if (K % 8 != 0 || !aligned16(W) || (reinterpret_cast<uintptr_t>(Wq) & 7) != 0 || (s && !aligned16(s)))
+        return SQ_ERR_ALIGN;
+    // a weight row is quantised exactly like a token row whose column multiplier is s
+    return quant_rows_common(W, dt, N, K, s, nullptr, nullptr, 0.0f, false,
+                             g == SQ_W_PER_CHANNEL ? SQ_PER_TOKEN_DYNAMIC : SQ_PER_TENSOR_DYNAMIC, Wq, w_scale,
+                             nullptr, workspace, ws_bytes, sq_workspace_bytes(SQ_OP_QUANT_WEIGHT, N, N, K),
+                             as_stream(stream));
+}
+
+sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_gran g, const float* col_mul,
+                       int8_t* Xq, float* x_scale, void* workspace, size_t ws_bytes, void* stream) {
+    if (!is_act_dtype(dt) || g < SQ_PER_TENSOR_STATIC || g > SQ_PER_TOKEN_DYNAMIC) return SQ_ERR_INVALID_ARG;
+    if (M < 0 || C < 0) return SQ_ERR_SHAPE;
+    if (M == 0 || C == 0) return SQ_OK;
+    if (!X || !Xq || !x_scale) return SQ_ERR_INVALID_ARG;
+    if (C % 8 != 0 || !aligned16(X) || (reinterpret_cast<uintptr_t>(Xq) & 7) != 0 ||
+        (col_mul && !aligned16(col_mul)))
+        return SQ_ERR_ALIGN;
+    return quant_rows_common(X, dt, M, C, col_mul, nullptr, nullptr, 0.0f, false, g, Xq, x_scale, nullptr,
+                             workspace, ws_bytes, sq_workspace_bytes(SQ_OP_QUANT_ACT, M, 0, C),
+                             as_stream(stream));
+}
+
+sq_status sq_ln_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma_hat,
+                      const void* beta_hat, float eps, sq_act_gran g, int8_t* Xq, float* x_scale,
+                      float* dbg_mean_rstd, void* workspace, size_t ws_bytes, void* stream) {
+    if (!is_act_dtype(dt) || g < SQ_PER_TENSOR_STATIC || g > SQ_PER_TOKEN_DYNAMIC || !(eps >= 0.0f))
+        return SQ_ERR_INVALID_ARG;
+    if (M < 0 || C < 0) return SQ_ERR_SHAPE;
+    if (M == 0 || C == 0) return SQ_OK;
+    if (!X || !Xq || !x_scale || !gamma_hat) return SQ_ERR_INVALID_ARG;
+    if (C % 8 != 0 || !aligned16(X) || (reinterpret_cast<uintptr_t>(Xq) & 7) != 0 || !aligned16(gamma_hat) ||
+        (beta_hat && !aligned16(beta_hat)))
+        return SQ_ERR_ALIGN;
+    return quant_rows_common(X, dt, M, C, nullptr, gamma_hat, beta_hat, eps, true, g, Xq, x_scale,
+                             dbg_mean_rstd, workspace, ws_bytes, sq_workspace_bytes(SQ_OP_LN_QUANT, M, 0, C),
+                             as_stream(stream));
+}
+
+sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
+                       const float* x_scale, int x_scale_is_per_token, const float* w_scale,
+                       int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt, sq_epilogue_act act,
+                       const float* requant_mul, int requant_is_per_channel, float* row_absmax_out, void* Y,
+                       sq_dtype out_dt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (M < 0 || N < 0 || K < 0) return SQ_ERR_SHAPE;
+    if (out_dt < SQ_F16 || out_dt > SQ_I32 || (act != SQ_EPI_NONE && act != SQ_EPI_RELU)) return SQ_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return SQ_OK;
+    if (K == 0) return SQ_ERR_SHAPE;
+    if (K > SQ_MAX_K) return SQ_ERR_UNSUPPORTED;
+    if (ldy < N) return SQ_ERR_SHAPE;
+    if (!Xq || !Wq || !Y) return SQ_ERR_INVALID_ARG;
+    if (out_dt != SQ_I32 && (!x_scale || !w_scale)) return SQ_ERR_INVALID_ARG;
+    if ((out_dt == SQ_I8) != (requant_mul != nullptr)) return SQ_ERR_INVALID_ARG;
+    if (bias && !is_act_dtype(bias_dt)) return SQ_ERR_INVALID_ARG;
+    if (K % 16 != 0 || !aligned16(Xq) || !aligned16(Wq)) return SQ_ERR_ALIGN;
+    if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_GEMM, M, N, K))) return SQ_ERR_WORKSPACE;
+    GemmArgs a{};
+    a.A = Xq; a.B = Wq;
+    a.batch = 1; a.heads = 1; a.M = M; a.N = N; a.K = K;
+    a.strideA[0] = M * K; a.strideA[1] = M * K; a.strideA[2] = K;
+    a.strideB[0] = N * K; a.strideB[1] = N * K; a.strideB[2] = K;
+    a.b_is_kn = 0;
+    a.x_scale = x_scale; a.x_per_row = x_scale_is_per_token;
+    a.w_scale = w_scale; a.w_per_col = w_scale_is_per_channel;
+    a.alpha = 1.0f;
+    a.bias = bias; a.bias_dt = bias_dt;
+    a.relu = act == SQ_EPI_RELU;
+    a.requant_mul = requant_mul; a.requant_per_col = requant_is_per_channel;
+    a.row_absmax_out = row_absmax_out;
+    a.C = Y; a.out_dt = out_dt;
+    a.strideC[0] = 0; a.strideC[1] = 0; a.strideC[2] = ldy;
+    a.status = reinterpret_cast<uint32_t*>(workspace);
+    return gemm_i8(a, as_stream(stream));
+}
+
+sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M, int64_t N,
+                      int64_t K, const int64_t strideA[3], const int64_t strideB[3], int b_is_kn, float alpha,
+                      const float* requant_mul, void* C, sq_dtype out_dt, const int64_t strideC[3],
+                      void* workspace, size_t ws_bytes, void* stream) {
+    if (batch < 0 || heads < 0 || M < 0 || N < 0 || K < 0) return SQ_ERR_SHAPE;
+    if (out_dt < SQ_F16 || out_dt > SQ_I32) return SQ_ERR_INVALID_ARG;
+    if (batch == 0 || heads == 0 || M == 0 || N == 0) return SQ_OK;
+    if (K == 0) return SQ_ERR_SHAPE;
+    if (K > SQ_MAX_K) return SQ_ERR_UNSUPPORTED;
+    if (!A || !B || !C || !strideA || !strideB || !strideC) return SQ_ERR_INVALID_ARG;
+    if ((out_dt == SQ_I8) != (requant_mul != nullptr)) return SQ_ERR_INVALID_ARG;
+    if (b_is_kn && N > 128) return SQ_ERR_UNSUPPORTED;
+    if (K % 16 != 0 || (b_is_kn && N % 16 != 0) || !aligned16(A) || !aligned16(B)) return SQ_ERR_ALIGN;
+    for (int i = 0; i < 3; ++i) {
+        if (strideA[i] < 0 || strideB[i] < 0 || strideC[i] < 0) return SQ_ERR_SHAPE;
+        if (strideA[i] % 16 != 0 || strideB[i] % 16 != 0) return SQ_ERR_ALIGN;
+    }
+    if (strideA[2] < K || strideB[2] < (b_is_kn ? N : K) || strideC[2] < N) return SQ_ERR_SHAPE;
+    if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_BMM, M, N, K))) return SQ_ERR_WORKSPACE;
+    GemmArgs a{};
+    a.A = A; a.B = B;
+    a.batch = batch; a.heads = heads; a.M = M; a.N = N; a.K = K;
+    for (int i = 0; i < 3; ++i) { a.strideA[i] = strideA[i]; a.strideB[i] = strideB[i]; a.strideC[i] = strideC[i]; }
+    a.b_is_kn = b_is_kn ? 1 : 0;
+    a.x_scale = nullptr; a.x_per_row = 0;
+    a.w_scale = nullptr; a.w_per_col = 0;
+    a.alpha = alpha;
+    a.bias = nullptr; a.bias_dt = SQ_F16;
+    a.relu = 0;
+    a.requant_mul = requant_mul; a.requant_per_col = 0;
+    a.row_absmax_out = nullptr;
+    a.C = C; a.out_dt = out_dt;
+    a.status = reinterpret_cast<uint32_t*>(workspace);
+    return gemm_i8(a, as_stream(stream));
+}
+
+sq_status sq_softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_t S, int8_t* Pq,
+                             void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (n_mat < 0 || S < 0) return SQ_ERR_SHAPE;
+    if (n_mat == 0 || S == 0) return SQ_OK;
+    if (!scores || !Pq) return SQ_ERR_INVALID_ARG;
+    if (S % 8 != 0 || !aligned16(scores) || (reinterpret_cast<uintptr_t>(Pq) & 7) != 0) return SQ_ERR_ALIGN;
+    return softmax_quant_p(scores, dt, n_mat, S, Pq, as_stream(stream));
+}
+
+sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out, void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (n < 0) return SQ_ERR_SHAPE;
+    if (n == 0) return SQ_OK;
+    if (!a || !b || !out) return SQ_ERR_INVALID_ARG;
+    if (n % 8 != 0 || !aligned16(a) || !aligned16(b) || !aligned16(out)) return SQ_ERR_ALIGN;
+    return residual_add(a, b, dt, n, out, as_stream(stream));
+}
+
+}  // extern "C"

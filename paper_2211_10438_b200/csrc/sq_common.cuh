@@ -1,0 +1,146 @@
+// Shared device/host helpers of libsq (CUDA side only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/sq.h"
+
+namespace sq {
+
+constexpr float kAbsmaxFloor = 1e-5f;  // smallest absolute maximum used as a divisor
+constexpr int kNumSMsB200 = 148;
+
+#define SQ_CUDA_OK(expr)                              \
+    do {                                              \
+        cudaError_t e__ = (expr);                     \
+        if (e__ != cudaSuccess) return SQ_ERR_CUDA;   \
+    } while (0)
+
+inline sq_status launch_status() {
+    return cudaPeekAtLastError() == cudaSuccess ? SQ_OK : (cudaGetLastError(), SQ_ERR_CUDA);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int sm_count();  // SMs of the current device (cached)
+
+// ---------------------------------------------------------------------------------------
+// 16-bit activation types: unpack 8 values (one 16-byte vector) to fp32, exactly.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+struct Act;
+
+template <>
+struct Act<__half> {
+    using T2 = __half2;
+    static __device__ __forceinline__ float2 to_float2(uint32_t u) {
+        return __half22float2(*reinterpret_cast<const __half2*>(&u));
+    }
+    static __device__ __forceinline__ float to_float(__half v) { return __half2float(v); }
+    static __device__ __forceinline__ __half from_float(float v) { return __float2half_rn(v); }
+    // |a| and max are exact in fp16, so packed forms may be used for absolute maxima
+    static __device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t v) {
+        __half2 r = __hmax2(*reinterpret_cast<const __half2*>(&acc),
+                            __habs2(*reinterpret_cast<const __half2*>(&v)));
+        return *reinterpret_cast<uint32_t*>(&r);
+    }
+    static __device__ __forceinline__ float hmax_of2(uint32_t u) {
+        float2 f = to_float2(u);
+        return fmaxf(f.x, f.y);
+    }
+};
+
+template <>
+struct Act<__nv_bfloat16> {
+    using T2 = __nv_bfloat162;
+    static __device__ __forceinline__ float2 to_float2(uint32_t u) {
+        // bf16 -> fp32 is a 16-bit shift
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+    }
+    static __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+    static __device__ __forceinline__ __nv_bfloat16 from_float(float v) {
+        return __float2bfloat16_rn(v);
+    }
+    static __device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t v) {
+        __nv_bfloat162 r = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&acc),
+                                   __habs2(*reinterpret_cast<const __nv_bfloat162*>(&v)));
+        return *reinterpret_cast<uint32_t*>(&r);
+    }
+    static __device__ __forceinline__ float hmax_of2(uint32_t u) {
+        float2 f = to_float2(u);
+        return fmaxf(f.x, f.y);
+    }
+};
+
+template <typename T>
+__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
+    float2 a = Act<T>::to_float2(v.x), b = Act<T>::to_float2(v.y), c = Act<T>::to_float2(v.z),
+           d = Act<T>::to_float2(v.w);
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+    f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+}
+
+// ---------------------------------------------------------------------------------------
+// Eq. 1 pieces.  Every operation is an explicitly rounded fp32 intrinsic so that the
+// compiler cannot contract or reassociate: the codes are a bit-exact contract.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float step_size(float absmax) {
+    return __fdiv_rn(fmaxf(absmax, kAbsmaxFloor), 127.0f);
+}
+__device__ __forceinline__ float recip_step(float delta) { return __fdiv_rn(1.0f, delta); }
+
+__device__ __forceinline__ int quant_code(float v, float inv) {
+    int q = __float2int_rn(__fmul_rn(v, inv));  // round-half-to-even; saturates on overflow
+    return max(-127, min(127, q));
+}
+__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
+    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
+           ((uint32_t)(d & 0xff) << 24);
+}
+__device__ __forceinline__ uint2 quant8(const float (&f)[8], float inv) {
+    uint2 r;
+    r.x = pack4(quant_code(f[0], inv), quant_code(f[1], inv), quant_code(f[2], inv),
+                quant_code(f[3], inv));
+    r.y = pack4(quant_code(f[4], inv), quant_code(f[5], inv), quant_code(f[6], inv),
+                quant_code(f[7], inv));
+    return r;
+}
+
+// ---------------------------------------------------------------------------------------
+// Reductions
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+// Block-wide reductions; `red` is shared scratch of >= 33 floats.  All threads get the result.
+template <bool IS_MAX>
+__device__ __forceinline__ float block_reduce(float v, float* red) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    __syncthreads();  // protect `red` from the previous use
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        float t = lane < nwarp ? red[lane] : (IS_MAX ? 0.0f : 0.0f);
+        t = IS_MAX ? warp_max(t) : warp_sum(t);
+        if (lane == 0) red[32] = t;
+    }
+    __syncthreads();
+    return red[32];
+}
+
+// max for non-negative floats through their (order-preserving) bit patterns
+__device__ __forceinline__ void atomic_max_nonneg(float* addr, float v) {
+    atomicMax(reinterpret_cast<unsigned int*>(addr), __float_as_uint(v));
+}
+
+}  // namespace sq

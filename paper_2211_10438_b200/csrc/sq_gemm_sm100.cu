@@ -1,0 +1,579 @@
+// INT8 GEMM / batched matmul on the 5th-generation tensor cores (sm_100a):
+//   acc[t, o] = sum_j A[t, j] * B[o, j]      (Eq. 2's integer factor, INT32 exact)
+// with the dequantisation of Eq. 2 (+ bias, ReLU, re-quantisation) fused into the epilogue.
+//
+// One persistent CTA per SM, three roles:
+//   warp 4 (one lane) : TMA producer -- streams 128-byte-wide K slices of A and B into a
+//                       ring of shared-memory stages (128B swizzle), mbarrier-tracked;
+//   warp 5 (one lane) : issues tcgen05.mma.kind::i8 (128 x BLOCK_N x 32 per instruction),
+//                       accumulating in tensor memory (TMEM), two accumulator slots;
+//   warps 0-3         : epilogue -- tcgen05.ld the finished slot, dequantise, store, while
+//                       the MMA warp already fills the other slot with the next tile.
+// Every wait is bounded: on expiry the CTA records SQ_ERR_TIMEOUT in the status word, lets
+// outstanding copies land, frees its TMEM and returns.
+#include <cuda.h>
+
+#include "sq_common.cuh"
+#include "sq_kernels.h"
+
+namespace sq {
+
+namespace {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 128;  // INT8 elements = bytes: exactly one 128-byte swizzle row
+constexpr int UMMA_K = 32;    // K per tcgen05.mma for 8-bit operands
+constexpr int NUM_THREADS = 192;
+constexpr int EPI_THREADS = 128;
+constexpr uint32_t kWaitCycles = 2000000000u;  // ~1 s at B200 clocks
+
+template <int BLOCK_N>
+struct Cfg {
+    static constexpr int A_BYTES = BLOCK_M * BLOCK_K;
+    static constexpr int B_BYTES = BLOCK_N * BLOCK_K;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;  // 4 at BLOCK_N=256, 6 at 128
+    static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;  // two accumulator slots
+    static constexpr int EPI_FLOATS = 3 * BLOCK_N;  // w_scale, bias, requant per column
+    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + STAGES * STAGE_BYTES +
+                                      EPI_FLOATS * 4 + (2 * STAGES + 4) * 8 + 64;
+};
+
+struct Params {
+    int64_t M, N, K;
+    int heads, batch;
+    int num_m, num_n;
+    int64_t total_tiles;
+    int num_kb;
+    int b_is_kn;
+    // coordinate slot (1..3) of the row / head / batch dimension in each tensor map
+    int a_slot_row, a_slot_head, a_slot_batch;
+    int b_slot_row, b_slot_head, b_slot_batch;
+    const float* x_scale; int x_per_row;
+    const float* w_scale; int w_per_col;
+    float alpha;
+    const void* bias; int bias_is_bf16;
+    int relu;
+    const float* requant_mul; int requant_per_col;
+    float* row_absmax_out;
+    void* C; int out_dt;
+    int64_t c_stride_batch, c_stride_head, c_stride_row;
+    int c_vec_ok;  // 16-byte vector stores allowed
+    uint32_t* status;
+};
+
+// ------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag + the global status word)
+// if the phase does not complete within the cycle budget or another role already aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* status, uint32_t where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) {
+                *abort_flag = 1u;
+                atomicCAS(status, 0u, ((uint32_t)SQ_ERR_TIMEOUT) | (where << 8));
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0,
+                                            int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+
+__device__ __forceinline__ void tcgen05_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], INT8 x INT8 -> INT32
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                        uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// mbarrier arrives once every MMA issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void epi_bar_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+}
+
+// Shared-memory matrix descriptor (sm_100 format): 128-byte swizzle, 8-row groups 1024 B
+// apart.  For a K-major tile the rows are M/N indices; for the [K, N]-stored B operand
+// ("MN-major") the rows are K indices and the 128 contiguous bytes are N indices.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;  // leading-dimension byte offset
+    d |= (uint64_t)(1024u >> 4) << 32;               // stride-dimension byte offset: 8 rows
+    d |= (uint64_t)1 << 46;                          // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+    return d;
+}
+
+// Instruction descriptor of tcgen05.mma kind::i8: signed 8-bit A and B, INT32 D, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int block_n, int b_is_kn) {
+    return (2u << 4)                       // D format: S32
+           | (1u << 7)                     // A format: signed 8-bit
+           | (1u << 10)                    // B format: signed 8-bit
+           | (0u << 15)                    // A is K-major
+           | ((uint32_t)(b_is_kn ? 1 : 0) << 16)  // B major-ness
+           | ((uint32_t)(block_n >> 3) << 17)     // N / 8
+           | ((uint32_t)(BLOCK_M >> 4) << 24);    // M / 16
+}
+
+// tile id -> (batch*heads index, m tile, n tile).  Within one matrix, tiles are visited in
+// bands of 16 m-tiles so that the CTAs running at the same time share A and B tiles in L2.
+__device__ __forceinline__ void tile_coords(int64_t tile, const Params& p, int& bh, int& mi, int& ni) {
+    const int64_t per_mat = (int64_t)p.num_m * p.num_n;
+    bh = (int)(tile / per_mat);
+    const int64_t t = tile - (int64_t)bh * per_mat;
+    constexpr int G = 16;
+    const int64_t band_tiles = (int64_t)G * p.num_n;
+    const int band = (int)(t / band_tiles);
+    const int band_h = min(G, p.num_m - band * G);
+    const int64_t r = t - (int64_t)band * band_tiles;
+    mi = band * G + (int)(r % band_h);
+    ni = (int)(r / band_h);
+}
+
+template <typename OutT>
+__device__ __forceinline__ OutT cvt_out(float v);
+template <>
+__device__ __forceinline__ __half cvt_out<__half>(float v) { return __float2half_rn(v); }
+template <>
+__device__ __forceinline__ __nv_bfloat16 cvt_out<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// ------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------
+template <int BLOCK_N>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               const Params p) {
+    using C = Cfg<BLOCK_N>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                               ~(uintptr_t)1023);
+    uint8_t* stage_base = smem;
+    float* epi_f = reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_f + C::EPI_FLOATS);
+    uint64_t* empty_bar = full_bar + C::STAGES;
+    uint64_t* tmem_full = empty_bar + C::STAGES;
+    uint64_t* tmem_empty = tmem_full + 2;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    volatile uint32_t* abort_flag = tmem_holder + 1;
+    volatile uint32_t* epi_go = tmem_holder + 2;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 4 * 32) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(full_bar + s, 1);
+            mbar_init(empty_bar + s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(tmem_full + s, 1);
+            mbar_init(tmem_empty + s, EPI_THREADS);
+        }
+        *abort_flag = 0u;
+        *epi_go = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {  // whole warp allocates the tensor memory columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_holder)), "n"(C::TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 4) {
+        // ============================ TMA producer ============================
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                int bh, mi, ni;
+                tile_coords(tile, p, bh, mi, ni);
+                const int b = bh / p.heads, h = bh - b * p.heads;
+                int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
+                ca[p.a_slot_row] = mi * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
+                cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
+                    uint8_t* sa = stage_base + stage * C::STAGE_BYTES;
+                    uint8_t* sb = sa + C::A_BYTES;
+                    mbar_expect_tx(full_bar + stage, C::STAGE_BYTES);
+                    ca[0] = kb * BLOCK_K;
+                    tma_load_4d(sa, &tmap_a, full_bar + stage, ca[0], ca[1], ca[2], ca[3]);
+                    if (p.b_is_kn) {  // B stored [K, N]: x walks N, the row slot walks K
+                        cb[0] = ni * BLOCK_N;
+                        cb[p.b_slot_row] = kb * BLOCK_K;
+                    } else {
+                        cb[0] = kb * BLOCK_K;
+                        cb[p.b_slot_row] = ni * BLOCK_N;
+                    }
+                    tma_load_4d(sb, &tmap_b, full_bar + stage, cb[0], cb[1], cb[2], cb[3]);
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ============================ MMA issuer ==============================
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(BLOCK_N, p.b_is_kn);
+            // bytes between consecutive K=32 slices inside a stage
+            const uint32_t b_kstep = p.b_is_kn ? (uint32_t)(UMMA_K * 128) : (uint32_t)UMMA_K;
+            int stage = 0;
+            uint32_t phase = 0;
+            int slot = 0;
+            uint32_t slot_phase = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(slot * BLOCK_N);
+                for (int kb = 0; kb < p.num_kb; ++kb) {
+                    if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 3))) break;
+                    tcgen05_fence_after();
+                    const uint32_t sa = smem_u32(stage_base + stage * C::STAGE_BYTES);
+                    const uint32_t sb = sa + C::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                        const uint64_t adesc = make_smem_desc(sa + k * UMMA_K, 16);
+                        const uint64_t bdesc = make_smem_desc(sb + k * b_kstep, p.b_is_kn ? 16384u : 16u);
+                        umma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar + stage);  // frees the stage once these MMAs retire
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(tmem_full + slot);  // accumulator complete -> epilogue
+                slot ^= 1;
+                if (slot == 0) slot_phase ^= 1u;
+            }
+        }
+    } else {
+        // ============================ epilogue (warps 0-3) ====================
+        float* s_wscale = epi_f;
+        float* s_bias = epi_f + BLOCK_N;
+        float* s_requant = epi_f + 2 * BLOCK_N;
+        const int et = threadIdx.x;  // 0..127
+        int slot = 0;
+        uint32_t slot_phase = 0;
+        for (int64_t tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+            int bh, mi, ni;
+            tile_coords(tile, p, bh, mi, ni);
+            const int b = bh / p.heads, h = bh - b * p.heads;
+            const int64_t col0 = (int64_t)ni * BLOCK_N;
+            // stage this tile's per-column constants
+            for (int c = et; c < BLOCK_N; c += EPI_THREADS) {
+                const int64_t col = col0 + c;
+                const bool in = col < p.N;
+                float ws = 1.0f, bs = 0.0f, rq = 1.0f;
+                if (in) {
+                    if (p.w_scale) ws = __ldg(p.w_scale + (p.w_per_col ? col : 0));
+                    if (p.bias)
+                        bs = p.bias_is_bf16
+                                 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
+                                 : __half2float(static_cast<const __half*>(p.bias)[col]);
+                    if (p.requant_mul) rq = __ldg(p.requant_mul + (p.requant_per_col ? col : 0));
+                }
+                s_wscale[c] = ws; s_bias[c] = bs; s_requant[c] = rq;
+            }
+            if (et == 0)
+                *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 4) ? 1u : 0u;
+            epi_bar_sync();  // constants staged; verdict of the wait visible to all 128 threads
+            if (*epi_go == 0u) break;
+            tcgen05_fence_after();
+
+            const int64_t row = (int64_t)mi * BLOCK_M + warp * 32 + lane;
+            const bool row_ok = row < p.M;
+            float xs = p.alpha;
+            if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
+            float row_max = 0.0f;
+            const int64_t c_off = (int64_t)b * p.c_stride_batch + (int64_t)h * p.c_stride_head +
+                                  row * p.c_stride_row + col0;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(slot * BLOCK_N);
+
+#pragma unroll 1
+            for (int cc = 0; cc < BLOCK_N / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(taddr + cc * 32, r);
+                tmem_ld_wait();
+                const int64_t ncols = p.N - (col0 + cc * 32);  // valid columns in this chunk
+                if (!row_ok || ncols <= 0) continue;
+                const bool full = ncols >= 32;
+                if (p.out_dt == SQ_I32) {
+                    int32_t* out = static_cast<int32_t*>(p.C) + c_off + cc * 32;
+                    if (full && p.c_vec_ok) {
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            reinterpret_cast<uint4*>(out)[v] =
+                                make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < ncols) out[j] = (int32_t)r[j];
+                    }
+                    continue;
+                }
+                float y[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float sc = __fmul_rn(xs, s_wscale[cc * 32 + j]);
+                    float v = __fmaf_rn(__int2float_rn((int32_t)r[j]), sc, s_bias[cc * 32 + j]);
+                    if (p.relu) v = fmaxf(v, 0.0f);
+                    y[j] = v;
+                }
+                if (p.row_absmax_out) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < ncols) row_max = fmaxf(row_max, fabsf(y[j]));
+                }
+                if (p.out_dt == SQ_I8) {
+                    int8_t* out = static_cast<int8_t*>(p.C) + c_off + cc * 32;
+                    uint32_t q[8];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        q[v] = pack4(quant_code(y[4 * v], s_requant[cc * 32 + 4 * v]),
+                                     quant_code(y[4 * v + 1], s_requant[cc * 32 + 4 * v + 1]),
+                                     quant_code(y[4 * v + 2], s_requant[cc * 32 + 4 * v + 2]),
+                                     quant_code(y[4 * v + 3], s_requant[cc * 32 + 4 * v + 3]));
+                    if (full && p.c_vec_ok) {
+                        reinterpret_cast<uint4*>(out)[0] = make_uint4(q[0], q[1], q[2], q[3]);
+                        reinterpret_cast<uint4*>(out)[1] = make_uint4(q[4], q[5], q[6], q[7]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < ncols) out[j] = (int8_t)((q[j >> 2] >> (8 * (j & 3))) & 0xff);
+                    }
+                } else {
+                    uint32_t hw[16];
+                    if (p.out_dt == SQ_BF16) {
+#pragma unroll
+                        for (int v = 0; v < 16; ++v) {
+                            __nv_bfloat162 t = __halves2bfloat162(__float2bfloat16_rn(y[2 * v]),
+                                                                  __float2bfloat16_rn(y[2 * v + 1]));
+                            hw[v] = *reinterpret_cast<uint32_t*>(&t);
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 16; ++v) {
+                            __half2 t = __halves2half2(__float2half_rn(y[2 * v]), __float2half_rn(y[2 * v + 1]));
+                            hw[v] = *reinterpret_cast<uint32_t*>(&t);
+                        }
+                    }
+                    uint16_t* out = static_cast<uint16_t*>(p.C) + c_off + cc * 32;
+                    if (full && p.c_vec_ok) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            reinterpret_cast<uint4*>(out)[v] =
+                                make_uint4(hw[4 * v], hw[4 * v + 1], hw[4 * v + 2], hw[4 * v + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < ncols) out[j] = (uint16_t)((hw[j >> 1] >> (16 * (j & 1))) & 0xffff);
+                    }
+                }
+            }
+            if (p.row_absmax_out && row_ok) atomic_max_nonneg(p.row_absmax_out + row, row_max);
+            // accumulator slot drained: hand it back to the MMA warp
+            tcgen05_fence_before();
+            mbar_arrive(tmem_empty + slot);
+            slot ^= 1;
+            if (slot == 0) slot_phase ^= 1u;
+            epi_bar_sync();  // nobody still reads the staged constants when the next tile overwrites them
+        }
+    }
+
+    // ---------------------------------- teardown ------------------------------------
+    __syncwarp();
+    if (*abort_flag) __nanosleep(1000000);  // let copies / MMAs in flight land before freeing
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "n"(C::TMEM_COLS)
+                     : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Host side: tensor maps + launch
+// ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// Rank-4 INT8 tensor map over {inner (contiguous), row, head, batch} with the three outer
+// dimensions ordered by ascending stride; reports which coordinate slot each one got.
+// box_inner x box_rows bytes are copied per request (128-byte swizzle).
+bool make_map(CUtensorMap* map, const int8_t* base, int64_t inner, int64_t rows, int64_t heads,
+              int64_t batch, int64_t s_row, int64_t s_head, int64_t s_batch, int box_inner, int box_rows,
+              int* slot_row, int* slot_head, int* slot_batch) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    struct Dim { int64_t extent, stride; int box; int* slot; };
+    Dim d[3] = {{rows, s_row, box_rows, slot_row}, {heads, s_head, 1, slot_head}, {batch, s_batch, 1, slot_batch}};
+    // extent-1 dimensions never move the address: give them a harmless large stride so that
+    // the order below stays ascending
+    int64_t span = std::max<int64_t>(inner, 16);
+    for (auto& x : d) if (x.extent > 1) span = std::max(span, x.extent * x.stride);
+    span = (span + 15) / 16 * 16;
+    for (auto& x : d) if (x.extent <= 1) x.stride = span;
+    std::stable_sort(d, d + 3, [](const Dim& a, const Dim& b) { return a.stride < b.stride; });
+    cuuint64_t gdim[4] = {(cuuint64_t)inner, (cuuint64_t)d[0].extent, (cuuint64_t)d[1].extent, (cuuint64_t)d[2].extent};
+    cuuint64_t gstr[3] = {(cuuint64_t)d[0].stride, (cuuint64_t)d[1].stride, (cuuint64_t)d[2].stride};
+    cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)d[0].box, (cuuint32_t)d[1].box, (cuuint32_t)d[2].box};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    for (int i = 0; i < 3; ++i) *d[i].slot = i + 1;
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(base), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int BLOCK_N>
+sq_status launch(const GemmArgs& a, cudaStream_t st) {
+    using C = Cfg<BLOCK_N>;
+    Params p;
+    p.M = a.M; p.N = a.N; p.K = a.K;
+    p.heads = (int)a.heads; p.batch = (int)a.batch;
+    p.num_m = (int)((a.M + BLOCK_M - 1) / BLOCK_M);
+    p.num_n = (int)((a.N + BLOCK_N - 1) / BLOCK_N);
+    p.total_tiles = (int64_t)p.num_m * p.num_n * a.heads * a.batch;
+    p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
+    p.b_is_kn = a.b_is_kn;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, a.A, a.K, a.M, a.heads, a.batch, a.strideA[2], a.strideA[1], a.strideA[0], BLOCK_K,
+                  BLOCK_M, &p.a_slot_row, &p.a_slot_head, &p.a_slot_batch))
+        return SQ_ERR_CUDA;
+    const bool okb =
+        a.b_is_kn ? make_map(&mb, a.B, a.N, a.K, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
+                             BLOCK_N, BLOCK_K, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch)
+                  : make_map(&mb, a.B, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
+                             BLOCK_K, BLOCK_N, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch);
+    if (!okb) return SQ_ERR_CUDA;
+    p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
+    p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
+    p.alpha = a.alpha;
+    p.bias = a.bias; p.bias_is_bf16 = a.bias_dt == SQ_BF16;
+    p.relu = a.relu;
+    p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
+    p.row_absmax_out = a.row_absmax_out;
+    p.C = a.C; p.out_dt = (int)a.out_dt;
+    p.c_stride_batch = a.strideC[0]; p.c_stride_head = a.strideC[1]; p.c_stride_row = a.strideC[2];
+    const int esz = a.out_dt == SQ_I32 ? 4 : (a.out_dt == SQ_I8 ? 1 : 2);
+    const int vec_elems = 16 / esz;
+    p.c_vec_ok = aligned16(a.C) && a.strideC[0] % vec_elems == 0 && a.strideC[1] % vec_elems == 0 &&
+                 a.strideC[2] % vec_elems == 0;
+    p.status = a.status;
+
+    static bool attr_set[64] = {false};  // once per device
+    int dev = 0;
+    SQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        C::SMEM_BYTES));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    const int grid = (int)std::min<int64_t>(p.total_tiles, sm_count());
+    gemm_i8_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(ma, mb, p);
+    return launch_status();
+}
+
+}  // namespace
+
+sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
+    // [K, N]-stored B is limited to one 128-byte swizzle row of N per tile
+    if (a.b_is_kn || a.N <= 128) return launch<128>(a, st);
+    return launch<256>(a, st);
+}
+
+}  // namespace sq

@@ -1,0 +1,61 @@
+// Internal launch interface between the C-ABI layer (sq_api.cu) and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
+
+#include "../../include/sq.h"
+
+namespace sq {
+
+// How a row kernel obtains its step size.
+enum RowMode {
+    ROW_DYNAMIC = 0,          // Delta_row = absmax(row)/127, written to scale[row]
+    ROW_GIVEN_SCALE = 1,      // Delta = scale[0], an input (static)
+    ROW_FROM_ABSMAX_WORD = 2, // Delta = step_size(*absmax_word); scale[0] receives it
+    ROW_ABSMAX_ONLY = 3       // no codes: atomically fold the row's absmax into *absmax_word
+};
+
+// Workspace layout (bytes).  Word 0 is the sticky device status.
+constexpr size_t kWsStatusOff = 0;
+constexpr size_t kWsAbsmaxOff = 16;   // per-tensor dynamic absmax word
+constexpr size_t kWsHeader = 256;     // per-row LayerNorm statistics / split-K partials start here
+
+sq_status calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld, float* a,
+                       cudaStream_t st);
+sq_status smooth_scales(const float* ax, const float* aw, int64_t C, float alpha, float* s, float* s_inv,
+                        cudaStream_t st);
+sq_status fold_ln_weight(const void* g, const void* b, sq_dtype dt, const float* s, int64_t C,
+                         void* go, void* bo, cudaStream_t st);
+sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul,
+                    const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
+                    float* scale, float* absmax_word, float* stats, int stats_are_input,
+                    cudaStream_t st);
+sq_status softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_t S, int8_t* Pq,
+                          cudaStream_t st);
+sq_status residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out,
+                       cudaStream_t st);
+
+// Batched INT8 GEMM on the tensor cores (tcgen05, kind::i8) with the fused epilogue.
+struct GemmArgs {
+    const int8_t* A;      // [batch, heads, M, K]  K contiguous
+    const int8_t* B;      // [batch, heads, N, K] (K contiguous) or [batch, heads, K, N] (b_is_kn)
+    int64_t batch, heads, M, N, K;
+    int64_t strideA[3];   // batch, head, row (elements)
+    int64_t strideB[3];
+    int b_is_kn;
+    const float* x_scale; int x_per_row;     // Delta_x[t] or Delta_x
+    const float* w_scale; int w_per_col;     // Delta_w[o] or Delta_w; nullptr = 1
+    float alpha;                             // used when x_scale == nullptr
+    const void* bias; sq_dtype bias_dt;      // nullable
+    int relu;
+    const float* requant_mul; int requant_per_col;
+    float* row_absmax_out;
+    void* C; sq_dtype out_dt;
+    int64_t strideC[3];   // batch, head, row (elements)
+    uint32_t* status;     // device status word
+};
+sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
+
+}  // namespace sq

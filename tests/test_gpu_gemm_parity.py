@@ -1,0 +1,156 @@
+"""GPU parity, tensor-core stages: INT8 GEMM accumulators (bit-exact), the dequantisation epilogue
+(tolerance stated by the benchmark spec: 1e-3 relative or 2 ULP; the arithmetic is fully specified, so exact
+equality is also checked), re-quantised INT8 outputs (bit-exact) and the attention BMMs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import assert_fp_close, dev, host
+from paper_2211_10438_b200 import binding as sq
+from paper_2211_10438_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ws():
+    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 4096, 32768, 32768))
+    yield w
+    assert sq.device_status(w) == 0, "a device-side wait timed out"
+
+
+# (M, N, K): one tile, several tiles, ragged M / N / K tails, single row, N < 128, wide K
+SHAPES = [(16, 512, 512), (128, 256, 128), (128, 128, 128), (129, 257, 144), (300, 520, 272),
+          (1, 64, 16), (200, 72, 2048), (256, 1024, 5120), (77, 2000, 1040), (515, 384, 640)]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_gemm_accumulators_exact(ws, M, N, K):
+    Xq = synth.int8_tensor(20, 1, (M, K))
+    Wq = synth.int8_tensor(20, 2, (N, K))
+    acc = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, ws, out_dtype=torch.int32)
+    assert np.array_equal(host(acc), oracle.gemm_i32(Xq, Wq))
+    assert sq.device_status(ws) == 0
+
+
+def test_gemm_all_127_and_identity(ws):
+    M, N, K = 130, 260, 1024
+    ones = np.full((M, K), 127, np.int8)
+    acc = sq.sq_w8a8_gemm(dev(ones), dev(np.full((N, K), -127, np.int8)), None, None, ws, out_dtype=torch.int32)
+    assert np.all(host(acc) == -16129 * K)
+    Xq = synth.int8_tensor(20, 3, (M, 256))
+    eye = (127 * np.eye(256)).astype(np.int8)
+    acc = sq.sq_w8a8_gemm(dev(Xq), dev(eye), None, None, ws, out_dtype=torch.int32)
+    assert np.array_equal(host(acc), 127 * Xq.astype(np.int32))
+
+
+def test_gemm_run_to_run_identical(ws):
+    Xq, Wq = synth.int8_tensor(20, 4, (384, 2048)), synth.int8_tensor(20, 5, (1536, 2048))
+    a = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, ws, out_dtype=torch.int32)
+    b = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, ws, out_dtype=torch.int32)
+    assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M,N,K", [(16, 512, 512), (129, 257, 144), (300, 520, 272), (256, 1024, 5120)])
+@pytest.mark.parametrize("per_token,per_channel,use_bias,relu", [(True, True, True, False), (False, False, False, False),
+                                                                 (True, False, True, True), (False, True, True, True)])
+def test_gemm_dequant_epilogue(ws, dtype, M, N, K, per_token, per_channel, use_bias, relu):
+    Xq = synth.int8_tensor(21, 1, (M, K))
+    Wq = synth.int8_tensor(21, 2, (N, K))
+    rng = synth.rng_for(21, 3)
+    xs = (rng.uniform(0.01, 0.2, M if per_token else 1)).astype(np.float32)
+    wsc = (rng.uniform(1e-4, 1e-3, N if per_channel else 1)).astype(np.float32)
+    bias = synth.bias(21, 4, N, dtype, std=0.5) if use_bias else None
+    tdt = {"f16": torch.float16, "bf16": torch.bfloat16}[dtype]
+    y = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=None if bias is None else dev(bias, dtype),
+                        relu=relu, out_dtype=tdt)
+    _, want = oracle.w8a8_linear(Xq, xs, Wq, wsc, bias=bias, relu=relu, out_dtype=dtype)
+    got = host(y)
+    assert_fp_close(got, want, dtype, "dequant epilogue")
+    assert np.array_equal(got, want), "epilogue arithmetic is fully specified: expected identical values"
+
+
+@pytest.mark.parametrize("per_col", [False, True])
+def test_gemm_requant_and_row_absmax(ws, per_col):
+    M, N, K = 200, 328, 1024
+    Xq = synth.int8_tensor(22, 1, (M, K))
+    Wq = synth.int8_tensor(22, 2, (N, K))
+    rng = synth.rng_for(22, 3)
+    xs = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = synth.bias(22, 4, N, "f16", std=0.5)
+    r = rng.uniform(0.5, 2.0, N if per_col else 1).astype(np.float32)
+    rmax = torch.zeros(M, dtype=torch.float32, device="cuda")
+    q = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True,
+                        requant_mul=dev(r), row_absmax_out=rmax, out_dtype=torch.int8)
+    acc = oracle.gemm_i32(Xq, Wq)
+    y = oracle.dequant(acc, xs, wsc, bias, relu=True)
+    assert np.array_equal(host(q), oracle.requant(y, r))
+    assert np.array_equal(host(rmax), np.abs(y).max(1))
+
+
+def test_gemm_strided_output(ws):
+    M, N, K, ldy = 64, 200, 256, 264
+    Xq, Wq = synth.int8_tensor(23, 1, (M, K)), synth.int8_tensor(23, 2, (N, K))
+    xs = np.full(1, 0.05, np.float32)
+    wsc = np.full(1, 0.002, np.float32)
+    buf = torch.full((M, ldy), -7.0, dtype=torch.float16, device="cuda")
+    sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, out=buf[:, :N])
+    _, want = oracle.w8a8_linear(Xq, xs, Wq, wsc, out_dtype="f16")
+    got = host(buf)
+    assert np.array_equal(got[:, :N], want)
+    assert np.all(got[:, N:] == -7.0)  # nothing written beyond the N columns
+
+
+def _qkv_views(B, H, S, d, seed):
+    T = B * S
+    qkv = synth.int8_tensor(24, seed, (T, 3 * H * d))
+    return qkv
+
+
+@pytest.mark.parametrize("B,H,S,d", [(1, 2, 128, 128), (2, 3, 512, 128), (1, 1, 200, 64), (2, 2, 136, 128)])
+def test_bmm_qk_from_fused_qkv_buffer(ws, B, H, S, d):
+    qkv = _qkv_views(B, H, S, d, 1)
+    row = 3 * H * d
+    qkv_d = dev(qkv)
+    alpha = np.float32(0.0123)
+    out = torch.empty((B, H, S, S), dtype=torch.float16, device="cuda")
+    acc = torch.empty((B, H, S, S), dtype=torch.int32, device="cuda")
+    q_view = qkv_d.view(-1)  # Q at column 0, K at column H*d
+    k_view = qkv_d.view(-1)[H * d:]
+    for o in (out, acc):
+        sq.sq_w8a8_bmm(q_view, k_view, B, H, S, S, d, (S * row, d, row), (S * row, d, row), False, alpha, o,
+                       (H * S * S, S * S, S), ws)
+    q = qkv.reshape(B, S, 3, H, d)[:, :, 0].transpose(0, 2, 1, 3)
+    k = qkv.reshape(B, S, 3, H, d)[:, :, 1].transpose(0, 2, 1, 3)
+    want_acc, want = oracle.w8a8_bmm(np.ascontiguousarray(q), np.ascontiguousarray(k), alpha, out_dtype="f16")
+    assert np.array_equal(host(acc), want_acc)
+    assert_fp_close(host(out), want, "f16", "QK^T")
+    assert np.array_equal(host(out), want)
+
+
+@pytest.mark.parametrize("B,H,S,d", [(1, 2, 128, 128), (2, 3, 512, 128), (1, 2, 144, 64), (1, 1, 256, 16)])
+def test_bmm_pv_with_kn_operand(ws, B, H, S, d):
+    qkv = _qkv_views(B, H, S, d, 2)
+    row = 3 * H * d
+    P = synth.int8_tensor(24, 3, (B, H, S, S), lo=0, hi=127)
+    alpha = np.float32(3.1e-4)
+    r = np.array([1.7], np.float32)
+    qkv_d = dev(qkv)
+    v_view = qkv_d.view(-1)[2 * H * d:]
+    acc = torch.empty((B * S, H * d), dtype=torch.int32, device="cuda")
+    o8 = torch.empty((B * S, H * d), dtype=torch.int8, device="cuda")
+    of = torch.empty((B * S, H * d), dtype=torch.float16, device="cuda")
+    Pd = dev(P)
+    for o, rq in ((acc, None), (o8, dev(r)), (of, None)):
+        sq.sq_w8a8_bmm(Pd, v_view, B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True, alpha, o,
+                       (S * H * d, d, H * d), ws, requant_mul=rq)
+    v = np.ascontiguousarray(qkv.reshape(B, S, 3, H, d)[:, :, 2].transpose(0, 2, 1, 3))  # [B,H,S,d]
+    want_acc, want_q = oracle.w8a8_bmm(P, v, alpha, b_is_kn=True, requant_mul=r)
+    _, want_f = oracle.w8a8_bmm(P, v, alpha, b_is_kn=True, out_dtype="f16")
+    to_rows = lambda a: a.transpose(0, 2, 1, 3).reshape(B * S, H * d)  # [B,H,S,d] -> [B*S, H*d]
+    assert np.array_equal(host(acc), to_rows(want_acc))
+    assert np.array_equal(host(o8), to_rows(want_q))
+    assert np.array_equal(host(of), to_rows(want_f))
