@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the W8A8 hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A "step" is one pass of the runtime path over one batch at the OPT-13B-shaped prefill workload
+(hidden 5120, 2048 tokens, bf16, per-token dynamic activations / per-channel weights): fused
+LayerNorm+quantise -> QKV GEMM, quantise -> out-proj GEMM, fused LayerNorm+quantise -> FC1 GEMM
+(+ReLU), quantise -> FC2 GEMM; 8 kernel launches.  The offline transform (calibration absmax,
+Eq. 4, folding, weight quantisation) runs once in set-up and is reported under "rows".
+Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent replica of the
+workload (the path has no exchange step), value is the aggregate.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+WORKLOAD = 2  # OPT-13B-shaped prefill linears
+SAMPLE_ROWS_BASELINE = 256
+SAMPLE_ROWS_REFERENCE = 64
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_burst=d["bf16_tflops"],
+                    bf16_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_block(device, seed_offset=0):
+    """Seeded synthetic OPT-13B-shaped block: weights N(0, 0.02), outlier-channel activations."""
+    from paper_2211_10438_b200 import binding as sq
+    from paper_2211_10438_b200 import pipeline as pl
+    from paper_2211_10438_b200 import synth
+    wl = synth.WORKLOADS[WORKLOAD]
+    M, H = wl.tokens[0], wl.hidden
+    dt = torch.bfloat16
+    ch, fac = wl.outliers()
+    seed = synth.SEED_BASE + 256 * WORKLOAD + seed_offset
+    ws = sq.new_workspace(4096, device)
+    t0 = time.perf_counter()
+    prepared = {}
+    for i, l in enumerate(wl.linears):
+        W = pl.synth_device_weights(l.N, l.K, dt, seed + 10 + i, device=device)
+        b = (torch.randn(l.N, generator=torch.Generator(device=device).manual_seed(seed + 20 + i),
+                         device=device) * 0.01).to(dt)
+        calib = gamma = beta = None
+        if l.ln_input:
+            # calibration samples of this linear's input (the LayerNorm output) keep the outlier channels
+            calib = [pl.synth_device_activations(512, l.K, dt, ch, fac, seed + 30 + 4 * i + j, device) for j in range(4)]
+            g = torch.Generator(device=device).manual_seed(seed + 50 + i)
+            gamma = (1 + 0.1 * torch.randn(l.K, generator=g, device=device)).to(dt)
+            beta = (0.1 * torch.randn(l.K, generator=g, device=device)).to(dt)
+        prepared[l.name] = pl.prepare_linear(l.name, W, b, l.relu, calib, wl.alpha, "per_channel", ws, gamma, beta)
+        del W
+    torch.cuda.synchronize()
+    offline_s = time.perf_counter() - t0
+    block = pl.LinearBlock(prepared["qkv"], prepared["out_proj"], prepared["fc1"], prepared["fc2"], M, dt)
+    x_in = pl.synth_device_activations(M, H, dt, ch, fac, seed + 1, device)
+    attn_out = pl.synth_device_activations(M, H, dt, ch, fac, seed + 2, device)
+    return wl, block, x_in, attn_out, offline_s
+
+
+def timed_rows(device, peaks):
+    """Short isolated timings of the other rows of the path (each: 3 warm-ups, 10 timed launches)."""
+    from paper_2211_10438_b200 import binding as sq
+    from paper_2211_10438_b200 import pipeline as pl
+    rows = {}
+
+    def t(fn, n=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n * 1e-3
+
+    ws = sq.new_workspace(1 << 20, device)
+    # MT-NLG-shaped streaming rows (inputs 671 MB > L2)
+    M, C = 16384, 20480
+    x = torch.randn((M, C), device=device, dtype=torch.bfloat16)
+    x[:, ::200] *= 100
+    Xq = torch.empty((M, C), dtype=torch.int8, device=device)
+    xs = torch.empty(M, dtype=torch.float32, device=device)
+    g = torch.ones(C, dtype=torch.bfloat16, device=device)
+    b = torch.zeros(C, dtype=torch.bfloat16, device=device)
+    a = torch.zeros(C, dtype=torch.float32, device=device)
+    s = t(lambda: sq.sq_quant_act(x, "per_token", Xq=Xq, x_scale=xs, workspace=ws))
+    rows["quant_act_per_token_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    s = t(lambda: sq.sq_ln_quant(x, g, b, 1e-5, "per_token", Xq=Xq, x_scale=xs, workspace=ws))
+    rows["ln_quant_per_token_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    s = t(lambda: sq.sq_calib_absmax(x, a))
+    rows["calib_absmax_16384x20480"] = {"GB/s": 2 * M * C / s / 1e9, "frac_hbm": 2 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    del x, Xq
+    # decode-shaped GEMM, GPT-3 FC1, M = 16 (weights 604 MB > L2)
+    Md, N, K = 16, 49152, 12288
+    Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=device)
+    Xd = torch.randint(-127, 128, (Md, K), dtype=torch.int8, device=device)
+    xsd = torch.rand(Md, device=device) * 0.1
+    wsd = torch.rand(N, device=device) * 0.001
+    Y = torch.empty((Md, N), dtype=torch.bfloat16, device=device)
+    s = t(lambda: sq.sq_w8a8_gemm(Xd, Wq, xsd, wsd, ws, out=Y))
+    byts = N * K + Md * K + 2 * Md * N
+    rows["decode_gemm_M16_49152x12288"] = {"GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6}
+    del Wq
+    return rows
+
+
+def cpu_oracle_step(wl, host, rows):
+    """The oracle's version of one step on `rows` sampled tokens; returns integer ops done."""
+    import oracle
+    ops = 0
+    for name in ("qkv", "out_proj", "fc1", "fc2"):
+        Wq, ws, bias, relu = host[name]
+        if name == "qkv":
+            Xq, xs, _ = oracle.ln_quant(host["x_in"][:rows], host["g1"], host["b1"], 1e-5, "per_token")
+        elif name == "out_proj":
+            Xq, xs = oracle.quant_act(host["attn_out"][:rows], "per_token")
+        elif name == "fc1":
+            Xq, xs, _ = oracle.ln_quant(y, host["g2"], host["b2"], 1e-5, "per_token")
+        else:
+            Xq, xs = oracle.quant_act(y, "per_token")
+        _, y = oracle.w8a8_linear(Xq, xs, Wq, ws, bias=bias, relu=relu, out_dtype="bf16")
+        ops += 2 * rows * Wq.shape[0] * Wq.shape[1]
+    return ops
+
+
+def host_model(wl):
+    """Host-side synthetic block for the oracle legs (numpy; quantised with the oracle itself)."""
+    import oracle
+    from paper_2211_10438_b200 import synth
+    ch, fac = wl.outliers()
+    rows = max(SAMPLE_ROWS_BASELINE, SAMPLE_ROWS_REFERENCE)
+    host = {"x_in": synth.activations(WORKLOAD, 1, rows, wl.hidden, "bf16", ch, fac),
+            "attn_out": synth.activations(WORKLOAD, 2, rows, wl.hidden, "bf16", ch, fac)}
+    host["g1"], host["b1"] = synth.ln_params(WORKLOAD, 3, wl.hidden, "bf16")
+    host["g2"], host["b2"] = synth.ln_params(WORKLOAD, 4, wl.hidden, "bf16")
+    rng = np.random.default_rng(1234)
+    for i, l in enumerate(wl.linears):
+        # weights drawn directly as INT8 codes + scales: the oracle legs time the runtime path
+        Wq = rng.integers(-127, 128, (l.N, l.K), dtype=np.int8)
+        ws = rng.uniform(1e-4, 1e-3, l.N).astype(np.float32)
+        host[l.name] = (Wq, ws, synth.bias(WORKLOAD, 10 + i, l.N, "bf16"), l.relu)
+    return host
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2211_10438_b200 import synth
+    wl = synth.WORKLOADS[WORKLOAD]
+    host = host_model(wl)
+    rows = SAMPLE_ROWS_REFERENCE
+    for _ in range(args.warmup):
+        cpu_oracle_step(wl, host, rows)
+    t0 = time.perf_counter()
+    ops = 0
+    for _ in range(args.steps):
+        ops += cpu_oracle_step(wl, host, rows)
+    dt = time.perf_counter() - t0
+    val = ops / dt / 1e12
+    sample = "%d of %d tokens per step, all four linears at full width" % (rows, wl.tokens[0])
+    print(json.dumps({
+        "impl": "reference", "metric": "W8A8 linear-layer throughput (4 GEMMs + activation quantisation)",
+        "value": val, "unit": "TOPS", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "opt13b-prefill (config 2): hidden 5120, M=2048, bf16, per-token/per-channel",
+                   "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-rows", action="store_true", help="skip the isolated per-row timings")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 50 and args.warmup == 5:
+            args.steps, args.warmup = 10, 3
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2211_10438_b200 import binding as sq
+    sq.lib()  # fail loudly if the extension is missing
+    peaks = measured_peaks()
+    wl, block, x_in, attn_out, offline_s = build_block(device, seed_offset=1000 * rank)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v):
+        if world > 1:
+            t = torch.tensor([v], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return v
+
+    # ---------------- device-resident timing ----------------
+    for _ in range(args.warmup):
+        block.step(x_in, attn_out)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    block.gemm_events = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        block.step(x_in, attn_out)
+    e1.record()
+    barrier()
+    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+    clocks = sampler.stop()
+    gemm_s = {}
+    for name, (a, b) in block.gemm_events:
+        gemm_s.setdefault(name, []).append(a.elapsed_time(b) * 1e-3)
+    block.gemm_events = None
+    status = sq.device_status(block.ws)
+    if status != 0:
+        raise SystemExit("device status word = %d: a bounded wait expired" % status)
+    ops_step = block.gemm_ops()
+    value = world * ops_step * args.steps / elapsed / 1e12
+    gemm_total = sum(sum(v) for v in gemm_s.values())
+    achieved = ops_step * args.steps / gemm_total / 1e12
+    peak_tops = 2.0 * peaks["bf16_sustained"]
+
+    # ---------------- end to end: host buffers in, host result out ----------------
+    hx = x_in.cpu().pin_memory()
+    ha = attn_out.cpu().pin_memory()
+    hy = torch.empty((block.M, wl.hidden), dtype=torch.bfloat16).pin_memory()
+    dx, da = torch.empty_like(x_in), torch.empty_like(attn_out)
+
+    def e2e_step():
+        dx.copy_(hx, non_blocking=True)
+        da.copy_(ha, non_blocking=True)
+        y = block.step(dx, da)
+        hy.copy_(y, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+    e2e_value = world * ops_step * args.steps / e2e_elapsed / 1e12
+
+    out = {
+        "metric": "W8A8 linear-layer throughput (4 GEMMs + activation quantisation)",
+        "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": elapsed / args.steps * 1e3, "us_per_layer_linears": elapsed / args.steps * 1e6,
+        "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": "opt13b-prefill (config 2): hidden 5120, M=2048 tokens, bf16 activations, "
+                               "per-token dynamic act / per-channel weight INT8, alpha=0.5",
+                   "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "working set per step ~0.6 GB (314 MB INT8 weights + activations) exceeds the 126 MB L2; no flush"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_elapsed / args.steps * 1e3,
+                "h2d_bytes_per_step": int(hx.numel() * 2 + ha.numel() * 2), "d2h_bytes_per_step": int(hy.numel() * 2)},
+        "gpu_launches": block.launches_per_step * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak_tops,
+                     "unit": "TOP/s", "frac": achieved / peak_tops,
+                     "peak_source": "2 x %s bf16 sustained (%s); int8:bf16 nominal ratio 2" % (peaks["bf16_sustained"], peaks["source"]),
+                     "frac_of_2x_bf16_burst": achieved / (2 * peaks["bf16_burst"]), "frac_of_nominal_4500": achieved / 4500.0,
+                     "per_gemm_us": {k: statistics.mean(v) * 1e6 for k, v in gemm_s.items()},
+                     "traffic": None},
+        "offline_setup_s": offline_s,
+    }
+    if rank == 0 and world == 1 and not args.no_rows:
+        out["rows"] = timed_rows(device, peaks)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        host = host_model(wl)
+        t0 = time.perf_counter()
+        ops = cpu_oracle_step(wl, host, SAMPLE_ROWS_BASELINE)
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": ops / dt / 1e12, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
+                               "seconds": dt,
+                               "sample": "%d of %d tokens, all four linears at full width, one pass" % (SAMPLE_ROWS_BASELINE, wl.tokens[0])}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
