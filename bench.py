@@ -18,6 +18,7 @@ import os
 import statistics
 import subprocess
 import sys
+import threading
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -42,47 +43,57 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Polls SM clock and clock-event reasons through NVML (read-only) from a thread while the
+    timed region runs; CUDA_VISIBLE_DEVICES is honoured by matching the device's PCI bus id."""
 
-    def __init__(self, gpu_index):
-        self.idx, self.proc = gpu_index, None
+    def __init__(self, cuda_index):
+        self.cuda_index = cuda_index
+        self.samples, self.reasons, self.smax = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._err = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            bus = torch.cuda.get_device_properties(self.cuda_index).pci_bus_id
+            h = None
+            for i in range(nv.nvmlDeviceGetCount()):
+                hi = nv.nvmlDeviceGetHandleByIndex(i)
+                if nv.nvmlDeviceGetPciInfo(hi).bus == bus:
+                    h = hi
+                    break
+            if h is None:
+                h = nv.nvmlDeviceGetHandleByIndex(self.cuda_index)
+            self.smax = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                     nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                     nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                     nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
+            while not self._stop.is_set():
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                for bit, n in names.items():
+                    if mask & bit:
+                        self.reasons.add(n)
+                time.sleep(0.002)
+        except Exception as e:  # NVML missing: report it, never fail the bench
+            self._err = repr(e)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except OSError:
-            self.proc = None
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        time.sleep(0.02)  # first sample lands before the timed region opens
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-            out, _ = self.proc.communicate()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1]))
-                smax.append(float(f[2]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self._stop.set()
+        self._thread.join(timeout=5)
+        if self._err or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.smax, "samples": 0,
+                    "reasons": ["nvml unavailable: %s" % self._err]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.smax,
+                "samples": len(self.samples), "reasons": sorted(self.reasons)}
 
 
 def build_block(device, seed_offset=0):
