@@ -158,6 +158,35 @@ sq_status sq_ln_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const vo
                       const void* beta_hat, float eps, sq_act_gran g, int8_t* Xq, float* x_scale,
                       float* dbg_mean_rstd, void* workspace, size_t ws_bytes, void* stream);
 
+/* Largest token count sq_ln_quant_tensor_noalloc accepts: it sizes the built-in scratch. */
+#define SQ_NOALLOC_MAX_ROWS 16384
+
+/*
+ * The paper has no counterpart for this call; it exists for deployment.  Some callers cannot
+ * give the library a workspace because they cannot allocate device memory at all: a plug-in
+ * that is handed only its input and output buffers, code inside a serving engine whose memory
+ * arena is sized up front, a latency-critical loop in which cudaMalloc (which may synchronise
+ * the device) is forbidden.  For them this is sq_ln_quant in its per-tensor DYNAMIC mode
+ * (one step size from the whole [M, C] of the call, written to x_scale[0]) with the scratch it
+ * needs -- one running-maximum word and two floats of LayerNorm statistics per row -- held
+ * in a fixed array inside the library image instead of a caller workspace.  It calls no
+ * allocation routine of any kind.  Results are identical to sq_ln_quant(...,
+ * SQ_PER_TENSOR_DYNAMIC, ...).
+ *
+ *  - M <= SQ_NOALLOC_MAX_ROWS, else SQ_ERR_UNSUPPORTED (nothing is launched).  The array costs
+ *    about 128 KB of device memory on every GPU that loads the library, until process exit.
+ *  - The first call on each device looks up the array's device address (a host-side query,
+ *    made with that device current).  Make that first call outside any stream capture.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents; the
+ *    call re-zeroes what must start at zero.  Calls that can overlap on the GPU (different
+ *    streams without an ordering between them, or concurrent host threads) race on it and
+ *    give wrong step sizes: order them, or use sq_ln_quant with separate workspaces.
+ *  - Other arguments, alignment rules and arithmetic: exactly as sq_ln_quant.
+ */
+sq_status sq_ln_quant_tensor_noalloc(const void* X, sq_dtype dt, int64_t M, int64_t C,
+                                     const void* gamma_hat, const void* beta_hat, float eps,
+                                     int8_t* Xq, float* x_scale, void* stream);
+
 /*
  * The W8A8 linear layer, Eq. 2:
  *     acc[t, o] = sum_j Xq[t, j] * Wq[o, j]                         (INT32, exact)

@@ -20,10 +20,11 @@ SQ_W_PER_TENSOR, SQ_W_PER_CHANNEL = 0, 1
 SQ_EPI_NONE, SQ_EPI_RELU = 0, 1
 SQ_OP_QUANT_ACT, SQ_OP_LN_QUANT, SQ_OP_QUANT_WEIGHT, SQ_OP_GEMM, SQ_OP_BMM = 0, 1, 2, 3, 4
 SQ_MAX_K = 133144
+SQ_NOALLOC_MAX_ROWS = 16384
 
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
-           "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add"]
+           "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -65,6 +66,7 @@ def lib():
                                   f32, vp, vp, i32, c.POINTER(i64), vp, sz, vp]
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
         L.sq_residual_add.argtypes = [vp, vp, i32, i64, vp, vp]
+        L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = i32
         _lib = L
@@ -226,3 +228,18 @@ def sq_residual_add(a, b, out=None):
     _check(lib().sq_residual_add(_ptr(a), _ptr(b), _DT[a.dtype], a.numel(), _ptr(out), _stream()),
            "sq_residual_add")
     return out
+
+
+def sq_ln_quant_tensor_noalloc(X, gamma_hat, beta_hat, eps, Xq=None, x_scale=None):
+    """Per-tensor-dynamic fused LayerNorm+quantise for callers that cannot allocate a workspace:
+    the library's built-in scratch array is used instead.  At most SQ_NOALLOC_MAX_ROWS rows; calls
+    that overlap on the GPU race on that array.  Make the first call outside any stream capture."""
+    M, C = X.shape
+    if Xq is None:
+        Xq = torch.empty((M, C), dtype=torch.int8, device=X.device)
+    if x_scale is None:
+        x_scale = torch.empty(1, dtype=torch.float32, device=X.device)
+    _check(lib().sq_ln_quant_tensor_noalloc(_ptr(X), _DT[X.dtype], M, C, _ptr(gamma_hat), _ptr(beta_hat),
+                                            float(eps), _ptr(Xq), _ptr(x_scale), _stream()),
+           "sq_ln_quant_tensor_noalloc")
+    return Xq, x_scale
