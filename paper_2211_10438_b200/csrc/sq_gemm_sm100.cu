@@ -2,11 +2,16 @@
 //   acc[t, o] = sum_j A[t, j] * B[o, j]      (Eq. 2's integer factor, INT32 exact)
 // with the dequantisation of Eq. 2 (+ bias, ReLU, re-quantisation) fused into the epilogue.
 //
-// One persistent CTA per SM, three roles:
+// Persistent kernel, one CTA per SM.  With CG = 1 every CTA owns 128 x BLOCK_N tiles; with
+// CG = 2 (tcgen05 cta_group::2) the two CTAs of a cluster own a 256 x BLOCK_N tile together:
+// each loads its own 128 rows of A and its own half of B, the even CTA issues one MMA for
+// both, and each CTA's tensor memory receives its 128 rows of the accumulator.  Pairing cuts
+// the shared-memory fill traffic per MMA by a third; no TMA multicast is involved.
+// Roles inside a CTA:
 //   warp 4 (one lane) : TMA producer -- streams 128-byte-wide K slices of A and B into a
 //                       ring of shared-memory stages (128B swizzle), mbarrier-tracked;
-//   warp 5 (one lane) : issues tcgen05.mma.kind::i8 (128 x BLOCK_N x 32 per instruction),
-//                       accumulating in tensor memory (TMEM), two accumulator slots;
+//   warp 5 (one lane) : issues tcgen05.mma.kind::i8 (K = 32 per instruction), accumulating
+//                       in tensor memory (TMEM), two accumulator slots;
 //   warps 0-3         : epilogue -- tcgen05.ld the finished slot, dequantise, store, while
 //                       the MMA warp already fills the other slot with the next tile.
 // Every wait is bounded: on expiry the CTA records SQ_ERR_TIMEOUT in the status word, lets
@@ -20,29 +25,38 @@ namespace sq {
 
 namespace {
 
-constexpr int BLOCK_M = 128;
+constexpr int BLOCK_M = 128;  // accumulator rows per CTA (TMEM lanes)
 constexpr int BLOCK_K = 128;  // INT8 elements = bytes: exactly one 128-byte swizzle row
 constexpr int UMMA_K = 32;    // K per tcgen05.mma for 8-bit operands
 constexpr int NUM_THREADS = 192;
 constexpr int EPI_THREADS = 128;
 constexpr uint32_t kWaitCycles = 2000000000u;  // ~1 s at B200 clocks
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu; // clears the CTA-rank bit of a shared::cluster address:
+                                               // the same offset in the EVEN CTA of the pair
 
-template <int BLOCK_N>
+template <int BLOCK_N, int CG>
 struct Cfg {
+    static constexpr int B_ROWS = BLOCK_N / CG;  // rows of B this CTA loads per K slice
     static constexpr int A_BYTES = BLOCK_M * BLOCK_K;
-    static constexpr int B_BYTES = BLOCK_N * BLOCK_K;
+    static constexpr int B_BYTES = B_ROWS * BLOCK_K;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;  // 4 at BLOCK_N=256, 6 at 128
-    static constexpr int TMEM_COLS = 2 * BLOCK_N < 32 ? 32 : 2 * BLOCK_N;  // two accumulator slots
+    static constexpr int STAGING_BYTES = 4 * 32 * 128;  // per epilogue warp: 32 rows x 128 bytes
+    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+    // column stride between the two accumulator slots (power of two keeps the allocation simple)
+    static constexpr int SLOT_COLS = BLOCK_N <= 32 ? 32 : BLOCK_N <= 64 ? 64 : BLOCK_N <= 128 ? 128 : 256;
+    static constexpr int TMEM_COLS = 2 * SLOT_COLS;
     static constexpr int EPI_FLOATS = 3 * BLOCK_N;  // w_scale, bias, requant per column
-    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + STAGES * STAGE_BYTES +
+    static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + STAGES * STAGE_BYTES + STAGING_BYTES +
                                       EPI_FLOATS * 4 + (2 * STAGES + 4) * 8 + 64;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(BLOCK_N % (16 * CG) == 0 && BLOCK_N <= 256, "MMA N constraint");
+    static_assert(B_ROWS % 8 == 0, "B tile must be whole 8-row swizzle groups");
 };
 
 struct Params {
     int64_t M, N, K;
     int heads, batch;
-    int num_m, num_n;
+    int num_m, num_n;  // tiles per matrix (num_m counts tiles of 128*CG rows)
     int64_t total_tiles;
     int num_kb;
     int b_is_kn;
@@ -58,7 +72,8 @@ struct Params {
     float* row_absmax_out;
     void* C; int out_dt;
     int64_t c_stride_batch, c_stride_head, c_stride_row;
-    int c_vec_ok;  // 16-byte vector stores allowed
+    int c_tma;  // C leaves through TMA stores (needs 16-byte aligned base and strides)
+    int c_slot_row, c_slot_head, c_slot_batch;
     uint32_t* status;
 };
 
@@ -67,6 +82,15 @@ struct Params {
 // ------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
@@ -78,6 +102,12 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// arrive on the barrier at the same shared-memory offset in the even CTA of the pair
+__device__ __forceinline__ void mbar_arrive_even_cta(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];"
+                 ::"r"(smem_u32(bar) & kPeerBitMask)
+                 : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -110,13 +140,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return true;
 }
 
+// Tiled TMA load of one box into this CTA's shared memory.  With CG = 2 the completion is
+// signalled on the EVEN CTA's barrier (same offset), which gathers both CTAs' bytes.
+template <int CG>
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0,
                                             int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
+    if (CG == 1) {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+            ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar) & kPeerBitMask), "r"(c0), "r"(c1), "r"(c2),
+            "r"(c3)
+            : "memory");
+    }
 }
 
 __device__ __forceinline__ void tcgen05_fence_before() {
@@ -126,20 +168,40 @@ __device__ __forceinline__ void tcgen05_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
 // D[tmem] (+)= A[smem] * B[smem], INT8 x INT8 -> INT32
+template <int CG>
 __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                         uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
-// mbarrier arrives once every MMA issued so far by this thread has completed
+// The barrier (in every CTA of the group, same offset) receives one arrival once every MMA
+// issued so far by this thread has completed.
+template <int CG>
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(smem_u32(bar))
-                 : "memory");
+    if (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     ::"r"(smem_u32(bar))
+                     : "memory");
+    } else {
+        const uint16_t mask = 3;  // both CTAs of the pair
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+            ::"r"(smem_u32(bar)), "h"(mask)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -160,6 +222,25 @@ __device__ __forceinline__ void tmem_ld_wait() {
 __device__ __forceinline__ void epi_bar_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
 }
+template <int CG>
+__device__ __forceinline__ void tmem_alloc(uint32_t* holder, uint32_t cols) {
+    if (CG == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(holder)), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(holder)), "r"(cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+}
+template <int CG>
+__device__ __forceinline__ void tmem_dealloc(uint32_t base, uint32_t cols) {
+    if (CG == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+    else
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+}
 
 // Shared-memory matrix descriptor (sm_100 format): 128-byte swizzle, 8-row groups 1024 B
 // apart.  For a K-major tile the rows are M/N indices; for the [K, N]-stored B operand
@@ -174,24 +255,24 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
     return d;
 }
 
-// Instruction descriptor of tcgen05.mma kind::i8: signed 8-bit A and B, INT32 D, M = 128.
-__host__ __device__ constexpr uint32_t make_idesc(int block_n, int b_is_kn) {
+// Instruction descriptor of tcgen05.mma kind::i8: signed 8-bit A and B, INT32 D.
+__host__ __device__ constexpr uint32_t make_idesc(int mma_m, int mma_n, int b_is_kn) {
     return (2u << 4)                       // D format: S32
            | (1u << 7)                     // A format: signed 8-bit
            | (1u << 10)                    // B format: signed 8-bit
            | (0u << 15)                    // A is K-major
            | ((uint32_t)(b_is_kn ? 1 : 0) << 16)  // B major-ness
-           | ((uint32_t)(block_n >> 3) << 17)     // N / 8
-           | ((uint32_t)(BLOCK_M >> 4) << 24);    // M / 16
+           | ((uint32_t)(mma_n >> 3) << 17)       // N / 8
+           | ((uint32_t)(mma_m >> 4) << 24);      // M / 16
 }
 
 // tile id -> (batch*heads index, m tile, n tile).  Within one matrix, tiles are visited in
-// bands of 16 m-tiles so that the CTAs running at the same time share A and B tiles in L2.
+// bands of G m-tiles so that the CTAs running at the same time share A and B tiles in L2.
 __device__ __forceinline__ void tile_coords(int64_t tile, const Params& p, int& bh, int& mi, int& ni) {
     const int64_t per_mat = (int64_t)p.num_m * p.num_n;
     bh = (int)(tile / per_mat);
     const int64_t t = tile - (int64_t)bh * per_mat;
-    constexpr int G = 16;
+    constexpr int G = 8;
     const int64_t band_tiles = (int64_t)G * p.num_n;
     const int band = (int)(t / band_tiles);
     const int band_h = min(G, p.num_m - band * G);
@@ -200,26 +281,160 @@ __device__ __forceinline__ void tile_coords(int64_t tile, const Params& p, int& 
     ni = (int)(r / band_h);
 }
 
-template <typename OutT>
-__device__ __forceinline__ OutT cvt_out(float v);
-template <>
-__device__ __forceinline__ __half cvt_out<__half>(float v) { return __float2half_rn(v); }
-template <>
-__device__ __forceinline__ __nv_bfloat16 cvt_out<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+// ------------------------------------------------------------------------------------
+// Epilogue of one 128 x BLOCK_N accumulator slot: Eq. 2 and the output conversions.
+// Called by the 128 epilogue threads; thread = one accumulator row (TMEM lane).
+// Output leaves through shared memory: each warp stages 32 rows x 128 bytes (128B swizzle,
+// conflict-free 16-byte writes) and one lane issues a TMA store, which also clips the M and N
+// tails.  If C is not 16-byte aligned the rows are written directly instead.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void* src, int c0, int c1, int c2,
+                                             int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(map), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() {  // staging buffer may be overwritten again
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() {
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+template <int BLOCK_N>
+__device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
+                                              uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
+                                              int h, int64_t c_off, const float* s_wscale,
+                                              const float* s_bias, const float* s_requant, int lane) {
+    const bool row_ok = row < p.M;
+    float xs = p.alpha;
+    if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
+    float row_max = 0.0f;
+    // 32-column chunks per 128-byte staging row: 1 (int32), 2 (fp16/bf16), 4 (int8)
+    const int chunks_per_store = p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2);
+    const int pieces = 8 / chunks_per_store;  // 16-byte pieces one chunk contributes to the row
+    int cc_coord[4] = {0, 0, 0, 0};
+    cc_coord[p.c_slot_row] = row0_warp; cc_coord[p.c_slot_head] = h; cc_coord[p.c_slot_batch] = b;
+#pragma unroll 1
+    for (int cc = 0; cc < BLOCK_N / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld32(taddr + cc * 32, r);  // warp-collective: executed by every lane
+        tmem_ld_wait();
+        const int64_t ncols = p.N - (col0 + cc * 32);  // valid columns in this chunk
+#ifdef SQ_EXP_NO_STORE  // measurement build: drain TMEM but write nothing
+        if (r[0] != 0x7fffffffu) continue;
+#endif
+        // ---- Eq. 2 on the chunk; w[] receives the packed output words ----
+        uint32_t w[32];
+        int nwords;
+        if (p.out_dt == SQ_I32) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) w[j] = r[j];
+            nwords = 32;
+        } else {
+            float y[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float sc = __fmul_rn(xs, s_wscale[cc * 32 + j]);
+                float v = __fmaf_rn(__int2float_rn((int32_t)r[j]), sc, s_bias[cc * 32 + j]);
+                if (p.relu) v = fmaxf(v, 0.0f);
+                y[j] = v;
+            }
+            if (p.row_absmax_out) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (j < ncols) row_max = fmaxf(row_max, fabsf(y[j]));
+            }
+            if (p.out_dt == SQ_I8) {
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                    w[v] = pack4(quant_code(y[4 * v], s_requant[cc * 32 + 4 * v]),
+                                 quant_code(y[4 * v + 1], s_requant[cc * 32 + 4 * v + 1]),
+                                 quant_code(y[4 * v + 2], s_requant[cc * 32 + 4 * v + 2]),
+                                 quant_code(y[4 * v + 3], s_requant[cc * 32 + 4 * v + 3]));
+                nwords = 8;
+            } else if (p.out_dt == SQ_BF16) {
+#pragma unroll
+                for (int v = 0; v < 16; ++v) {
+                    __nv_bfloat162 t = __halves2bfloat162(__float2bfloat16_rn(y[2 * v]), __float2bfloat16_rn(y[2 * v + 1]));
+                    w[v] = *reinterpret_cast<uint32_t*>(&t);
+                }
+                nwords = 16;
+            } else {
+#pragma unroll
+                for (int v = 0; v < 16; ++v) {
+                    __half2 t = __halves2half2(__float2half_rn(y[2 * v]), __float2half_rn(y[2 * v + 1]));
+                    w[v] = *reinterpret_cast<uint32_t*>(&t);
+                }
+                nwords = 16;
+            }
+        }
+        if (p.c_tma) {
+            // ---- staged TMA store: lane = row of the 32 x 128-byte staging tile ----
+            const int sub = cc % chunks_per_store;
+            if (sub == 0) {  // previous store must have finished READING the staging tile
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+            }
+            uint8_t* srow = stg + lane * 128;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                if (v < pieces) {
+                    const int j = sub * pieces + v;  // 16-byte piece index inside the 128-byte row
+                    *reinterpret_cast<uint4*>(srow + ((j ^ (lane & 7)) << 4)) =
+                        make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+                }
+            }
+            if (sub == chunks_per_store - 1) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy
+                __syncwarp();
+                const int64_t gcol = col0 + (int64_t)(cc - sub) * 32;  // first column of the staged group
+                if (lane == 0 && gcol < p.N && row0_warp < p.M) {
+                    cc_coord[0] = (int)gcol;
+                    tma_store_4d(tmap_c, stg, cc_coord[0], cc_coord[1], cc_coord[2], cc_coord[3]);
+                }
+            }
+            continue;
+        }
+        // ---- direct stores (unaligned C) ----
+        if (!row_ok || ncols <= 0) continue;
+        const bool full = ncols >= 32;
+        if (p.out_dt == SQ_I32) {
+            int32_t* out = static_cast<int32_t*>(p.C) + c_off + cc * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (full || j < ncols) out[j] = (int32_t)w[j];
+        } else if (p.out_dt == SQ_I8) {
+            int8_t* out = static_cast<int8_t*>(p.C) + c_off + cc * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (full || j < ncols) out[j] = (int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xff);
+        } else {
+            uint16_t* out = static_cast<uint16_t*>(p.C) + c_off + cc * 32;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (full || j < ncols) out[j] = (uint16_t)((w[j >> 1] >> (16 * (j & 1))) & 0xffff);
+        }
+        (void)nwords;
+    }
+    if (p.row_absmax_out && row_ok) atomic_max_nonneg(p.row_absmax_out + row, row_max);
+}
 
 // ------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N>
+template <int BLOCK_N, int CG>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const Params p) {
-    using C = Cfg<BLOCK_N>;
+               const __grid_constant__ CUtensorMap tmap_c, const Params p) {
+    using C = Cfg<BLOCK_N, CG>;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                               ~(uintptr_t)1023);
+    // identical layout in both CTAs of a pair (the MMA addresses both with one descriptor)
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_base = smem;
-    float* epi_f = reinterpret_cast<float*>(smem + C::STAGES * C::STAGE_BYTES);
+    uint8_t* staging = smem + C::STAGES * C::STAGE_BYTES;  // 1024-byte aligned: swizzle pattern matches TMA's
+    float* epi_f = reinterpret_cast<float*>(staging + C::STAGING_BYTES);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_f + C::EPI_FLOATS);
     uint64_t* empty_bar = full_bar + C::STAGES;
     uint64_t* tmem_full = empty_bar + C::STAGES;
@@ -229,31 +444,29 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     volatile uint32_t* epi_go = tmem_holder + 2;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = CG == 1 ? 0 : (int)cluster_ctarank();  // 0 = even CTA: issues the MMAs
+    const int64_t first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
     if (threadIdx.x == 4 * 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+        if (p.c_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_c) : "memory");
         for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(full_bar + s, 1);
-            mbar_init(empty_bar + s, 1);
+            mbar_init(full_bar + s, 1);   // the even CTA's arrive.expect_tx
+            mbar_init(empty_bar + s, 1);  // one tcgen05.commit
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(tmem_full + s, 1);
-            mbar_init(tmem_empty + s, EPI_THREADS);
+            mbar_init(tmem_empty + s, EPI_THREADS * CG);  // epilogue threads of the whole group
         }
         *abort_flag = 0u;
         *epi_go = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 5) {  // whole warp allocates the tensor memory columns
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_holder)), "n"(C::TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 5) tmem_alloc<CG>(tmem_holder, C::TMEM_COLS);  // whole warp (in both CTAs of a pair)
     tcgen05_fence_before();
-    __syncthreads();
+    if (CG == 1) __syncthreads(); else cluster_sync_all();  // peers' barriers are live before any remote signal
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
@@ -263,36 +476,40 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 const int b = bh / p.heads, h = bh - b * p.heads;
                 int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
-                ca[p.a_slot_row] = mi * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
+                ca[p.a_slot_row] = (mi * CG + rank) * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
                 cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
+                const int b_row0 = ni * BLOCK_N + rank * C::B_ROWS;  // this CTA's share of the B tile
                 for (int kb = 0; kb < p.num_kb; ++kb) {
+#ifdef SQ_EXP_MMA_ONLY  // measurement build: no loads at all (MMA issue ceiling)
+                    break;
+#endif
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
                     uint8_t* sa = stage_base + stage * C::STAGE_BYTES;
                     uint8_t* sb = sa + C::A_BYTES;
-                    mbar_expect_tx(full_bar + stage, C::STAGE_BYTES);
+                    if (rank == 0) mbar_expect_tx(full_bar + stage, C::STAGE_BYTES * CG);
                     ca[0] = kb * BLOCK_K;
-                    tma_load_4d(sa, &tmap_a, full_bar + stage, ca[0], ca[1], ca[2], ca[3]);
+                    tma_load_4d<CG>(sa, &tmap_a, full_bar + stage, ca[0], ca[1], ca[2], ca[3]);
                     if (p.b_is_kn) {  // B stored [K, N]: x walks N, the row slot walks K
-                        cb[0] = ni * BLOCK_N;
+                        cb[0] = b_row0;
                         cb[p.b_slot_row] = kb * BLOCK_K;
                     } else {
                         cb[0] = kb * BLOCK_K;
-                        cb[p.b_slot_row] = ni * BLOCK_N;
+                        cb[p.b_slot_row] = b_row0;
                     }
-                    tma_load_4d(sb, &tmap_b, full_bar + stage, cb[0], cb[1], cb[2], cb[3]);
+                    tma_load_4d<CG>(sb, &tmap_b, full_bar + stage, cb[0], cb[1], cb[2], cb[3]);
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 5) {
-        // ============================ MMA issuer ==============================
-        if (lane == 0) {
-            const uint32_t idesc = make_idesc(BLOCK_N, p.b_is_kn);
+        // ============================ MMA issuer (even CTA only) ==============
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc(BLOCK_M * CG, BLOCK_N, p.b_is_kn);
             // bytes between consecutive K=32 slices inside a stage
             const uint32_t b_kstep = p.b_is_kn ? (uint32_t)(UMMA_K * 128) : (uint32_t)UMMA_K;
             int stage = 0;
@@ -300,12 +517,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
                 tcgen05_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(slot * BLOCK_N);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
+#ifndef SQ_EXP_MMA_ONLY
                     if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 3))) break;
+#endif
                     tcgen05_fence_after();
                     const uint32_t sa = smem_u32(stage_base + stage * C::STAGE_BYTES);
                     const uint32_t sb = sa + C::A_BYTES;
@@ -313,13 +532,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         const uint64_t adesc = make_smem_desc(sa + k * UMMA_K, 16);
                         const uint64_t bdesc = make_smem_desc(sb + k * b_kstep, p.b_is_kn ? 16384u : 16u);
-                        umma_i8(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
-                    umma_commit(empty_bar + stage);  // frees the stage once these MMAs retire
+                    umma_commit<CG>(empty_bar + stage);  // frees the stage (in both CTAs) once these MMAs retire
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(tmem_full + slot);  // accumulator complete -> epilogue
+                umma_commit<CG>(tmem_full + slot);  // accumulator complete -> epilogue (of both CTAs)
                 slot ^= 1;
                 if (slot == 0) slot_phase ^= 1u;
             }
@@ -332,7 +551,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int et = threadIdx.x;  // 0..127
         int slot = 0;
         uint32_t slot_phase = 0;
-        for (int64_t tile = blockIdx.x; tile < p.total_tiles; tile += gridDim.x) {
+        for (int64_t tile = first_tile; tile < p.total_tiles; tile += tile_step) {
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
             const int b = bh / p.heads, h = bh - b * p.heads;
@@ -345,9 +564,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (in) {
                     if (p.w_scale) ws = __ldg(p.w_scale + (p.w_per_col ? col : 0));
                     if (p.bias)
-                        bs = p.bias_is_bf16
-                                 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
-                                 : __half2float(static_cast<const __half*>(p.bias)[col]);
+                        bs = p.bias_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
+                                            : __half2float(static_cast<const __half*>(p.bias)[col]);
                     if (p.requant_mul) rq = __ldg(p.requant_mul + (p.requant_per_col ? col : 0));
                 }
                 s_wscale[c] = ws; s_bias[c] = bs; s_requant[c] = rq;
@@ -358,116 +576,32 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             if (*epi_go == 0u) break;
             tcgen05_fence_after();
 
-            const int64_t row = (int64_t)mi * BLOCK_M + warp * 32 + lane;
-            const bool row_ok = row < p.M;
-            float xs = p.alpha;
-            if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
-            float row_max = 0.0f;
+            const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + warp * 32 + lane;
             const int64_t c_off = (int64_t)b * p.c_stride_batch + (int64_t)h * p.c_stride_head +
                                   row * p.c_stride_row + col0;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(slot * BLOCK_N);
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS);
+            const int row0_warp = (mi * CG + rank) * BLOCK_M + warp * 32;
+            epilogue_slot<BLOCK_N>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
+                                   c_off, s_wscale, s_bias, s_requant, lane);
 
-#pragma unroll 1
-            for (int cc = 0; cc < BLOCK_N / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(taddr + cc * 32, r);
-                tmem_ld_wait();
-                const int64_t ncols = p.N - (col0 + cc * 32);  // valid columns in this chunk
-                if (!row_ok || ncols <= 0) continue;
-                const bool full = ncols >= 32;
-                if (p.out_dt == SQ_I32) {
-                    int32_t* out = static_cast<int32_t*>(p.C) + c_off + cc * 32;
-                    if (full && p.c_vec_ok) {
-#pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            reinterpret_cast<uint4*>(out)[v] =
-                                make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < ncols) out[j] = (int32_t)r[j];
-                    }
-                    continue;
-                }
-                float y[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const float sc = __fmul_rn(xs, s_wscale[cc * 32 + j]);
-                    float v = __fmaf_rn(__int2float_rn((int32_t)r[j]), sc, s_bias[cc * 32 + j]);
-                    if (p.relu) v = fmaxf(v, 0.0f);
-                    y[j] = v;
-                }
-                if (p.row_absmax_out) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (j < ncols) row_max = fmaxf(row_max, fabsf(y[j]));
-                }
-                if (p.out_dt == SQ_I8) {
-                    int8_t* out = static_cast<int8_t*>(p.C) + c_off + cc * 32;
-                    uint32_t q[8];
-#pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        q[v] = pack4(quant_code(y[4 * v], s_requant[cc * 32 + 4 * v]),
-                                     quant_code(y[4 * v + 1], s_requant[cc * 32 + 4 * v + 1]),
-                                     quant_code(y[4 * v + 2], s_requant[cc * 32 + 4 * v + 2]),
-                                     quant_code(y[4 * v + 3], s_requant[cc * 32 + 4 * v + 3]));
-                    if (full && p.c_vec_ok) {
-                        reinterpret_cast<uint4*>(out)[0] = make_uint4(q[0], q[1], q[2], q[3]);
-                        reinterpret_cast<uint4*>(out)[1] = make_uint4(q[4], q[5], q[6], q[7]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < ncols) out[j] = (int8_t)((q[j >> 2] >> (8 * (j & 3))) & 0xff);
-                    }
-                } else {
-                    uint32_t hw[16];
-                    if (p.out_dt == SQ_BF16) {
-#pragma unroll
-                        for (int v = 0; v < 16; ++v) {
-                            __nv_bfloat162 t = __halves2bfloat162(__float2bfloat16_rn(y[2 * v]),
-                                                                  __float2bfloat16_rn(y[2 * v + 1]));
-                            hw[v] = *reinterpret_cast<uint32_t*>(&t);
-                        }
-                    } else {
-#pragma unroll
-                        for (int v = 0; v < 16; ++v) {
-                            __half2 t = __halves2half2(__float2half_rn(y[2 * v]), __float2half_rn(y[2 * v + 1]));
-                            hw[v] = *reinterpret_cast<uint32_t*>(&t);
-                        }
-                    }
-                    uint16_t* out = static_cast<uint16_t*>(p.C) + c_off + cc * 32;
-                    if (full && p.c_vec_ok) {
-#pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            reinterpret_cast<uint4*>(out)[v] =
-                                make_uint4(hw[4 * v], hw[4 * v + 1], hw[4 * v + 2], hw[4 * v + 3]);
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < ncols) out[j] = (uint16_t)((hw[j >> 1] >> (16 * (j & 1))) & 0xffff);
-                    }
-                }
-            }
-            if (p.row_absmax_out && row_ok) atomic_max_nonneg(p.row_absmax_out + row, row_max);
-            // accumulator slot drained: hand it back to the MMA warp
+            // accumulator slot drained: hand it back to the MMA warp (in the even CTA)
             tcgen05_fence_before();
-            mbar_arrive(tmem_empty + slot);
+            if (CG == 1) mbar_arrive(tmem_empty + slot); else mbar_arrive_even_cta(tmem_empty + slot);
             slot ^= 1;
             if (slot == 0) slot_phase ^= 1u;
             epi_bar_sync();  // nobody still reads the staged constants when the next tile overwrites them
         }
+        if (p.c_tma && lane == 0) tma_store_wait_all();  // this warp's stores have landed before the CTA exits
     }
 
     // ---------------------------------- teardown ------------------------------------
     __syncwarp();
     if (*abort_flag) __nanosleep(1000000);  // let copies / MMAs in flight land before freeing
     tcgen05_fence_before();
-    __syncthreads();
+    if (CG == 1) __syncthreads(); else cluster_sync_all();  // the peer may still signal this CTA's barriers
     if (warp == 5) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "n"(C::TMEM_COLS)
-                     : "memory");
+        tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
     }
 }
 
@@ -494,7 +628,7 @@ EncodeTiledFn encode_fn() {
 // Rank-4 INT8 tensor map over {inner (contiguous), row, head, batch} with the three outer
 // dimensions ordered by ascending stride; reports which coordinate slot each one got.
 // box_inner x box_rows bytes are copied per request (128-byte swizzle).
-bool make_map(CUtensorMap* map, const int8_t* base, int64_t inner, int64_t rows, int64_t heads,
+bool make_map(CUtensorMap* map, const void* base, int esz, int64_t inner, int64_t rows, int64_t heads,
               int64_t batch, int64_t s_row, int64_t s_head, int64_t s_batch, int box_inner, int box_rows,
               int* slot_row, int* slot_head, int* slot_batch) {
     EncodeTiledFn fn = encode_fn();
@@ -503,7 +637,10 @@ bool make_map(CUtensorMap* map, const int8_t* base, int64_t inner, int64_t rows,
     Dim d[3] = {{rows, s_row, box_rows, slot_row}, {heads, s_head, 1, slot_head}, {batch, s_batch, 1, slot_batch}};
     // extent-1 dimensions never move the address: give them a harmless large stride so that
     // the order below stays ascending
-    int64_t span = std::max<int64_t>(inner, 16);
+    // strides are given in elements of `esz` bytes
+    s_row *= esz; s_head *= esz; s_batch *= esz;
+    d[0].stride = s_row; d[1].stride = s_head; d[2].stride = s_batch;
+    int64_t span = std::max<int64_t>(inner * esz, 16);
     for (auto& x : d) if (x.extent > 1) span = std::max(span, x.extent * x.stride);
     span = (span + 15) / 16 * 16;
     for (auto& x : d) if (x.extent <= 1) x.stride = span;
@@ -513,32 +650,34 @@ bool make_map(CUtensorMap* map, const int8_t* base, int64_t inner, int64_t rows,
     cuuint32_t box[4] = {(cuuint32_t)box_inner, (cuuint32_t)d[0].box, (cuuint32_t)d[1].box, (cuuint32_t)d[2].box};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     for (int i = 0; i < 3; ++i) *d[i].slot = i + 1;
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(base), gdim, gstr, box, estr,
+    const CUtensorMapDataType ty = esz == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
+                                   : esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_INT32;
+    CUresult r = fn(map, ty, 4, const_cast<void*>(base), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
-template <int BLOCK_N>
+template <int BLOCK_N, int CG>
 sq_status launch(const GemmArgs& a, cudaStream_t st) {
-    using C = Cfg<BLOCK_N>;
+    using C = Cfg<BLOCK_N, CG>;
     Params p;
     p.M = a.M; p.N = a.N; p.K = a.K;
     p.heads = (int)a.heads; p.batch = (int)a.batch;
-    p.num_m = (int)((a.M + BLOCK_M - 1) / BLOCK_M);
+    p.num_m = (int)((a.M + BLOCK_M * CG - 1) / (BLOCK_M * CG));
     p.num_n = (int)((a.N + BLOCK_N - 1) / BLOCK_N);
     p.total_tiles = (int64_t)p.num_m * p.num_n * a.heads * a.batch;
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     p.b_is_kn = a.b_is_kn;
     CUtensorMap ma, mb;
-    if (!make_map(&ma, a.A, a.K, a.M, a.heads, a.batch, a.strideA[2], a.strideA[1], a.strideA[0], BLOCK_K,
+    if (!make_map(&ma, a.A, 1, a.K, a.M, a.heads, a.batch, a.strideA[2], a.strideA[1], a.strideA[0], BLOCK_K,
                   BLOCK_M, &p.a_slot_row, &p.a_slot_head, &p.a_slot_batch))
         return SQ_ERR_CUDA;
     const bool okb =
-        a.b_is_kn ? make_map(&mb, a.B, a.N, a.K, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
-                             BLOCK_N, BLOCK_K, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch)
-                  : make_map(&mb, a.B, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
-                             BLOCK_K, BLOCK_N, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch);
+        a.b_is_kn ? make_map(&mb, a.B, 1, a.N, a.K, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
+                             C::B_ROWS, BLOCK_K, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch)
+                  : make_map(&mb, a.B, 1, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0],
+                             BLOCK_K, C::B_ROWS, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch);
     if (!okb) return SQ_ERR_CUDA;
     p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
     p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
@@ -551,29 +690,65 @@ sq_status launch(const GemmArgs& a, cudaStream_t st) {
     p.c_stride_batch = a.strideC[0]; p.c_stride_head = a.strideC[1]; p.c_stride_row = a.strideC[2];
     const int esz = a.out_dt == SQ_I32 ? 4 : (a.out_dt == SQ_I8 ? 1 : 2);
     const int vec_elems = 16 / esz;
-    p.c_vec_ok = aligned16(a.C) && a.strideC[0] % vec_elems == 0 && a.strideC[1] % vec_elems == 0 &&
-                 a.strideC[2] % vec_elems == 0;
+    p.c_tma = aligned16(a.C) && a.strideC[0] % vec_elems == 0 && a.strideC[1] % vec_elems == 0 &&
+              a.strideC[2] % vec_elems == 0;
+    p.c_slot_row = 1; p.c_slot_head = 2; p.c_slot_batch = 3;
+    CUtensorMap mc = ma;  // placeholder when C is written directly
+    if (p.c_tma && !make_map(&mc, a.C, esz, a.N, a.M, a.heads, a.batch, a.strideC[2], a.strideC[1], a.strideC[0],
+                             128 / esz, 32, &p.c_slot_row, &p.c_slot_head, &p.c_slot_batch))
+        return SQ_ERR_CUDA;
     p.status = a.status;
 
     static bool attr_set[64] = {false};  // once per device
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         C::SMEM_BYTES));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const int grid = (int)std::min<int64_t>(p.total_tiles, sm_count());
-    gemm_i8_kernel<BLOCK_N><<<grid, NUM_THREADS, C::SMEM_BYTES, st>>>(ma, mb, p);
+    const int groups = (int)std::min<int64_t>(p.total_tiles, sm_count() / CG);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(groups * CG));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CG > 1 ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BLOCK_N, CG>, ma, mb, mc, p) != cudaSuccess) {
+        cudaGetLastError();
+        return SQ_ERR_CUDA;
+    }
     return launch_status();
+}
+
+// Relative cost of covering the problem with tiles of (128*cg) x bn on `sms` SMs: full waves
+// of tiles times the tile's MMA time, which is proportional to bn.
+double tiling_cost(const GemmArgs& a, int bn, int cg, int sms) {
+    const int64_t tiles = ((a.M + 128 * cg - 1) / (128 * cg)) * ((a.N + bn - 1) / bn) * a.heads * a.batch;
+    const int64_t groups = sms / cg;
+    const int64_t waves = (tiles + groups - 1) / groups;
+    return (double)waves * bn;
 }
 
 }  // namespace
 
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
     // [K, N]-stored B is limited to one 128-byte swizzle row of N per tile
-    if (a.b_is_kn || a.N <= 128) return launch<128>(a, st);
-    return launch<256>(a, st);
+    if (a.b_is_kn || a.N <= 128) return launch<128, 1>(a, st);
+    if (a.M <= 128) return launch<256, 1>(a, st);
+    // CTA pairs; pick the tile width that leaves the fewest idle SMs in the last wave
+    const int sms = sm_count();
+    const double c256 = tiling_cost(a, 256, 2, sms), c192 = tiling_cost(a, 192, 2, sms) * 1.02,
+                 c128 = tiling_cost(a, 128, 2, sms) * 1.10;  // narrower tiles re-read A more often
+    if (c256 <= c192 && c256 <= c128) return launch<256, 2>(a, st);
+    if (c192 <= c128) return launch<192, 2>(a, st);
+    return launch<128, 2>(a, st);
 }
 
 }  // namespace sq

@@ -22,7 +22,9 @@ def ws():
 
 # (M, N, K): one tile, several tiles, ragged M / N / K tails, single row, N < 128, wide K
 SHAPES = [(16, 512, 512), (128, 256, 128), (128, 128, 128), (129, 257, 144), (300, 520, 272),
-          (1, 64, 16), (200, 72, 2048), (256, 1024, 5120), (77, 2000, 1040), (515, 384, 640)]
+          (1, 64, 16), (200, 72, 2048), (256, 1024, 5120), (77, 2000, 1040), (515, 384, 640),
+          # CTA-pair kernel: many tiles per pair, each of the three tile widths, odd tile counts
+          (2048, 768, 512), (1000, 5120, 1024), (384, 640, 256), (640, 1344, 384), (2048, 5120, 256)]
 
 
 @pytest.mark.parametrize("M,N,K", SHAPES)
@@ -102,6 +104,26 @@ def test_gemm_strided_output(ws):
     got = host(buf)
     assert np.array_equal(got[:, :N], want)
     assert np.all(got[:, N:] == -7.0)  # nothing written beyond the N columns
+
+
+@pytest.mark.parametrize("out", ["f16", "i8", "i32"])
+def test_gemm_unaligned_output_rows(ws, out):
+    # row stride that is not a multiple of 16 bytes: the epilogue writes rows directly instead of by TMA
+    M, N, K, ldy = 150, 201, 256, 203
+    Xq, Wq = synth.int8_tensor(23, 3, (M, K)), synth.int8_tensor(23, 4, (N, K))
+    xs = np.full(1, 0.05, np.float32)
+    wsc = np.full(1, 0.002, np.float32)
+    tdt = {"f16": torch.float16, "i8": torch.int8, "i32": torch.int32}[out]
+    buf = torch.full((M, ldy), 5, dtype=tdt, device="cuda")
+    r = np.array([0.9], np.float32)
+    sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, out=buf[:, :N],
+                    requant_mul=dev(r) if out == "i8" else None)
+    acc = oracle.gemm_i32(Xq, Wq)
+    y = oracle.dequant(acc, xs, wsc)
+    want = {"f16": oracle.round_to(y, "f16"), "i8": oracle.requant(y, r), "i32": acc}[out]
+    got = host(buf)
+    assert np.array_equal(got[:, :N], want)
+    assert np.all(got[:, N:] == 5)
 
 
 def _qkv_views(B, H, S, d, seed):
