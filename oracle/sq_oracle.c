@@ -109,13 +109,15 @@ float sqo_step_size(float absmax) {
     return m / 127.0f;
 }
 
-/* Eq. 1: X_bar = round(X / Delta), evaluated as X * (1/Delta) with one fp32
- * reciprocal per step size, round-half-to-even, clamped to [-127, 127] (the
- * symmetric range 2^(N-1)-1 of Eq. 1; -128 is never produced). */
+/* Eq. 1: X_bar = round(X / Delta), evaluated as round(X * inv) with one fp32
+ * reciprocal inv = 1/Delta per step size.  The product is NOT rounded before
+ * the rounding function is applied: the product of two floats is exact in
+ * double, so rint() below sees x * inv itself.  Round-half-to-even, clamped to
+ * [-127, 127] (the symmetric range 2^(N-1)-1 of Eq. 1; -128 is never produced). */
 static inline int8_t sqo_q(float v, float inv) {
-    float r = rintf(v * inv);
-    if (r > 127.0f) r = 127.0f;
-    if (r < -127.0f) r = -127.0f;
+    double r = rint((double)v * (double)inv);
+    if (r > 127.0) r = 127.0;
+    if (r < -127.0) r = -127.0;
     return (int8_t)r;
 }
 
@@ -173,15 +175,18 @@ void sqo_ln_stats_f64(const float *X, int64_t M, int64_t C, int64_t ld, double e
 }
 
 /* Normative element-wise part of the folded LayerNorm, given fp32 row
- * statistics: y = fma((x - mu) * rstd, gamma_hat_j, beta_hat_j), all fp32, and
+ * statistics, as two fused multiply-adds in fp32:
+ *   n = fma(x, rstd, -(mu * rstd)),  y = fma(n, gamma_hat_j, beta_hat_j);
  * y is NOT rounded to fp16/bf16 before it is quantised. */
 void sqo_ln_apply(const float *X, int64_t M, int64_t C, int64_t ld, const float *mu,
                   const float *rstd, const float *gamma_hat, const float *beta_hat, float *Y) {
-    for (int64_t t = 0; t < M; ++t)
+    for (int64_t t = 0; t < M; ++t) {
+        float shift = -(mu[t] * rstd[t]);
         for (int64_t j = 0; j < C; ++j) {
-            float n = (X[t * ld + j] - mu[t]) * rstd[t];
+            float n = fmaf(X[t * ld + j], rstd[t], shift);
             Y[t * C + j] = fmaf(n, gamma_hat[j], beta_hat ? beta_hat[j] : 0.0f);
         }
+    }
 }
 
 /* fp64 LayerNorm output, for pins. */

@@ -91,20 +91,28 @@ __device__ __forceinline__ float step_size(float absmax) {
 }
 __device__ __forceinline__ float recip_step(float delta) { return __fdiv_rn(1.0f, delta); }
 
-__device__ __forceinline__ int quant_code(float v, float inv) {
-    int q = __float2int_rn(__fmul_rn(v, inv));  // round-half-to-even; saturates on overflow
-    return max(-127, min(127, q));
+// round(v * inv) with ONE rounding: the fused multiply-add adds 1.5 * 2^23 to the exact
+// product, so the fp32 result is rounded (half to even) at integer granularity and the code
+// sits in the low mantissa bits as a two's-complement byte.  CLAMP keeps it in [-127, 127];
+// without it the caller guarantees |v * inv| < 127.5 (dynamic step sizes).
+constexpr float kRoundMagic = 12582912.0f;
+template <bool CLAMP = true>
+__device__ __forceinline__ uint32_t quant_code(float v, float inv) {
+    float r = __fmaf_rn(v, inv, kRoundMagic);
+    if (CLAMP) r = fminf(fmaxf(r, kRoundMagic - 127.0f), kRoundMagic + 127.0f);
+    return __float_as_uint(r);  // low byte = the INT8 code
 }
-__device__ __forceinline__ uint32_t pack4(int a, int b, int c, int d) {
-    return (uint32_t)(a & 0xff) | ((uint32_t)(b & 0xff) << 8) | ((uint32_t)(c & 0xff) << 16) |
-           ((uint32_t)(d & 0xff) << 24);
+// low bytes of four words -> one word
+__device__ __forceinline__ uint32_t pack4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
 }
+template <bool CLAMP = true>
 __device__ __forceinline__ uint2 quant8(const float (&f)[8], float inv) {
     uint2 r;
-    r.x = pack4(quant_code(f[0], inv), quant_code(f[1], inv), quant_code(f[2], inv),
-                quant_code(f[3], inv));
-    r.y = pack4(quant_code(f[4], inv), quant_code(f[5], inv), quant_code(f[6], inv),
-                quant_code(f[7], inv));
+    r.x = pack4(quant_code<CLAMP>(f[0], inv), quant_code<CLAMP>(f[1], inv), quant_code<CLAMP>(f[2], inv),
+                quant_code<CLAMP>(f[3], inv));
+    r.y = pack4(quant_code<CLAMP>(f[4], inv), quant_code<CLAMP>(f[5], inv), quant_code<CLAMP>(f[6], inv),
+                quant_code<CLAMP>(f[7], inv));
     return r;
 }
 

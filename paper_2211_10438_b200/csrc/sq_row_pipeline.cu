@@ -1,0 +1,326 @@
+// Fused LayerNorm + smooth + absmax + INT8 quantise (and the plain quantiser) as a persistent,
+// bulk-copy-fed pipeline: the HBM-bound runtime stage in front of every W8A8 GEMM.
+//
+//   * one CTA per SM, 1024 threads split into groups of GROUP threads; a group owns one row
+//     (token) at a time and walks the rows assigned to it;
+//   * rows arrive through a ring of shared-memory stages filled by cp.async.bulk (one bulk
+//     copy per row, completion on an mbarrier), so the next rows stream in from HBM while
+//     the current one is being reduced and quantised;
+//   * the folded LayerNorm parameters gamma_hat / beta_hat live in shared memory for the whole
+//     kernel; a row is unpacked once into registers (at most 32 values per thread), so HBM
+//     sees 2 bytes in + 1 byte out per element and nothing else;
+//   * reductions (sum, sum of squares, absmax) are warp shuffles + one named barrier each.
+// Arithmetic is the normative fp32 sequence: n = fma(x, rstd, -(mu*rstd)),
+// y = fma(n, gamma_hat, beta_hat), Delta = max(|y|, 1e-5)/127, q = round(y * (1/Delta)).
+// The kernel is instruction-issue sensitive (about 11 instructions per element at 3 bytes of
+// HBM traffic per element), hence the single-FMA rounding and byte-permute packing.
+#include "sq_common.cuh"
+#include "sq_kernels.h"
+
+namespace sq {
+
+namespace {
+
+constexpr int CTA_THREADS = 1024;
+constexpr uint32_t kWaitCycles = 2000000000u;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity))
+        if ((++spins & 63u) == 0u && (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) return false;
+    return true;
+}
+// one row: global -> shared, completion counted in bytes on `bar` (addresses 16-byte aligned)
+__device__ __forceinline__ void bulk_load_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+template <int GROUP>
+__device__ __forceinline__ void group_sync(int g) {
+    if (GROUP == CTA_THREADS) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(GROUP) : "memory");
+}
+// All GROUP threads get the reduction of v; `red` holds GROUP/32 floats owned by this call site.
+template <bool IS_MAX, int GROUP>
+__device__ __forceinline__ float group_reduce(float v, float* red, int g, int gwarp, int lane) {
+    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    if (lane == 0) red[gwarp] = v;
+    group_sync<GROUP>(g);
+    constexpr int NW = GROUP / 32;
+    // every thread folds the NW partials in the same order (identical result in all threads)
+    float r = lane < NW ? red[lane] : (IS_MAX ? 0.0f : 0.0f);
+    if (NW > 1) r = IS_MAX ? warp_max(r) : warp_sum(r);
+    return __shfl_sync(0xffffffffu, r, 0);
+}
+
+template <typename T, int GROUP, int V, bool LN>
+__global__ void __launch_bounds__(CTA_THREADS, 1)
+row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__ gamma,
+                const T* __restrict__ beta, float eps, int mode, int stages, int8_t* __restrict__ Xq,
+                float* __restrict__ scale, float* __restrict__ absmax_word, float* __restrict__ stats,
+                int stats_are_input, uint32_t* __restrict__ status) {
+    constexpr int G = CTA_THREADS / GROUP;  // rows in flight per CTA
+    constexpr int NW = GROUP / 32;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int row_bytes = C * 2;
+    const int nvec = C >> 3;
+    uint8_t* s_gamma = smem;                                   // [C] T   (LN only)
+    uint8_t* s_beta = smem + (LN ? row_bytes : 0);             // [C] T   (LN only)
+    uint8_t* s_rows = smem + (LN ? 2 * row_bytes : 0);         // [G][stages][C] T
+    uint64_t* full = reinterpret_cast<uint64_t*>(s_rows + (size_t)G * stages * row_bytes);  // [G][stages]
+    float* s_red = reinterpret_cast<float*>(full + G * stages);                             // [G][3][NW]
+
+    const int tid = threadIdx.x;
+    const int g = tid / GROUP, gt = tid % GROUP, gwarp = gt >> 5, lane = tid & 31;
+    const int64_t first = (int64_t)blockIdx.x * G + g;
+    const int64_t stride = (int64_t)gridDim.x * G;
+    uint64_t* my_full = full + g * stages;
+    uint8_t* my_rows = s_rows + (size_t)g * stages * row_bytes;
+    float* red = s_red + g * 3 * NW;
+    volatile uint32_t* my_flag = reinterpret_cast<volatile uint32_t*>(s_red + G * 3 * NW) + g;
+
+    if (gt == 0) {
+        for (int s = 0; s < stages; ++s) mbar_init(my_full + s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // prologue: fill the ring
+        for (int s = 0; s < stages; ++s) {
+            const int64_t r = first + (int64_t)s * stride;
+            if (r < M) {
+                mbar_expect_tx(my_full + s, (uint32_t)row_bytes);
+                bulk_load_row(my_rows + (size_t)s * row_bytes, X + r * C, (uint32_t)row_bytes, my_full + s);
+            }
+        }
+    }
+    if (LN) {  // parameters: global -> shared once per CTA
+        const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
+        const uint4* b4 = reinterpret_cast<const uint4*>(beta);
+        for (int v = tid; v < nvec; v += CTA_THREADS) {
+            reinterpret_cast<uint4*>(s_gamma)[v] = __ldg(g4 + v);
+            reinterpret_cast<uint4*>(s_beta)[v] = beta ? __ldg(b4 + v) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+    __syncthreads();
+
+    float tensor_delta = 0.0f;
+    if (mode == ROW_GIVEN_SCALE) tensor_delta = __ldg(scale);
+    else if (mode == ROW_FROM_ABSMAX_WORD) {
+        tensor_delta = step_size(__ldg(absmax_word));
+        if (blockIdx.x == 0 && tid == 0) scale[0] = tensor_delta;
+    }
+    float group_max = 0.0f;  // ROW_ABSMAX_ONLY: one atomic per group at the end
+
+    int it = 0;
+    for (int64_t row = first; row < M; row += stride, ++it) {
+        const int s = it % stages;
+        const uint32_t parity = (uint32_t)(it / stages) & 1u;
+        // One thread waits (bounded) for the row's bulk copy; its verdict reaches the group through
+        // shared memory so that every thread takes the same branch.
+        if (gt == 0) {
+            const bool ok = mbar_wait_bounded(my_full + s, parity);
+            if (!ok && status != nullptr) atomicCAS(status, 0u, (uint32_t)SQ_ERR_TIMEOUT | (5u << 8));
+            *my_flag = ok ? 1u : 0u;
+        }
+        group_sync<GROUP>(g);
+        if (*my_flag == 0u) break;  // the copy never landed: stop this group
+        const uint4* srow = reinterpret_cast<const uint4*>(my_rows + (size_t)s * row_bytes);
+        uint4 raw[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int v = gt + i * GROUP;
+            raw[i] = v < nvec ? srow[v] : make_uint4(0u, 0u, 0u, 0u);
+        }
+        // After the next group-wide barrier everyone holds the row in registers and the stage can
+        // be refilled with the row `stages` iterations ahead.
+        bool refilled = false;
+        auto refill = [&]() {
+            if (!refilled && gt == 0) {
+                const int64_t nxt = row + (int64_t)stages * stride;
+                if (nxt < M) {
+                    mbar_expect_tx(my_full + s, (uint32_t)row_bytes);
+                    bulk_load_row(my_rows + (size_t)s * row_bytes, X + nxt * C, (uint32_t)row_bytes, my_full + s);
+                }
+            }
+            refilled = true;
+        };
+        if ((LN && stats_are_input) || (!LN && mode != ROW_DYNAMIC && mode != ROW_ABSMAX_ONLY)) {
+            group_sync<GROUP>(g);  // no reduction follows on this path: synchronise explicitly
+            refill();
+        }
+
+        float m = 0.0f;
+        float y[V][8];
+#pragma unroll
+        for (int i = 0; i < V; ++i) unpack8<T>(raw[i], y[i]);
+        if (LN) {
+            float mu, rstd;
+            if (stats_are_input) {
+                mu = stats[2 * row];
+                rstd = stats[2 * row + 1];
+            } else {
+                float sum = 0.0f;
+#pragma unroll
+                for (int i = 0; i < V; ++i) {  // zero-filled vectors add nothing
+                    const float* f = y[i];
+                    sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
+                }
+                mu = group_reduce<false, GROUP>(sum, red, g, gwarp, lane) / (float)C;
+                refill();
+                float ss = 0.0f;
+#pragma unroll
+                for (int i = 0; i < V; ++i) {
+                    if (gt + i * GROUP < nvec) {
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float d = y[i][k] - mu;
+                            ss = fmaf(d, d, ss);
+                        }
+                    }
+                }
+                const float var = group_reduce<false, GROUP>(ss, red + NW, g, gwarp, lane) / (float)C;
+                rstd = __fdiv_rn(1.0f, __fsqrt_rn(var + eps));
+                if (stats != nullptr && gt == 0) {
+                    stats[2 * row] = mu;
+                    stats[2 * row + 1] = rstd;
+                }
+            }
+            const float shift = -__fmul_rn(mu, rstd);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const int v = gt + i * GROUP;
+                if (v < nvec) {
+                    float ga[8], be[8];
+                    unpack8<T>(reinterpret_cast<const uint4*>(s_gamma)[v], ga);
+                    unpack8<T>(reinterpret_cast<const uint4*>(s_beta)[v], be);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const float t = __fmaf_rn(__fmaf_rn(y[i][k], rstd, shift), ga[k], be[k]);
+                        y[i][k] = t;
+                        m = fmaxf(m, fabsf(t));
+                    }
+                }
+            }
+        } else if (mode == ROW_DYNAMIC || mode == ROW_ABSMAX_ONLY) {
+            uint32_t pm = 0u;  // packed running max of |x|: exact in fp16/bf16
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                pm = Act<T>::absmax2(pm, raw[i].x); pm = Act<T>::absmax2(pm, raw[i].y);
+                pm = Act<T>::absmax2(pm, raw[i].z); pm = Act<T>::absmax2(pm, raw[i].w);
+            }
+            m = Act<T>::hmax_of2(pm);
+        }
+
+        float delta = tensor_delta;
+        if (mode == ROW_DYNAMIC || mode == ROW_ABSMAX_ONLY) {
+            m = group_reduce<true, GROUP>(m, red + 2 * NW, g, gwarp, lane);
+            refill();
+            if (mode == ROW_ABSMAX_ONLY) {
+                group_max = fmaxf(group_max, m);
+                continue;
+            }
+            delta = step_size(m);
+            if (gt == 0) scale[row] = delta;
+        }
+        const float inv = recip_step(delta);
+        uint2* qrow = reinterpret_cast<uint2*>(Xq + row * C);
+        if (mode == ROW_GIVEN_SCALE) {  // a calibrated step may be exceeded at run time: saturate
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const int v = gt + i * GROUP;
+                if (v < nvec) qrow[v] = quant8<true>(y[i], inv);
+            }
+        } else {  // |y| <= absmax by construction: |y * inv| < 127.5, no clamp needed
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const int v = gt + i * GROUP;
+                if (v < nvec) qrow[v] = quant8<false>(y[i], inv);
+            }
+        }
+    }
+    if (mode == ROW_ABSMAX_ONLY && gt == 0) atomic_max_nonneg(absmax_word, group_max);
+}
+
+template <typename T, int GROUP, int V, bool LN>
+sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, const void* beta, float eps,
+                      int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats, int stats_are_input,
+                      uint32_t* status, cudaStream_t st) {
+    constexpr int G = CTA_THREADS / GROUP;
+    const size_t row_bytes = (size_t)C * 2;
+    const size_t fixed = (LN ? 2 * row_bytes : 0) + 2048 /*barriers + reduction scratch*/;
+    const size_t budget = 220 * 1024;
+    if (budget < fixed + G * row_bytes) return SQ_ERR_UNSUPPORTED;
+    int stages = (int)((budget - fixed) / (G * row_bytes));
+    stages = std::min(stages, 8);
+    const size_t smem = (LN ? 2 * row_bytes : 0) + (size_t)G * stages * row_bytes + (size_t)G * stages * 8 +
+                        (size_t)G * 3 * (GROUP / 32) * 4 + (size_t)G * 4 + 128;
+    auto kern = row_pipe_kernel<T, GROUP, V, LN>;
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    SQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        SQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    const int grid = (int)std::min<int64_t>((M + G - 1) / G, sm_count());
+    kern<<<grid, CTA_THREADS, smem, st>>>(static_cast<const T*>(X), M, (int)C, static_cast<const T*>(gamma),
+                                          static_cast<const T*>(beta), eps, mode, stages, Xq, scale, absmax_word,
+                                          stats, stats_are_input, status);
+    return launch_status();
+}
+
+template <typename T, bool LN>
+sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, const void* beta, float eps,
+                        int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats,
+                        int stats_are_input, uint32_t* status, cudaStream_t st) {
+    const int64_t nvec = C / 8;
+#define SQ_PIPE(GROUP, V)                                                                                  \
+    return launch_pipe<T, GROUP, V, LN>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,    \
+                                        stats_are_input, status, st)
+    if (nvec <= 128 * 3) SQ_PIPE(128, 3);    // C <= 3072
+    if (nvec <= 256 * 3) SQ_PIPE(256, 3);    // C <= 6144   (5120)
+    if (nvec <= 512 * 3) SQ_PIPE(512, 3);    // C <= 12288  (7168, 12288)
+    if (nvec <= 1024 * 3) SQ_PIPE(1024, 3);  // C <= 24576  (20480)
+    SQ_PIPE(1024, 4);                        // C <= 32768  (28672)
+#undef SQ_PIPE
+}
+
+}  // namespace
+
+bool row_pipeline_supports(int64_t M, int64_t C, bool has_col_mul) {
+    return !has_col_mul && M > 0 && C % 8 == 0 && C / 8 <= 1024 * 4;
+}
+
+sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma, const void* beta,
+                       float eps, bool ln, int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats,
+                       int stats_are_input, uint32_t* status, cudaStream_t st) {
+    if (dt == SQ_F16)
+        return ln ? dispatch_pipe<__half, true>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,
+                                                stats_are_input, status, st)
+                  : dispatch_pipe<__half, false>(X, M, C, nullptr, nullptr, 0.f, mode, Xq, scale, absmax_word,
+                                                 nullptr, 0, status, st);
+    return ln ? dispatch_pipe<__nv_bfloat16, true>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,
+                                                   stats_are_input, status, st)
+              : dispatch_pipe<__nv_bfloat16, false>(X, M, C, nullptr, nullptr, 0.f, mode, Xq, scale, absmax_word,
+                                                    nullptr, 0, status, st);
+}
+
+}  // namespace sq

@@ -264,9 +264,9 @@ row_quant_kernel(const T* __restrict__ X, int64_t M, int64_t C, const float* __r
 #pragma unroll
                 for (int k = 0; k < 8; ++k) b[k] = 0.0f;
             }
+            const float shift = -__fmul_rn(mu, rstd);
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-                f[k] = __fmaf_rn(__fmul_rn(__fsub_rn(f[k], mu), rstd), g[k], b[k]);
+            for (int k = 0; k < 8; ++k) f[k] = __fmaf_rn(__fmaf_rn(f[k], rstd, shift), g[k], b[k]);
         }
         if (HAS_MUL) {
             const float4 m0 = __ldg(reinterpret_cast<const float4*>(col_mul) + 2 * v);
@@ -381,6 +381,10 @@ sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const floa
                     const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
                     float* scale, float* absmax_word, float* stats, int stats_are_input,
                     cudaStream_t st) {
+    // rows up to 32768 elements without a column multiplier take the bulk-copy pipeline
+    if (row_pipeline_supports(M, C, col_mul != nullptr))
+        return row_pipeline(X, dt, M, C, gamma, beta, eps, ln, mode, Xq, scale, absmax_word, stats,
+                            stats_are_input, nullptr, st);
 #define SQ_DISPATCH(T)                                                                           \
     (ln ? launch_rows<T, true, false>(X, M, C, nullptr, gamma, beta, eps, mode, Xq, scale,       \
                                       absmax_word, stats, stats_are_input, st)                   \
