@@ -1,14 +1,16 @@
 // Fused LayerNorm + smooth + absmax + INT8 quantise (and the plain quantiser) as a persistent,
 // bulk-copy-fed pipeline: the HBM-bound runtime stage in front of every W8A8 GEMM.
 //
-//   * one CTA per SM, 1024 threads split into groups of GROUP threads; a group owns one row
-//     (token) at a time and walks the rows assigned to it;
+//   * one CTA per SM, 512 threads split into groups of GROUP threads; a group owns one row
+//     (token) at a time and walks the rows assigned to it.  A thread holds up to 80 values of
+//     its row: per-row costs (three reductions, barrier, ring bookkeeping) are paid once per
+//     thread and row, so few threads per row keep the instruction count per element low;
 //   * rows arrive through a ring of shared-memory stages filled by cp.async.bulk (one bulk
 //     copy per row, completion on an mbarrier), so the next rows stream in from HBM while
 //     the current one is being reduced and quantised;
 //   * the folded LayerNorm parameters gamma_hat / beta_hat live in shared memory for the whole
-//     kernel; a row is unpacked once into registers (at most 32 values per thread), so HBM
-//     sees 2 bytes in + 1 byte out per element and nothing else;
+//     kernel; a row is unpacked once into registers, so HBM sees 2 bytes in + 1 byte out per
+//     element and nothing else;
 //   * reductions (sum, sum of squares, absmax) are warp shuffles + one named barrier each.
 // Arithmetic is the normative fp32 sequence: n = fma(x, rstd, -(mu*rstd)),
 // y = fma(n, gamma_hat, beta_hat), Delta = max(|y|, 1e-5)/127, q = round(y * (1/Delta)).
@@ -21,7 +23,7 @@ namespace sq {
 
 namespace {
 
-constexpr int CTA_THREADS = 1024;
+constexpr int CTA_THREADS = 512;
 constexpr uint32_t kWaitCycles = 2000000000u;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -62,14 +64,16 @@ __device__ __forceinline__ void group_sync(int g) {
 // All GROUP threads get the reduction of v; `red` holds GROUP/32 floats owned by this call site.
 template <bool IS_MAX, int GROUP>
 __device__ __forceinline__ float group_reduce(float v, float* red, int g, int gwarp, int lane) {
-    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    // non-negative floats order like their bit patterns: one redux instruction per level
+    v = IS_MAX ? __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(v))) : warp_sum(v);
     if (lane == 0) red[gwarp] = v;
     group_sync<GROUP>(g);
     constexpr int NW = GROUP / 32;
     // every thread folds the NW partials in the same order (identical result in all threads)
-    float r = lane < NW ? red[lane] : (IS_MAX ? 0.0f : 0.0f);
-    if (NW > 1) r = IS_MAX ? warp_max(r) : warp_sum(r);
-    return __shfl_sync(0xffffffffu, r, 0);
+    float r = red[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) r = IS_MAX ? fmaxf(r, red[i]) : r + red[i];
+    return r;
 }
 
 template <typename T, int GROUP, int V, bool LN>
@@ -129,10 +133,9 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     }
     float group_max = 0.0f;  // ROW_ABSMAX_ONLY: one atomic per group at the end
 
-    int it = 0;
-    for (int64_t row = first; row < M; row += stride, ++it) {
-        const int s = it % stages;
-        const uint32_t parity = (uint32_t)(it / stages) & 1u;
+    int s = 0;
+    uint32_t parity = 0;
+    for (int64_t row = first; row < M; row += stride) {
         // One thread waits (bounded) for the row's bulk copy; its verdict reaches the group through
         // shared memory so that every thread takes the same branch.
         if (gt == 0) {
@@ -235,6 +238,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
             refill();
             if (mode == ROW_ABSMAX_ONLY) {
                 group_max = fmaxf(group_max, m);
+                if (++s == stages) { s = 0; parity ^= 1u; }
                 continue;
             }
             delta = step_size(m);
@@ -255,8 +259,10 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 if (v < nvec) qrow[v] = quant8<false>(y[i], inv);
             }
         }
+        if (++s == stages) { s = 0; parity ^= 1u; }
     }
     if (mode == ROW_ABSMAX_ONLY && gt == 0) atomic_max_nonneg(absmax_word, group_max);
+    (void)parity;
 }
 
 template <typename T, int GROUP, int V, bool LN>
@@ -295,18 +301,20 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
 #define SQ_PIPE(GROUP, V)                                                                                  \
     return launch_pipe<T, GROUP, V, LN>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,    \
                                         stats_are_input, status, st)
-    if (nvec <= 128 * 3) SQ_PIPE(128, 3);    // C <= 3072
-    if (nvec <= 256 * 3) SQ_PIPE(256, 3);    // C <= 6144   (5120)
-    if (nvec <= 512 * 3) SQ_PIPE(512, 3);    // C <= 12288  (7168, 12288)
-    if (nvec <= 1024 * 3) SQ_PIPE(1024, 3);  // C <= 24576  (20480)
-    SQ_PIPE(1024, 4);                        // C <= 32768  (28672)
+    if (nvec <= 64 * 8) SQ_PIPE(64, 8);      // C <= 4096
+    if (nvec <= 64 * 10) SQ_PIPE(64, 10);    // C <= 5120
+    if (nvec <= 128 * 8) SQ_PIPE(128, 8);    // C <= 8192   (7168)
+    if (nvec <= 128 * 10) SQ_PIPE(128, 10);  // C <= 10240
+    if (nvec <= 256 * 8) SQ_PIPE(256, 8);    // C <= 16384  (12288)
+    if (nvec <= 256 * 10) SQ_PIPE(256, 10);  // C <= 20480
+    SQ_PIPE(512, 8);                         // C <= 32768  (28672)
 #undef SQ_PIPE
 }
 
 }  // namespace
 
 bool row_pipeline_supports(int64_t M, int64_t C, bool has_col_mul) {
-    return !has_col_mul && M > 0 && C % 8 == 0 && C / 8 <= 1024 * 4;
+    return !has_col_mul && M > 0 && C % 8 == 0 && C / 8 <= 512 * 8;
 }
 
 sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma, const void* beta,
