@@ -378,3 +378,55 @@ def linear_f64(X, W, b=None):
     _lib.sqo_linear_f64(_p(X, _f64p), _p(W, _f64p), _p(bb, _f64p), _i64(M), _i64(N), _i64(K),
                         _p(Y, _f64p))
     return Y
+
+
+# --------------------------------------------------------------------------- #
+# Whole decoder block (Fig. 6), static per-tensor activation steps (O3)
+# --------------------------------------------------------------------------- #
+def decoder_block_static(x, p, B, S, H, d, dtype="f16", eps=1e-5):
+    """One pre-LayerNorm decoder block in the precision mapping of Fig. 6: INT8 for the four
+    linear layers and the two attention BMMs, floating point for LayerNorm, softmax, ReLU and
+    the residual adds.  `x` is [B*S, H*d] (A-valued float32); `p` holds, per linear
+    ("qkv", "out_proj", "fc1", "fc2"), the INT8 weight `Wq`, `w_scale`, `bias`, and the static
+    steps `d_ln1, d_q, d_k, d_v, d_attn, d_ln2, d_fc1` plus folded LayerNorm parameters
+    `g1, b1, g2, b2`.  Every intermediate is returned for stage-by-stage comparison."""
+    f32 = np.float32
+    hid = H * d
+    out = {}
+    # LN1 (smoothing folded) -> INT8, static step
+    out["x1q"], _, _ = ln_quant(x, p["g1"], p["b1"], eps, "per_tensor_static", static_scale=p["d_ln1"])
+    # QKV projection, re-quantised to INT8 with one static step per q / k / v
+    acc = gemm_i32(out["x1q"], p["qkv"]["Wq"])
+    y = dequant(acc, p["d_ln1"], p["qkv"]["w_scale"], p["qkv"]["bias"])
+    r = np.concatenate([np.full(hid, f32(1) / f32(p["d_q"]), f32), np.full(hid, f32(1) / f32(p["d_k"]), f32),
+                        np.full(hid, f32(1) / f32(p["d_v"]), f32)])
+    out["qkv"] = requant(y, r)
+    qkv = out["qkv"].reshape(B, S, 3, H, d)
+    q = np.ascontiguousarray(qkv[:, :, 0].transpose(0, 2, 1, 3))
+    k = np.ascontiguousarray(qkv[:, :, 1].transpose(0, 2, 1, 3))
+    v = np.ascontiguousarray(qkv[:, :, 2].transpose(0, 2, 1, 3))
+    # scores = Q K^T * (d_q d_k / sqrt(d)), rounded to the activation dtype
+    alpha_qk = f32(f32(p["d_q"]) * f32(p["d_k"])) / f32(np.sqrt(f32(d)))
+    _, out["scores"] = w8a8_bmm(q, k, float(alpha_qk), out_dtype=dtype)
+    # causal softmax in floating point, P quantised with the fixed step 1/127
+    Pq = np.empty((B, H, S, S), np.int8)
+    for b in range(B):
+        for h in range(H):
+            Pq[b, h], _ = softmax_quant_p(out["scores"][b, h])
+    out["P"] = Pq
+    # attention output = P V * (d_v / 127), re-quantised with the out-projection's static input step
+    alpha_pv = f32(p["d_v"]) / f32(127.0)
+    _, o = w8a8_bmm(Pq, v, float(alpha_pv), b_is_kn=True, requant_mul=f32(1) / f32(p["d_attn"]))
+    out["attn"] = np.ascontiguousarray(o.transpose(0, 2, 1, 3)).reshape(B * S, hid)
+    # out-projection -> activation dtype, residual add
+    _, out["proj"] = w8a8_linear(out["attn"], p["d_attn"], p["out_proj"]["Wq"], p["out_proj"]["w_scale"],
+                                 bias=p["out_proj"]["bias"], out_dtype=dtype)
+    out["h"] = round_to(_f32(x) + out["proj"], dtype)
+    # LN2 (smoothing folded) -> INT8; FC1 + ReLU -> INT8; FC2 -> activation dtype; residual add
+    out["x2q"], _, _ = ln_quant(out["h"], p["g2"], p["b2"], eps, "per_tensor_static", static_scale=p["d_ln2"])
+    _, out["f1q"] = w8a8_linear(out["x2q"], p["d_ln2"], p["fc1"]["Wq"], p["fc1"]["w_scale"], bias=p["fc1"]["bias"],
+                                relu=True, requant_mul=f32(1) / f32(p["d_fc1"]))
+    _, out["fc2"] = w8a8_linear(out["f1q"], p["d_fc1"], p["fc2"]["Wq"], p["fc2"]["w_scale"], bias=p["fc2"]["bias"],
+                                out_dtype=dtype)
+    out["y"] = round_to(out["h"] + out["fc2"], dtype)
+    return out

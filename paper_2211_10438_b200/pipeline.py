@@ -114,3 +114,70 @@ def synth_device_weights(N, K, dtype, seed, std=0.02, device="cuda"):
     g = torch.Generator(device=device)
     g.manual_seed(int(seed))
     return (torch.randn((N, K), generator=g, device=device, dtype=torch.float32) * std).to(dtype)
+
+
+class DecoderBlockStatic:
+    """A full W8A8 decoder block with per-tensor STATIC activation steps (level O3), as eleven
+    libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> Q.K^T BMM -> softmax+quantise P ->
+    P.V BMM (INT8 out) -> out-proj GEMM -> residual -> LN2+quantise -> FC1 GEMM (+ReLU, INT8 out)
+    -> FC2 GEMM -> residual.  Q, K, V are read in place from the fused QKV buffer.
+
+    `lin` maps "qkv" / "out_proj" / "fc1" / "fc2" to PreparedLinear; `steps` holds the calibrated
+    static steps d_ln1, d_q, d_k, d_v, d_attn, d_ln2, d_fc1 (python floats)."""
+
+    def __init__(self, lin, steps, B, S, H, d, act_dtype, eps=1e-5):
+        self.lin, self.B, self.S, self.H, self.d, self.dt, self.eps = lin, B, S, H, d, act_dtype, eps
+        dev = lin["qkv"].Wq.device
+        M, hid, ffn = B * S, H * d, lin["fc1"].Wq.shape[0]
+        self.M, self.hid = M, hid
+        f32 = lambda v: torch.tensor([v], dtype=torch.float32, device=dev)
+        self.steps = dict(steps)
+        self.s = {k: f32(v) for k, v in steps.items()}
+        one = torch.tensor(1.0, dtype=torch.float32)
+        inv = lambda v: float(one / torch.tensor(v, dtype=torch.float32))  # fp32 reciprocal, as the oracle takes it
+        self.r_qkv = torch.cat([torch.full((hid,), inv(steps["d_q"])), torch.full((hid,), inv(steps["d_k"])),
+                                torch.full((hid,), inv(steps["d_v"]))]).to(torch.float32).to(dev)
+        self.r_attn = f32(inv(steps["d_attn"]))
+        self.r_fc1 = f32(inv(steps["d_fc1"]))
+        t32 = lambda v: torch.tensor(v, dtype=torch.float32)
+        self.alpha_qk = float((t32(steps["d_q"]) * t32(steps["d_k"])) / torch.sqrt(t32(float(d))))
+        self.alpha_pv = float(t32(steps["d_v"]) / t32(127.0))
+        e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        self.x1q, self.qkv = e((M, hid), torch.int8), e((M, 3 * hid), torch.int8)
+        self.scores, self.P = e((B * H, S, S), act_dtype), e((B * H, S, S), torch.int8)
+        self.attn, self.proj, self.h = e((M, hid), torch.int8), e((M, hid), act_dtype), e((M, hid), act_dtype)
+        self.x2q, self.f1q = e((M, hid), torch.int8), e((M, ffn), torch.int8)
+        self.fc2, self.y = e((M, hid), act_dtype), e((M, hid), act_dtype)
+        self.ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid), dev)
+        self.launches_per_step = 11
+
+    def forward(self, x):
+        L, s, B, S, H, d, hid = self.lin, self.s, self.B, self.S, self.H, self.d, self.hid
+        row = 3 * hid
+        sq.sq_ln_quant(x, L["qkv"].gamma_hat, L["qkv"].beta_hat, self.eps, "per_tensor_static", Xq=self.x1q,
+                       x_scale=s["d_ln1"], workspace=self.ws)
+        sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
+                        requant_mul=self.r_qkv, out=self.qkv)
+        flat = self.qkv.view(-1)
+        sq.sq_w8a8_bmm(flat, flat[hid:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False,
+                       self.alpha_qk, self.scores, (H * S * S, S * S, S), self.ws)
+        sq.sq_softmax_quant_p(self.scores, self.P)
+        sq.sq_w8a8_bmm(self.P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
+                       self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn)
+        sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
+                        bias=L["out_proj"].bias, out=self.proj)
+        sq.sq_residual_add(x, self.proj, out=self.h)
+        sq.sq_ln_quant(self.h, L["fc1"].gamma_hat, L["fc1"].beta_hat, self.eps, "per_tensor_static", Xq=self.x2q,
+                       x_scale=s["d_ln2"], workspace=self.ws)
+        sq.sq_w8a8_gemm(self.x2q, L["fc1"].Wq, s["d_ln2"], L["fc1"].w_scale, self.ws, bias=L["fc1"].bias, relu=True,
+                        requant_mul=self.r_fc1, out=self.f1q)
+        sq.sq_w8a8_gemm(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, bias=L["fc2"].bias,
+                        out=self.fc2)
+        sq.sq_residual_add(self.h, self.fc2, out=self.y)
+        return self.y
+
+    def ops(self):
+        """Integer ops of the four GEMMs and two BMMs of one forward."""
+        M, hid, S, d = self.M, self.hid, self.S, self.d
+        lin = sum(2 * M * l.Wq.shape[0] * l.Wq.shape[1] for l in self.lin.values())
+        return lin + 2 * (2 * self.B * self.H * S * S * d)
