@@ -165,18 +165,91 @@ def timed_rows(device, peaks):
     s = t(lambda: sq.sq_calib_absmax(x, a))
     rows["calib_absmax_16384x20480"] = {"GB/s": 2 * M * C / s / 1e9, "frac_hbm": 2 * M * C / s / 1e9 / peaks["hbm_gbs"]}
     del x, Xq
-    # decode-shaped GEMM, GPT-3 FC1, M = 16 (weights 604 MB > L2)
-    Md, N, K = 16, 49152, 12288
-    Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=device)
-    Xd = torch.randint(-127, 128, (Md, K), dtype=torch.int8, device=device)
-    xsd = torch.rand(Md, device=device) * 0.1
-    wsd = torch.rand(N, device=device) * 0.001
-    Y = torch.empty((Md, N), dtype=torch.bfloat16, device=device)
-    s = t(lambda: sq.sq_w8a8_gemm(Xd, Wq, xsd, wsd, ws, out=Y))
-    byts = N * K + Md * K + 2 * Md * N
-    rows["decode_gemm_M16_49152x12288"] = {"GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6}
-    del Wq
+    # decode-shaped GEMMs at GPT-3 / OPT-175B shapes (weights 453-604 MB > L2); per-token dynamic
+    # quantisation of the bf16 input runs in front of the GEMM and is inside the timed call
+    for name, (N, K) in (("qkv", (36864, 12288)), ("fc1", (49152, 12288)), ("fc2", (12288, 49152))):
+        Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=device)
+        wsd = torch.rand(N, device=device) * 0.001
+        for Md in (1, 16):
+            xd = torch.randn((Md, K), device=device, dtype=torch.bfloat16)
+            Xd = torch.empty((Md, K), dtype=torch.int8, device=device)
+            xsd = torch.empty(Md, dtype=torch.float32, device=device)
+            Y = torch.empty((Md, N), dtype=torch.bfloat16, device=device)
+
+            def call():
+                sq.sq_quant_act(xd, "per_token", Xq=Xd, x_scale=xsd, workspace=ws)
+                sq.sq_w8a8_gemm(Xd, Wq, xsd, wsd, ws, out=Y)
+            s = t(call)
+            byts = N * K + 3 * Md * K + 2 * Md * N
+            rows["decode_%s_M%d_%dx%d" % (name, Md, N, K)] = {
+                "GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6}
+        del Wq
+    # MT-NLG-shaped prefill GEMM (FC1 81920 x 20480 at M = 4096): 13.7 TOP per launch
+    M5, N5, K5 = 4096, 81920, 20480
+    Wq = torch.randint(-127, 128, (N5, K5), dtype=torch.int8, device=device)
+    X5 = torch.randint(-127, 128, (M5, K5), dtype=torch.int8, device=device)
+    xs5 = torch.rand(M5, device=device) * 0.1
+    ws5 = torch.rand(N5, device=device) * 0.001
+    Y5 = torch.empty((M5, N5), dtype=torch.bfloat16, device=device)
+    s = t(lambda: sq.sq_w8a8_gemm(X5, Wq, xs5, ws5, ws, out=Y5), n=5)
+    rows["prefill_gemm_mtnlg_fc1_M4096"] = {"TOPS": 2 * M5 * N5 * K5 / s / 1e12, "us": s * 1e6,
+                                            "frac_of_2x_bf16_sustained": 2 * M5 * N5 * K5 / s / 1e12 / (2 * peaks["bf16_sustained"])}
+    del Wq, X5, Y5
+    rows.update(block_rows(device))
     return rows
+
+
+def block_rows(device):
+    """OPT-30B-shaped full W8A8 decoder block (static steps), one CUDA graph per batch size:
+    microseconds per layer at batch 1, 4, 16 x 512 tokens."""
+    from paper_2211_10438_b200 import pipeline as pl
+    from paper_2211_10438_b200 import synth
+    from paper_2211_10438_b200 import binding as sq
+    wl = synth.WORKLOADS[3]
+    H, d, hid, ffn, S = wl.heads, wl.head_dim, wl.hidden, wl.ffn, wl.extra["seq"]
+    dt = torch.float16
+    ch, fac = wl.outliers()
+    seed = synth.SEED_BASE + 256 * 3
+    ws = sq.new_workspace(4096, device)
+    lin = {}
+    for i, l in enumerate(wl.linears):
+        W = pl.synth_device_weights(l.N, l.K, dt, seed + 10 + i, device=device)
+        b = (torch.randn(l.N, device=device) * 0.01).to(dt)
+        calib = gamma = beta = None
+        if l.ln_input:
+            calib = [pl.synth_device_activations(S, l.K, dt, ch, fac, seed + 30 + 4 * i + j, device) for j in range(4)]
+            gamma = (1 + 0.1 * torch.randn(l.K, device=device)).to(dt)
+            beta = (0.1 * torch.randn(l.K, device=device)).to(dt)
+        lin[l.name] = pl.prepare_linear(l.name, W, b, l.relu, calib, wl.alpha, "per_channel", ws, gamma, beta)
+        del W
+    # static steps from 2 calibration samples of [512, 7168] (the full 128-sample set only changes the values)
+    cal = [pl.synth_device_activations(S, hid, dt, ch, fac, seed + 60 + j, device) for j in range(2)]
+    steps = pl.calibrate_static_steps(lin, cal, 1, S, H, d, dt)
+    out = {}
+    for B in (1, 4, 16):
+        blk = pl.DecoderBlockStatic(lin, steps, B, S, H, d, dt)
+        x = pl.synth_device_activations(B * S, hid, dt, ch, fac, seed + 70 + B, device)
+        for _ in range(3):
+            blk.forward(x)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            blk.forward(x)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 10
+        a.record()
+        for _ in range(n):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / n * 1e3
+        out["opt30b_block_static_b%d_s512" % B] = {"us_per_layer": us, "TOPS": blk.ops() / us / 1e6,
+                                                   "status": sq.device_status(blk.ws)}
+        del blk, g
+    return out
 
 
 def cpu_oracle_step(wl, host, rows):

@@ -181,3 +181,62 @@ class DecoderBlockStatic:
         M, hid, S, d = self.M, self.hid, self.S, self.d
         lin = sum(2 * M * l.Wq.shape[0] * l.Wq.shape[1] for l in self.lin.values())
         return lin + 2 * (2 * self.B * self.H * S * S * d)
+
+
+def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
+    """Static per-tensor steps for DecoderBlockStatic from calibration batches (each [B*S, H*d]):
+    the block is walked with DYNAMIC steps and floating-point intermediates, and the running
+    maximum of every tensor that will later be quantised statically is kept (Section 5.1:
+    smoothing factors and static steps are calibrated once, offline).  Every tensor operation is
+    a libsq call; only the final max-over-batches of a handful of scalars is host bookkeeping."""
+    dev = lin["qkv"].Wq.device
+    M, hid, ffn = B * S, H * d, lin["fc1"].Wq.shape[0]
+    row = 3 * hid
+    ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid), dev)
+    e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+    x1q, xs = e((M, hid), torch.int8), e(1, torch.float32)
+    qkv_f, qkv_q = e((M, row), act_dtype), e((M, row), torch.int8)
+    scores, P = e((B * H, S, S), act_dtype), e((B * H, S, S), torch.int8)
+    attn_f, attn_q = e((M, hid), act_dtype), e((M, hid), torch.int8)
+    proj, h = e((M, hid), act_dtype), e((M, hid), act_dtype)
+    x2q, xs2 = e((M, hid), torch.int8), e(1, torch.float32)
+    f1 = e((M, ffn), act_dtype)
+    mx = {k: 0.0 for k in ("d_ln1", "d_q", "d_k", "d_v", "d_attn", "d_ln2", "d_fc1")}
+    t32 = lambda v: torch.tensor(v, dtype=torch.float32)
+    step = lambda absmax: float(torch.clamp(t32(absmax), min=1e-5) / t32(127.0))
+
+    def tensor_absmax(t, lo=0, hi=None):
+        a = torch.zeros(t.shape[1], dtype=torch.float32, device=dev)
+        sq.sq_calib_absmax(t, a)
+        return float(a[lo:hi].max())
+
+    for x in calib_batches:
+        sq.sq_ln_quant(x, lin["qkv"].gamma_hat, lin["qkv"].beta_hat, eps, "per_tensor_dynamic", Xq=x1q, x_scale=xs,
+                       workspace=ws)
+        sq.sq_w8a8_gemm(x1q, lin["qkv"].Wq, xs, lin["qkv"].w_scale, ws, bias=lin["qkv"].bias, out=qkv_f)
+        d_ln1 = float(xs.item())
+        dq, dk, dv = (step(tensor_absmax(qkv_f, i * hid, (i + 1) * hid)) for i in range(3))
+        one = t32(1.0)
+        r = torch.cat([torch.full((hid,), float(one / t32(v))) for v in (dq, dk, dv)]).to(torch.float32).to(dev)
+        sq.sq_w8a8_gemm(x1q, lin["qkv"].Wq, xs, lin["qkv"].w_scale, ws, bias=lin["qkv"].bias, requant_mul=r, out=qkv_q)
+        flat = qkv_q.view(-1)
+        sq.sq_w8a8_bmm(flat, flat[hid:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False,
+                       float(t32(dq) * t32(dk) / torch.sqrt(t32(float(d)))), scores, (H * S * S, S * S, S), ws)
+        sq.sq_softmax_quant_p(scores, P)
+        sq.sq_w8a8_bmm(P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
+                       float(t32(dv) / t32(127.0)), attn_f, (S * hid, d, hid), ws)
+        d_attn = step(tensor_absmax(attn_f))
+        ra = torch.tensor([float(one / t32(d_attn))], dtype=torch.float32, device=dev)
+        sq.sq_w8a8_bmm(P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
+                       float(t32(dv) / t32(127.0)), attn_q, (S * hid, d, hid), ws, requant_mul=ra)
+        da = torch.tensor([d_attn], dtype=torch.float32, device=dev)
+        sq.sq_w8a8_gemm(attn_q, lin["out_proj"].Wq, da, lin["out_proj"].w_scale, ws, bias=lin["out_proj"].bias, out=proj)
+        sq.sq_residual_add(x, proj, out=h)
+        sq.sq_ln_quant(h, lin["fc1"].gamma_hat, lin["fc1"].beta_hat, eps, "per_tensor_dynamic", Xq=x2q, x_scale=xs2,
+                       workspace=ws)
+        sq.sq_w8a8_gemm(x2q, lin["fc1"].Wq, xs2, lin["fc1"].w_scale, ws, bias=lin["fc1"].bias, relu=True, out=f1)
+        d_fc1 = step(tensor_absmax(f1))
+        for k, v in (("d_ln1", d_ln1), ("d_q", dq), ("d_k", dk), ("d_v", dv), ("d_attn", d_attn),
+                     ("d_ln2", float(xs2.item())), ("d_fc1", d_fc1)):
+            mx[k] = max(mx[k], v)
+    return mx
