@@ -148,7 +148,7 @@ def timed_rows(device, peaks):
         torch.cuda.synchronize()
         return a.elapsed_time(b) / n * 1e-3
 
-    ws = sq.new_workspace(1 << 20, device)
+    ws = sq.new_workspace(max(1 << 20, sq.workspace_bytes(sq.SQ_OP_GEMM, 16, 49152, 49152)), device)
     # MT-NLG-shaped streaming rows (inputs 671 MB > L2)
     M, C = 16384, 20480
     x = torch.randn((M, C), device=device, dtype=torch.bfloat16)

@@ -60,12 +60,13 @@ const char* sq_status_str(sq_status s) {
 }
 
 size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K) {
-    (void)N; (void)K;
+    (void)K;
     switch (op) {
         case SQ_OP_LN_QUANT: return kWsHeader + (size_t)(M > 0 ? M : 0) * 2 * sizeof(float);
+        case SQ_OP_GEMM:  // decode-shaped calls keep split-K partial sums in the workspace
+            return (M > 0 && M <= 16 && N > 0) ? decode_workspace_bytes(N) : kWsHeader;
         case SQ_OP_QUANT_ACT:
         case SQ_OP_QUANT_WEIGHT:
-        case SQ_OP_GEMM:
         case SQ_OP_BMM: return kWsHeader;
     }
     return kWsHeader;
@@ -162,6 +163,7 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
     if (K % 16 != 0 || !aligned16(Xq) || !aligned16(Wq)) return SQ_ERR_ALIGN;
     if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_GEMM, M, N, K))) return SQ_ERR_WORKSPACE;
     GemmArgs a{};
+    a.ws_bytes = ws_bytes;
     a.A = Xq; a.B = Wq;
     a.batch = 1; a.heads = 1; a.M = M; a.N = N; a.K = K;
     a.strideA[0] = M * K; a.strideA[1] = M * K; a.strideA[2] = K;
@@ -200,6 +202,7 @@ sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t h
     if (strideA[2] < K || strideB[2] < (b_is_kn ? N : K) || strideC[2] < N) return SQ_ERR_SHAPE;
     if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_BMM, M, N, K))) return SQ_ERR_WORKSPACE;
     GemmArgs a{};
+    a.ws_bytes = ws_bytes;
     a.A = A; a.B = B;
     a.batch = batch; a.heads = heads; a.M = M; a.N = N; a.K = K;
     for (int i = 0; i < 3; ++i) { a.strideA[i] = strideA[i]; a.strideB[i] = strideB[i]; a.strideC[i] = strideC[i]; }

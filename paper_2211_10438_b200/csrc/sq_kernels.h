@@ -58,8 +58,14 @@ struct GemmArgs {
     float* row_absmax_out;
     void* C; sq_dtype out_dt;
     int64_t strideC[3];   // batch, head, row (elements)
-    uint32_t* status;     // device status word
+    uint32_t* status;     // device status word (= workspace base)
+    size_t ws_bytes;      // size of the caller's workspace
 };
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
+
+// Decode-shaped path (M <= 16): swapped operands, split-K with INT32 scratch in the workspace.
+size_t decode_workspace_bytes(int64_t N);
+bool decode_supports(const GemmArgs& a);
+sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st);
 
 }  // namespace sq

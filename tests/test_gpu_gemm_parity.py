@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def ws():
-    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 4096, 32768, 32768))
+    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 16, 65536, 32768))  # decode scratch is the largest
     yield w
     assert sq.device_status(w) == 0, "a device-side wait timed out"
 
@@ -104,6 +104,39 @@ def test_gemm_strided_output(ws):
     got = host(buf)
     assert np.array_equal(got[:, :N], want)
     assert np.all(got[:, N:] == -7.0)  # nothing written beyond the N columns
+
+
+# decode-shaped calls (M <= 16): swapped operands, K splits with INT32 scratch in the workspace
+DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
+                 (16, 36864, 1024), (2, 4096, 49152)]
+
+
+@pytest.mark.parametrize("M,N,K", DECODE_SHAPES)
+def test_decode_gemm_exact_and_workspace_restored(ws, M, N, K):
+    Xq = synth.int8_tensor(25, 1, (M, K))
+    Wq = synth.int8_tensor(25, 2, (N, K))
+    rng = synth.rng_for(25, 3)
+    xs = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = synth.bias(25, 4, N, "bf16", std=0.5)
+    want_acc = oracle.gemm_i32(Xq, Wq)
+    Xd, Wd = dev(Xq), dev(Wq)
+    for _ in range(2):  # the second call must find the scratch zeroed by the first
+        acc = sq.sq_w8a8_gemm(Xd, Wd, None, None, ws, out_dtype=torch.int32)
+        assert np.array_equal(host(acc), want_acc)
+        y = sq.sq_w8a8_gemm(Xd, Wd, dev(xs), dev(wsc), ws, bias=dev(bias, "bf16"), relu=True, out_dtype=torch.bfloat16)
+        want = oracle.round_to(oracle.dequant(want_acc, xs, wsc, bias, relu=True), "bf16")
+        assert np.array_equal(host(y), want)
+    assert sq.device_status(ws) == 0
+    assert not ws[4:].any(), "workspace not handed back zero-filled"
+
+
+def test_decode_gemm_without_scratch_falls_back_to_single_split():
+    M, N, K = 4, 256, 8192
+    Xq, Wq = synth.int8_tensor(25, 5, (M, K)), synth.int8_tensor(25, 6, (N, K))
+    small = sq.new_workspace(256)
+    with pytest.raises(sq.SqError):  # the documented size is required
+        sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, small, out_dtype=torch.int32)
 
 
 @pytest.mark.parametrize("out", ["f16", "i8", "i32"])
