@@ -31,6 +31,9 @@ import torch
 WORKLOAD = 2  # OPT-13B-shaped prefill linears
 SAMPLE_ROWS_BASELINE = 256
 SAMPLE_ROWS_REFERENCE = 64
+# dram__bytes_read.sum + dram__bytes_write.sum per gemm_i8_kernel launch, mean over the four GEMMs of one step,
+# from the ncu capture summarised in profiles/gemm_i8_kernel__opt13b_prefill.md
+GEMM_DRAM_BYTES_PER_LAUNCH = 146.5e6
 
 
 def measured_peaks():
@@ -435,7 +438,7 @@ def main():
                      "peak_source": "2 x %s bf16 sustained (%s); int8:bf16 nominal ratio 2" % (peaks["bf16_sustained"], peaks["source"]),
                      "frac_of_2x_bf16_burst": achieved / (2 * peaks["bf16_burst"]), "frac_of_nominal_4500": achieved / 4500.0,
                      "per_gemm_us": {k: statistics.mean(v) * 1e6 for k, v in gemm_s.items()},
-                     "traffic": None},
+                     "traffic": GEMM_DRAM_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": block.gemm_bytes() / 4},
         "offline_setup_s": offline_s,
     }
     if rank == 0 and world == 1 and not args.no_rows:

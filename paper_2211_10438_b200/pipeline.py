@@ -98,6 +98,11 @@ class LinearBlock:
     def gemm_ops(self):
         return sum(2 * self.M * l.Wq.shape[0] * l.Wq.shape[1] for l in self.lin.values())
 
+    def gemm_bytes(self):
+        """Algorithmic bytes of the four GEMMs: M*K + N*K (INT8) + M*N outputs in the activation dtype."""
+        return sum(self.M * l.Wq.shape[1] + l.Wq.shape[0] * l.Wq.shape[1] + 2 * self.M * l.Wq.shape[0]
+                   for l in self.lin.values())
+
 
 def synth_device_activations(M, C, dtype, channels, factors, seed, device="cuda"):
     """Device-side draw of the outlier-channel activation model (inputs only, no method math)."""
