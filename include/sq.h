@@ -226,10 +226,14 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
  * most 128 (the head dimension).  alpha carries the operands' static step sizes (and
  * 1/sqrt(d) for Q.K^T).  requant_mul: device pointer to one fp32, required iff out_dt == SQ_I8.
  * Strided views let Q, K, V be read in place from the fused QKV GEMM output [T, 3*H*d].
+ * causal != 0 declares causal self-attention (M == number of keys).  For Q.K^T, score tiles that
+ * lie entirely above the diagonal (first key > last query of the tile) are then neither computed
+ * nor written -- sq_softmax_quant_p never reads them.  For P.V, where P is zero above the
+ * diagonal, the K slices beyond a tile's last query are skipped; the result is unchanged.
  */
 sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M,
                       int64_t N, int64_t K, const int64_t strideA[3], const int64_t strideB[3],
-                      int b_is_kn, float alpha, const float* requant_mul, void* C, sq_dtype out_dt,
+                      int b_is_kn, int causal, float alpha, const float* requant_mul, void* C, sq_dtype out_dt,
                       const int64_t strideC[3], void* workspace, size_t ws_bytes, void* stream);
 
 /*

@@ -62,7 +62,7 @@ def lib():
         L.sq_ln_quant.argtypes = [vp, i32, i64, i64, vp, vp, f32, i32, vp, vp, vp, vp, sz, vp]
         L.sq_w8a8_gemm.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, i32, vp, i32, i32, vp, i32, vp,
                                    vp, i32, i64, vp, sz, vp]
-        L.sq_w8a8_bmm.argtypes = [vp, vp, i64, i64, i64, i64, i64, c.POINTER(i64), c.POINTER(i64), i32,
+        L.sq_w8a8_bmm.argtypes = [vp, vp, i64, i64, i64, i64, i64, c.POINTER(i64), c.POINTER(i64), i32, i32,
                                   f32, vp, vp, i32, c.POINTER(i64), vp, sz, vp]
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
         L.sq_residual_add.argtypes = [vp, vp, i32, i64, vp, vp]
@@ -202,12 +202,13 @@ def sq_w8a8_gemm(Xq, Wq, x_scale, w_scale, workspace, bias=None, relu=False, req
 
 
 def sq_w8a8_bmm(A, B, batch, heads, M, N, K, strideA, strideB, b_is_kn, alpha, C, strideC, workspace,
-                requant_mul=None):
+                requant_mul=None, causal=False):
     """A, B, C are base tensors (any shape); strides are (batch, head, row) in elements."""
     arr = ctypes.c_int64 * 3
     wp, wn = _ws(workspace)
     _check(lib().sq_w8a8_bmm(_ptr(A), _ptr(B), batch, heads, M, N, K, arr(*strideA), arr(*strideB),
-                             1 if b_is_kn else 0, float(alpha), _ptr(requant_mul), _ptr(C), _DT[C.dtype],
+                             1 if b_is_kn else 0, 1 if causal else 0, float(alpha), _ptr(requant_mul), _ptr(C),
+                             _DT[C.dtype],
                              arr(*strideC), wp, wn, _stream()), "sq_w8a8_bmm")
     return C
 

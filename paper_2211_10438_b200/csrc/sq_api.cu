@@ -183,7 +183,8 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
 }
 
 sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M, int64_t N,
-                      int64_t K, const int64_t strideA[3], const int64_t strideB[3], int b_is_kn, float alpha,
+                      int64_t K, const int64_t strideA[3], const int64_t strideB[3], int b_is_kn, int causal,
+                      float alpha,
                       const float* requant_mul, void* C, sq_dtype out_dt, const int64_t strideC[3],
                       void* workspace, size_t ws_bytes, void* stream) {
     if (batch < 0 || heads < 0 || M < 0 || N < 0 || K < 0) return SQ_ERR_SHAPE;
@@ -207,6 +208,7 @@ sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t h
     a.batch = batch; a.heads = heads; a.M = M; a.N = N; a.K = K;
     for (int i = 0; i < 3; ++i) { a.strideA[i] = strideA[i]; a.strideB[i] = strideB[i]; a.strideC[i] = strideC[i]; }
     a.b_is_kn = b_is_kn ? 1 : 0;
+    a.causal = causal ? 1 : 0;
     a.x_scale = nullptr; a.x_per_row = 0;
     a.w_scale = nullptr; a.w_per_col = 0;
     a.alpha = alpha;

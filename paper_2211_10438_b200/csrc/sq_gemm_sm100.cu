@@ -25,22 +25,25 @@ namespace {
 
 using namespace tc;
 
-constexpr int NUM_THREADS = 192;
 
-template <int BLOCK_N, int CG>
+// EW: epilogue warps, 4 (one per TMEM lane quarter) or 8 (two per quarter, each taking half the
+// columns -- for short reductions, where draining the accumulator is the bottleneck).
+template <int BLOCK_N, int CG, int EW>
 struct Cfg {
+    static constexpr int NUM_THREADS = EW * 32 + 64;  // + TMA producer warp + MMA/TMEM warp
+    static constexpr int EPI_THREADS = EW * 32;
     static constexpr int B_ROWS = BLOCK_N / CG;  // rows of B this CTA loads per K slice
     static constexpr int A_BYTES = BLOCK_M * BLOCK_K;
     static constexpr int B_BYTES = B_ROWS * BLOCK_K;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGING_BYTES = 4 * 32 * 128;  // per epilogue warp: 32 rows x 128 bytes
-    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+    static constexpr int STAGING_BYTES = EW * 32 * 128;  // per epilogue warp: 32 rows x 128 bytes
+    static constexpr int STAGES = ((EW == 8 ? 176 : 192) * 1024) / STAGE_BYTES;
     // column stride between the two accumulator slots (power of two keeps the allocation simple)
     static constexpr int SLOT_COLS = BLOCK_N <= 32 ? 32 : BLOCK_N <= 64 ? 64 : BLOCK_N <= 128 ? 128 : 256;
     static constexpr int TMEM_COLS = 2 * SLOT_COLS;
-    static constexpr int EPI_FLOATS = 3 * BLOCK_N;  // w_scale, bias, requant per column
+    static constexpr int EPI_BYTES = BLOCK_N * 3 * 4;  // per column: w_scale, requant, bias as fp32
     static constexpr int SMEM_BYTES = 1024 /*alignment slack*/ + STAGES * STAGE_BYTES + STAGING_BYTES +
-                                      EPI_FLOATS * 4 + (2 * STAGES + 4) * 8 + 64;
+                                      EPI_BYTES + (2 * STAGES + 4) * 8 + 64;
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(BLOCK_N % (16 * CG) == 0 && BLOCK_N <= 256, "MMA N constraint");
     static_assert(B_ROWS % 8 == 0, "B tile must be whole 8-row swizzle groups");
@@ -53,6 +56,7 @@ struct Params {
     int64_t total_tiles;
     int num_kb;
     int b_is_kn;
+    int causal;  // attention: A = Q (skip score tiles above the diagonal) or A = P (skip K slices right of it)
     // coordinate slot (1..3) of the row / head / batch dimension in each tensor map
     int a_slot_row, a_slot_head, a_slot_batch;
     int b_slot_row, b_slot_head, b_slot_batch;
@@ -85,6 +89,16 @@ __device__ __forceinline__ void tile_coords(int64_t tile, const Params& p, int& 
     ni = (int)(r / band_h);
 }
 
+// Causal attention: a score tile whose first key lies beyond the tile's last query is never
+// needed (softmax masks it), and for P.V the K slices beyond the last query hold only zeros.
+__device__ __forceinline__ bool tile_skipped(const Params& p, int mi, int ni, int tile_m, int block_n) {
+    return p.causal && !p.b_is_kn && (int64_t)ni * block_n > (int64_t)(mi + 1) * tile_m - 1;
+}
+__device__ __forceinline__ int tile_num_kb(const Params& p, int mi, int tile_m) {
+    if (p.causal && p.b_is_kn) return min(p.num_kb, (int)(((int64_t)(mi + 1) * tile_m + BLOCK_K - 1) / BLOCK_K));
+    return p.num_kb;
+}
+
 // ------------------------------------------------------------------------------------
 // Epilogue of one 128 x BLOCK_N accumulator slot: Eq. 2 and the output conversions.
 // Called by the 128 epilogue threads; thread = one accumulator row (TMEM lane).
@@ -96,7 +110,8 @@ template <int BLOCK_N>
 __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
                                               uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
                                               int h, int64_t c_off, const float* s_wscale,
-                                              const float* s_bias, const float* s_requant, int lane) {
+                                              const float* s_bias, const float* s_requant, int lane,
+                                              int cc_begin, int cc_end) {
     const bool row_ok = row < p.M;
     float xs = p.alpha;
     if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
@@ -106,15 +121,13 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
     const int pieces = 8 / chunks_per_store;  // 16-byte pieces one chunk contributes to the row
     int cc_coord[4] = {0, 0, 0, 0};
     cc_coord[p.c_slot_row] = row0_warp; cc_coord[p.c_slot_head] = h; cc_coord[p.c_slot_batch] = b;
+    const bool scalar_scale = p.w_scale == nullptr && p.bias == nullptr;  // attention BMMs: y = acc * alpha
 #pragma unroll 1
-    for (int cc = 0; cc < BLOCK_N / 32; ++cc) {
+    for (int cc = cc_begin; cc < cc_end; ++cc) {
         uint32_t r[32];
         tmem_ld32(taddr + cc * 32, r);  // warp-collective: executed by every lane
         tmem_ld_wait();
         const int64_t ncols = p.N - (col0 + cc * 32);  // valid columns in this chunk
-#ifdef SQ_EXP_NO_STORE  // measurement build: drain TMEM but write nothing
-        if (r[0] != 0x7fffffffu) continue;
-#endif
         // ---- Eq. 2 on the chunk; w[] receives the packed output words ----
         uint32_t w[32];
         int nwords;
@@ -124,12 +137,21 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
             nwords = 32;
         } else {
             float y[32];
+            if (scalar_scale) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float sc = __fmul_rn(xs, s_wscale[cc * 32 + j]);
-                float v = __fmaf_rn(__int2float_rn((int32_t)r[j]), sc, s_bias[cc * 32 + j]);
-                if (p.relu) v = fmaxf(v, 0.0f);
-                y[j] = v;
+                for (int j = 0; j < 32; ++j) {
+                    float v = __fmul_rn(__int2float_rn((int32_t)r[j]), xs);  // == fma(acc, xs * 1, 0)
+                    if (p.relu) v = fmaxf(v, 0.0f);
+                    y[j] = v;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float sc = __fmul_rn(xs, s_wscale[cc * 32 + j]);
+                    float v = __fmaf_rn(__int2float_rn((int32_t)r[j]), sc, s_bias[cc * 32 + j]);
+                    if (p.relu) v = fmaxf(v, 0.0f);
+                    y[j] = v;
+                }
             }
             if (p.row_absmax_out) {
 #pragma unroll
@@ -163,11 +185,12 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
         if (p.c_tma) {
             // ---- staged TMA store: lane = row of the 32 x 128-byte staging tile ----
             const int sub = cc % chunks_per_store;
-            if (sub == 0) {  // previous store must have finished READING the staging tile
+            uint8_t* buf = stg;
+            if (sub == 0) {  // the previous store must have finished READING the staging tile
                 if (lane == 0) tma_store_wait_read();
                 __syncwarp();
             }
-            uint8_t* srow = stg + lane * 128;
+            uint8_t* srow = buf + lane * 128;
 #pragma unroll
             for (int v = 0; v < 8; ++v) {
                 if (v < pieces) {
@@ -182,7 +205,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                 const int64_t gcol = col0 + (int64_t)(cc - sub) * 32;  // first column of the staged group
                 if (lane == 0 && gcol < p.N && row0_warp < p.M) {
                     cc_coord[0] = (int)gcol;
-                    tma_store_4d(tmap_c, stg, cc_coord[0], cc_coord[1], cc_coord[2], cc_coord[3]);
+                    tma_store_4d(tmap_c, buf, cc_coord[0], cc_coord[1], cc_coord[2], cc_coord[3]);
                 }
             }
             continue;
@@ -214,18 +237,18 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
 // ------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N, int CG>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+template <int BLOCK_N, int CG, int EW>
+__global__ void __launch_bounds__(EW * 32 + 64, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_c, const Params p) {
-    using C = Cfg<BLOCK_N, CG>;
+    using C = Cfg<BLOCK_N, CG, EW>;
     extern __shared__ uint8_t smem_raw[];
     // identical layout in both CTAs of a pair (the MMA addresses both with one descriptor)
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* stage_base = smem;
     uint8_t* staging = smem + C::STAGES * C::STAGE_BYTES;  // 1024-byte aligned: swizzle pattern matches TMA's
     float* epi_f = reinterpret_cast<float*>(staging + C::STAGING_BYTES);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(epi_f + C::EPI_FLOATS);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(epi_f) + C::EPI_BYTES);
     uint64_t* empty_bar = full_bar + C::STAGES;
     uint64_t* tmem_full = empty_bar + C::STAGES;
     uint64_t* tmem_empty = tmem_full + 2;
@@ -237,7 +260,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const int rank = CG == 1 ? 0 : (int)cluster_ctarank();  // 0 = even CTA: issues the MMAs
     const int64_t first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
-    if (threadIdx.x == 4 * 32) {
+    if (threadIdx.x == EW * 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
         if (p.c_tma) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_c) : "memory");
@@ -247,20 +270,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(tmem_full + s, 1);
-            mbar_init(tmem_empty + s, EPI_THREADS * CG);  // epilogue threads of the whole group
+            mbar_init(tmem_empty + s, C::EPI_THREADS * CG);  // epilogue threads of the whole group
         }
         *abort_flag = 0u;
         *epi_go = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 5) tmem_alloc<CG>(tmem_holder, C::TMEM_COLS);  // whole warp (in both CTAs of a pair)
+    if (warp == EW + 1) tmem_alloc<CG>(tmem_holder, C::TMEM_COLS);  // whole warp (in both CTAs of a pair)
     tcgen05_fence_before();
     if (CG == 1) __syncthreads(); else cluster_sync_all();  // peers' barriers are live before any remote signal
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    if (warp == 4) {
+    if (warp == EW) {
         // ============================ TMA producer ============================
         if (lane == 0) {
             int stage = 0;
@@ -269,15 +292,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
+                if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
+                const int tile_kb = tile_num_kb(p, mi, BLOCK_M * CG);
                 const int b = bh / p.heads, h = bh - b * p.heads;
                 int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
                 ca[p.a_slot_row] = (mi * CG + rank) * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
                 cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
                 const int b_row0 = ni * BLOCK_N + rank * C::B_ROWS;  // this CTA's share of the B tile
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-#ifdef SQ_EXP_MMA_ONLY  // measurement build: no loads at all (MMA issue ceiling)
-                    break;
-#endif
+                for (int kb = 0; kb < tile_kb; ++kb) {
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
                     uint8_t* sa = stage_base + stage * C::STAGE_BYTES;
                     uint8_t* sb = sa + C::A_BYTES;
@@ -296,7 +318,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == EW + 1) {
         // ============================ MMA issuer (even CTA only) ==============
         if (lane == 0 && rank == 0) {
             const uint32_t idesc = make_idesc(BLOCK_M * CG, BLOCK_N, p.b_is_kn);
@@ -308,13 +330,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             uint32_t slot_phase = 0;
             bool ok = true;
             for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
+                int bh, mi, ni;
+                tile_coords(tile, p, bh, mi, ni);
+                if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
+                const int tile_kb = tile_num_kb(p, mi, BLOCK_M * CG);
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
-                for (int kb = 0; kb < p.num_kb; ++kb) {
-#ifndef SQ_EXP_MMA_ONLY
+                for (int kb = 0; kb < tile_kb; ++kb) {
                     if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 3))) break;
-#endif
                     tcgen05_fence_after();
                     const uint32_t sa = smem_u32(stage_base + stage * C::STAGE_BYTES);
                     const uint32_t sb = sa + C::A_BYTES;
@@ -334,23 +358,26 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
     } else {
-        // ============================ epilogue (warps 0-3) ====================
+        // ============================ epilogue (warps 0 .. EW-1) ===============
+        // warp w reads TMEM lanes 32*(w%4).. (hardware rule) and the column half w/4 of the tile
         float* s_wscale = epi_f;
-        float* s_bias = epi_f + BLOCK_N;
-        float* s_requant = epi_f + 2 * BLOCK_N;
-        const int et = threadIdx.x;  // 0..127
+        float* s_requant = epi_f + BLOCK_N;
+        float* s_bias = epi_f + 2 * BLOCK_N;
+        const int et = threadIdx.x;
+        const int quarter = warp & 3, half = warp >> 2;
         int slot = 0;
         uint32_t slot_phase = 0;
         for (int64_t tile = first_tile; tile < p.total_tiles; tile += tile_step) {
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
+            if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
             const int b = bh / p.heads, h = bh - b * p.heads;
             const int64_t col0 = (int64_t)ni * BLOCK_N;
             // stage this tile's per-column constants
-            for (int c = et; c < BLOCK_N; c += EPI_THREADS) {
+            for (int c = et; c < BLOCK_N; c += C::EPI_THREADS) {
                 const int64_t col = col0 + c;
                 const bool in = col < p.N;
-                float ws = 1.0f, bs = 0.0f, rq = 1.0f;
+                float ws = 1.0f, rq = 1.0f, bs = 0.0f;
                 if (in) {
                     if (p.w_scale) ws = __ldg(p.w_scale + (p.w_per_col ? col : 0));
                     if (p.bias)
@@ -362,24 +389,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             if (et == 0)
                 *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 4) ? 1u : 0u;
-            epi_bar_sync();  // constants staged; verdict of the wait visible to all 128 threads
+            epi_bar_sync<C::EPI_THREADS>();  // constants staged; verdict of the wait visible to all epilogue threads
             if (*epi_go == 0u) break;
             tcgen05_fence_after();
 
-            const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + warp * 32 + lane;
+            const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
             const int64_t c_off = (int64_t)b * p.c_stride_batch + (int64_t)h * p.c_stride_head +
                                   row * p.c_stride_row + col0;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS);
-            const int row0_warp = (mi * CG + rank) * BLOCK_M + warp * 32;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS);
+            const int row0_warp = (mi * CG + rank) * BLOCK_M + quarter * 32;
+            // split the tile's 32-column chunks between the two warps of this lane quarter, in whole
+            // store groups (a staged TMA store covers 128 bytes of a row = 1, 2 or 4 chunks)
+            const int cps = p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2);
+            const int groups = (BLOCK_N / 32 + cps - 1) / cps;
+            const int g_split = EW == 8 ? (groups + 1) / 2 : groups;
+            const int cc_begin = half == 0 ? 0 : g_split * cps;
+            const int cc_end = half == 0 ? min(g_split * cps, BLOCK_N / 32) : BLOCK_N / 32;
             epilogue_slot<BLOCK_N>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
-                                   c_off, s_wscale, s_bias, s_requant, lane);
+                                   c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
 
             // accumulator slot drained: hand it back to the MMA warp (in the even CTA)
             tcgen05_fence_before();
             if (CG == 1) mbar_arrive(tmem_empty + slot); else mbar_arrive_even_cta(tmem_empty + slot);
             slot ^= 1;
             if (slot == 0) slot_phase ^= 1u;
-            epi_bar_sync();  // nobody still reads the staged constants when the next tile overwrites them
+            epi_bar_sync<C::EPI_THREADS>();  // nobody still reads the staged constants when the next tile overwrites them
         }
         if (p.c_tma && lane == 0) tma_store_wait_all();  // this warp's stores have landed before the CTA exits
     }
@@ -389,7 +423,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (*abort_flag) __nanosleep(1000000);  // let copies / MMAs in flight land before freeing
     tcgen05_fence_before();
     if (CG == 1) __syncthreads(); else cluster_sync_all();  // the peer may still signal this CTA's barriers
-    if (warp == 5) {
+    if (warp == EW + 1) {
         tcgen05_fence_after();
         tmem_dealloc<CG>(tmem_base, C::TMEM_COLS);
     }
@@ -398,9 +432,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // ------------------------------------------------------------------------------------
 // Host side: tensor maps + launch
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N, int CG>
-sq_status launch(const GemmArgs& a, cudaStream_t st) {
-    using C = Cfg<BLOCK_N, CG>;
+template <int BLOCK_N, int CG, int EW>
+sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
+    using C = Cfg<BLOCK_N, CG, EW>;
     Params p;
     p.M = a.M; p.N = a.N; p.K = a.K;
     p.heads = (int)a.heads; p.batch = (int)a.batch;
@@ -409,6 +443,7 @@ sq_status launch(const GemmArgs& a, cudaStream_t st) {
     p.total_tiles = (int64_t)p.num_m * p.num_n * a.heads * a.batch;
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     p.b_is_kn = a.b_is_kn;
+    p.causal = a.causal;
     CUtensorMap ma, mb;
     if (!make_map(&ma, a.A, 1, a.K, a.M, a.heads, a.batch, a.strideA[2], a.strideA[1], a.strideA[0], BLOCK_K,
                   BLOCK_M, &p.a_slot_row, &p.a_slot_head, &p.a_slot_batch))
@@ -443,14 +478,14 @@ sq_status launch(const GemmArgs& a, cudaStream_t st) {
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         C::SMEM_BYTES));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int groups = (int)std::min<int64_t>(p.total_tiles, sm_count() / CG);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(groups * CG));
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(C::NUM_THREADS);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -460,11 +495,18 @@ sq_status launch(const GemmArgs& a, cudaStream_t st) {
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = CG > 1 ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BLOCK_N, CG>, ma, mb, mc, p) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BLOCK_N, CG, EW>, ma, mb, mc, p) != cudaSuccess) {
         cudaGetLastError();
         return SQ_ERR_CUDA;
     }
     return launch_status();
+}
+
+// Short reductions (few K slices per tile) are bound by draining the accumulators: give them
+// eight epilogue warps; long ones keep four, which leaves the MMA and TMA lanes more issue slots.
+template <int BLOCK_N, int CG>
+sq_status launch(const GemmArgs& a, cudaStream_t st) {
+    return a.K <= 1024 ? launch_ew<BLOCK_N, CG, 8>(a, st) : launch_ew<BLOCK_N, CG, 4>(a, st);
 }
 
 // Relative cost of covering the problem with tiles of (128*cg) x bn on `sms` SMs: full waves
@@ -488,8 +530,9 @@ sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
     // (narrower tiles move more operand bytes per MAC: 28 KB per 128x192x128 vs 32 KB per 128x256x128)
     const double c256 = tiling_cost(a, 256, 2, sms), c192 = tiling_cost(a, 192, 2, sms) * 1.10,
                  c128 = tiling_cost(a, 128, 2, sms) * 1.25;
-    if (c256 <= c192 && c256 <= c128) return launch<256, 2>(a, st);
-    if (c192 <= c128) return launch<192, 2>(a, st);
+    const bool allow192 = a.out_dt != SQ_I8;  // 192 columns are not a whole number of 128-column INT8 store groups
+    if ((c256 <= c192 || !allow192) && c256 <= c128) return launch<256, 2>(a, st);
+    if (allow192 && c192 <= c128) return launch<192, 2>(a, st);
     return launch<128, 2>(a, st);
 }
 

@@ -49,6 +49,7 @@ struct GemmArgs {
     int64_t strideA[3];   // batch, head, row (elements)
     int64_t strideB[3];
     int b_is_kn;
+    int causal;           // attention BMMs only: skip work above the diagonal
     const float* x_scale; int x_per_row;     // Delta_x[t] or Delta_x
     const float* w_scale; int w_per_col;     // Delta_w[o] or Delta_w; nullptr = 1
     float alpha;                             // used when x_scale == nullptr

@@ -409,6 +409,9 @@ softmax_quant_p_kernel(const T* __restrict__ scores, int64_t n_rows, int S, int8
     const int i = (int)(r % S);  // query position: keys j <= i are visible
     const uint4* srow = reinterpret_cast<const uint4*>(scores + r * S);
     const int nvec = S >> 3;
+    // Only the vectors that hold a visible key (8 * vi <= i) are loaded and exponentiated; the
+    // rest of the row is written as zeros.  exp(s - max) is evaluated as exp2(s * log2(e) -
+    // max * log2(e)) and the division by the row sum as one reciprocal per row.
     float f[VPL][8];
     float mx = -INFINITY;
 #pragma unroll
@@ -421,31 +424,39 @@ softmax_quant_p_kernel(const T* __restrict__ scores, int64_t n_rows, int S, int8
                 if (vi * 8 + k > i) f[v][k] = -INFINITY;
                 mx = fmaxf(mx, f[v][k]);
             }
-        } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) f[v][k] = -INFINITY;
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    const float kLog2e = 1.4426950408889634f;
+    const float shift = -mx * kLog2e;
     float sum = 0.0f;
 #pragma unroll
-    for (int v = 0; v < VPL; ++v)
+    for (int v = 0; v < VPL; ++v) {
+        const int vi = lane + 32 * v;
+        if (vi < nvec && vi * 8 <= i) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            f[v][k] = expf(f[v][k] - mx);  // exp(-inf) = 0 for masked positions
-            sum += f[v][k];
+            for (int k = 0; k < 8; ++k) {
+                f[v][k] = exp2f(fmaf(f[v][k], kLog2e, shift));  // exp2(-inf) = 0 for masked positions
+                sum += f[v][k];
+            }
         }
+    }
     sum = warp_sum(sum);
+    const float inv = __fdiv_rn(1.0f, sum);
     uint2* prow = reinterpret_cast<uint2*>(Pq + r * S);
 #pragma unroll
     for (int v = 0; v < VPL; ++v) {
         const int vi = lane + 32 * v;
         if (vi < nvec) {
-            float p[8];
+            if (vi * 8 <= i) {
+                float p[8];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) p[k] = __fdiv_rn(f[v][k], sum);
-            __stcs(prow + vi, quant8(p, 127.0f));
+                for (int k = 0; k < 8; ++k) p[k] = f[v][k] * inv;
+                __stcs(prow + vi, quant8<false>(p, 127.0f));  // p <= 1: the code cannot exceed 127
+            } else {
+                __stcs(prow + vi, make_uint2(0u, 0u));
+            }
         }
     }
 }

@@ -13,7 +13,6 @@ namespace tc {
 constexpr int BLOCK_M = 128;  // accumulator rows per CTA (TMEM lanes)
 constexpr int BLOCK_K = 128;  // INT8 elements = bytes: exactly one 128-byte swizzle row
 constexpr int UMMA_K = 32;    // K per tcgen05.mma for 8-bit operands
-constexpr int EPI_THREADS = 128;
 constexpr uint32_t kWaitCycles = 2000000000u;  // ~1 s at B200 clocks
 constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu; // clears the CTA-rank bit of a shared::cluster address:
                                                // the same offset in the EVEN CTA of the pair
@@ -160,8 +159,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tmem_ld_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+template <int THREADS>
 __device__ __forceinline__ void epi_bar_sync() {
-    asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS) : "memory");
 }
 template <int CG>
 __device__ __forceinline__ void tmem_alloc(uint32_t* holder, uint32_t cols) {
@@ -214,7 +214,7 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, const void*
                  : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-__device__ __forceinline__ void tma_store_wait_read() {  // staging buffer may be overwritten again
+__device__ __forceinline__ void tma_store_wait_read() {  // staging tile may be overwritten again
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 __device__ __forceinline__ void tma_store_wait_all() {

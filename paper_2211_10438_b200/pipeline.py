@@ -165,10 +165,10 @@ class DecoderBlockStatic:
                         requant_mul=self.r_qkv, out=self.qkv)
         flat = self.qkv.view(-1)
         sq.sq_w8a8_bmm(flat, flat[hid:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False,
-                       self.alpha_qk, self.scores, (H * S * S, S * S, S), self.ws)
+                       self.alpha_qk, self.scores, (H * S * S, S * S, S), self.ws, causal=True)
         sq.sq_softmax_quant_p(self.scores, self.P)
         sq.sq_w8a8_bmm(self.P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
-                       self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn)
+                       self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn, causal=True)
         sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
                         bias=L["out_proj"].bias, out=self.proj)
         sq.sq_residual_add(x, self.proj, out=self.h)

@@ -75,8 +75,8 @@ def test_gemm_dequant_epilogue(ws, dtype, M, N, K, per_token, per_channel, use_b
 
 
 @pytest.mark.parametrize("per_col", [False, True])
-def test_gemm_requant_and_row_absmax(ws, per_col):
-    M, N, K = 200, 328, 1024
+@pytest.mark.parametrize("M,N,K", [(200, 328, 1024), (2048, 5120, 256), (1024, 640, 384)])
+def test_gemm_requant_and_row_absmax(ws, per_col, M, N, K):
     Xq = synth.int8_tensor(22, 1, (M, K))
     Wq = synth.int8_tensor(22, 2, (N, K))
     rng = synth.rng_for(22, 3)
@@ -209,3 +209,33 @@ def test_bmm_pv_with_kn_operand(ws, B, H, S, d):
     assert np.array_equal(host(acc), to_rows(want_acc))
     assert np.array_equal(host(o8), to_rows(want_q))
     assert np.array_equal(host(of), to_rows(want_f))
+
+
+@pytest.mark.parametrize("B,H,S,d", [(1, 2, 512, 128), (2, 1, 384, 64), (1, 1, 208, 128)])
+def test_bmm_causal_skips_only_what_attention_never_reads(ws, B, H, S, d):
+    qkv = _qkv_views(B, H, S, d, 7)
+    row = 3 * H * d
+    qkv_d = dev(qkv)
+    flat = qkv_d.view(-1)
+    alpha = np.float32(0.004)
+    sentinel = -777.0
+    scores = torch.full((B, H, S, S), sentinel, dtype=torch.float16, device="cuda")
+    sq.sq_w8a8_bmm(flat, flat[H * d:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False, alpha, scores,
+                   (H * S * S, S * S, S), ws, causal=True)
+    q = np.ascontiguousarray(qkv.reshape(B, S, 3, H, d)[:, :, 0].transpose(0, 2, 1, 3))
+    k = np.ascontiguousarray(qkv.reshape(B, S, 3, H, d)[:, :, 1].transpose(0, 2, 1, 3))
+    v = np.ascontiguousarray(qkv.reshape(B, S, 3, H, d)[:, :, 2].transpose(0, 2, 1, 3))
+    _, want = oracle.w8a8_bmm(q, k, alpha, out_dtype="f16")
+    got = host(scores)
+    tril = np.tril(np.ones((S, S), bool))
+    assert np.array_equal(got[..., tril], want[..., tril])  # every score a causal softmax reads
+    upper = got[..., ~tril]
+    assert np.all((upper == sentinel) | (upper == want[..., ~tril]))  # the rest: computed or left alone
+    # P.V with a lower-triangular P: causal K-slice skipping leaves the result unchanged
+    P = np.tril(synth.int8_tensor(24, 8, (B, H, S, S), lo=0, hi=127))
+    a2 = np.float32(2.5e-4)
+    acc = torch.empty((B * S, H * d), dtype=torch.int32, device="cuda")
+    sq.sq_w8a8_bmm(dev(P), flat[2 * H * d:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True, a2, acc,
+                   (S * H * d, d, H * d), ws, causal=True)
+    want_acc, _ = oracle.w8a8_bmm(P, v, a2, b_is_kn=True, out_dtype="f16")
+    assert np.array_equal(host(acc), want_acc.transpose(0, 2, 1, 3).reshape(B * S, H * d))

@@ -68,9 +68,9 @@ def test_validation_without_cuda(lib):
     assert args(64, out_dt=sq.SQ_I8) == 1
     assert args(64, rq=p) == 1
     arr = ctypes.c_int64 * 3
-    assert lib.sq_w8a8_bmm(i8, i8, 1, 1, 16, 256, 64, arr(0, 0, 64), arr(0, 0, 256), 1, 1.0, None, p,
+    assert lib.sq_w8a8_bmm(i8, i8, 1, 1, 16, 256, 64, arr(0, 0, 64), arr(0, 0, 256), 1, 0, 1.0, None, p,
                            sq.SQ_F16, arr(0, 0, 256), ws, 256, None) == 4  # [K,N] B limited to N <= 128
-    assert lib.sq_w8a8_bmm(i8, i8, 1, 1, 16, 64, 64, arr(0, 0, 72), arr(0, 0, 64), 0, 1.0, None, p,
+    assert lib.sq_w8a8_bmm(i8, i8, 1, 1, 16, 64, 64, arr(0, 0, 72), arr(0, 0, 64), 0, 0, 1.0, None, p,
                            sq.SQ_F16, arr(0, 0, 64), ws, 256, None) == 3  # stride not a multiple of 16
 
 
