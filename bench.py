@@ -29,7 +29,7 @@ import numpy as np
 import torch
 
 WORKLOAD = 2  # OPT-13B-shaped prefill linears
-SAMPLE_ROWS_BASELINE = 256
+SAMPLE_ROWS_BASELINE = 1024
 SAMPLE_ROWS_REFERENCE = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per gemm_i8_kernel launch, mean over the four GEMMs of one step,
 # from the ncu capture summarised in profiles/gemm_i8_kernel__opt13b_prefill.md
