@@ -99,6 +99,13 @@ class ClockSampler:
                 "samples": len(self.samples), "reasons": sorted(self.reasons)}
 
 
+def aggregate_replicas(ops_per_step, steps, elapsed_local_s, world, reduce_max):
+    """Whole-job throughput of `world` independent replicas: every rank did ops_per_step * steps,
+    the job took as long as its slowest rank (reduce_max = max over ranks of a python float)."""
+    elapsed = reduce_max(elapsed_local_s)
+    return world * ops_per_step * steps / elapsed / 1e12, elapsed
+
+
 def build_block(device, seed_offset=0):
     """Seeded synthetic OPT-13B-shaped block: weights N(0, 0.02), outlier-channel activations."""
     from paper_2211_10438_b200 import binding as sq
@@ -381,7 +388,8 @@ def main():
         block.step(x_in, attn_out)
     e1.record()
     barrier()
-    elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
+    ops_step = block.gemm_ops()
+    value, elapsed = aggregate_replicas(ops_step, args.steps, e0.elapsed_time(e1) * 1e-3, world, max_over_ranks)
     clocks = sampler.stop()
     gemm_s = {}
     for name, (a, b) in block.gemm_events:
@@ -390,8 +398,6 @@ def main():
     status = sq.device_status(block.ws)
     if status != 0:
         raise SystemExit("device status word = %d: a bounded wait expired" % status)
-    ops_step = block.gemm_ops()
-    value = world * ops_step * args.steps / elapsed / 1e12
     gemm_total = sum(sum(v) for v in gemm_s.values())
     achieved = ops_step * args.steps / gemm_total / 1e12
     peak_tops = 2.0 * peaks["bf16_sustained"]
@@ -416,8 +422,7 @@ def main():
         e2e_step()
     e1.record()
     barrier()
-    e2e_elapsed = max_over_ranks(e0.elapsed_time(e1) * 1e-3)
-    e2e_value = world * ops_step * args.steps / e2e_elapsed / 1e12
+    e2e_value, e2e_elapsed = aggregate_replicas(ops_step, args.steps, e0.elapsed_time(e1) * 1e-3, world, max_over_ranks)
 
     out = {
         "metric": "W8A8 linear-layer throughput (4 GEMMs + activation quantisation)",

@@ -389,7 +389,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             if (et == 0)
                 *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 4) ? 1u : 0u;
-            epi_bar_sync<C::EPI_THREADS>();  // constants staged; verdict of the wait visible to all epilogue threads
+            epi_bar_sync<C::EPI_THREADS>();  // constants staged; outcome of the wait visible to all epilogue threads
             if (*epi_go == 0u) break;
             tcgen05_fence_after();
 

@@ -137,7 +137,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     int s = 0;
     uint32_t parity = 0;
     for (int64_t row = first; row < M; row += stride) {
-        // One thread waits (bounded) for the row's bulk copy; its verdict reaches the group through
+        // One thread waits (bounded) for the row's bulk copy; its outcome reaches the group through
         // shared memory so that every thread takes the same branch.
         if (gt == 0) {
             const bool ok = mbar_wait_bounded(my_full + s, parity);
