@@ -53,7 +53,9 @@ struct Params {
     int64_t M, N, K;
     int heads, batch;
     int num_m, num_n;  // tiles per matrix (num_m counts tiles of 128*CG rows)
-    int64_t total_tiles;
+    uint32_t total_tiles, per_mat;  // tiles over all matrices / per matrix (after causal compaction)
+    int causal_compact;             // per-matrix tiles are enumerated through causal_prefix (num_m <= 32)
+    uint32_t causal_prefix[33];     // first compact tile index of every m tile
     int num_kb;
     int b_is_kn;
     int causal;  // attention: A = Q (skip score tiles above the diagonal) or A = P (skip K slices right of it)
@@ -76,17 +78,28 @@ struct Params {
 
 // tile id -> (batch*heads index, m tile, n tile).  Within one matrix, tiles are visited in
 // bands of G m-tiles so that the CTAs running at the same time share A and B tiles in L2.
-__device__ __forceinline__ void tile_coords(int64_t tile, const Params& p, int& bh, int& mi, int& ni) {
-    const int64_t per_mat = (int64_t)p.num_m * p.num_n;
-    bh = (int)(tile / per_mat);
-    const int64_t t = tile - (int64_t)bh * per_mat;
-    constexpr int G = 8;
-    const int64_t band_tiles = (int64_t)G * p.num_n;
-    const int band = (int)(t / band_tiles);
-    const int band_h = min(G, p.num_m - band * G);
-    const int64_t r = t - (int64_t)band * band_tiles;
-    mi = band * G + (int)(r % band_h);
-    ni = (int)(r / band_h);
+// (32-bit arithmetic: with a single K slice per tile this runs on the critical path of the
+// single-lane producer and MMA roles.)  For causal score matrices only the tiles on or below the
+// diagonal are enumerated, so every CTA gets the same share of real work.
+__device__ __forceinline__ void tile_coords(uint32_t tile, const Params& p, int& bh, int& mi, int& ni) {
+    const uint32_t b = tile / p.per_mat;
+    const uint32_t t = tile - b * p.per_mat;
+    bh = (int)b;
+    if (p.causal_compact) {
+        int m = 0;
+        while (t >= p.causal_prefix[m + 1]) ++m;
+        mi = m;
+        ni = (int)(t - p.causal_prefix[m]);
+        return;
+    }
+    constexpr uint32_t G = 8;
+    const uint32_t band_tiles = G * (uint32_t)p.num_n;
+    const uint32_t band = t / band_tiles;
+    const uint32_t band_h = min(G, (uint32_t)p.num_m - band * G);
+    const uint32_t r = t - band * band_tiles;
+    const uint32_t q = r / band_h;
+    mi = (int)(band * G + (r - q * band_h));
+    ni = (int)q;
 }
 
 // Causal attention: a score tile whose first key lies beyond the tile's last query is never
@@ -258,7 +271,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = CG == 1 ? 0 : (int)cluster_ctarank();  // 0 = even CTA: issues the MMAs
-    const int64_t first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
+    const uint32_t first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
 
     if (threadIdx.x == EW * 32) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
@@ -289,7 +302,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
+            for (uint32_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -329,7 +342,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
-            for (int64_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
+            for (uint32_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -367,7 +380,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int quarter = warp & 3, half = warp >> 2;
         int slot = 0;
         uint32_t slot_phase = 0;
-        for (int64_t tile = first_tile; tile < p.total_tiles; tile += tile_step) {
+        for (uint32_t tile = first_tile; tile < p.total_tiles; tile += tile_step) {
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
             if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -440,7 +453,23 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     p.heads = (int)a.heads; p.batch = (int)a.batch;
     p.num_m = (int)((a.M + BLOCK_M * CG - 1) / (BLOCK_M * CG));
     p.num_n = (int)((a.N + BLOCK_N - 1) / BLOCK_N);
-    p.total_tiles = (int64_t)p.num_m * p.num_n * a.heads * a.batch;
+    // tiles per matrix; for causal score matrices only those on or below the diagonal
+    p.causal_compact = 0;
+    p.per_mat = (uint32_t)p.num_m * (uint32_t)p.num_n;
+    if (a.causal && !a.b_is_kn && p.num_m <= 32) {
+        p.causal_compact = 1;
+        uint32_t acc = 0;
+        for (int mi = 0; mi < p.num_m; ++mi) {
+            p.causal_prefix[mi] = acc;
+            const int64_t last_query = (int64_t)(mi + 1) * BLOCK_M * CG - 1;
+            acc += (uint32_t)std::min<int64_t>(p.num_n, last_query / BLOCK_N + 1);
+        }
+        p.causal_prefix[p.num_m] = acc;
+        p.per_mat = acc;
+    }
+    const int64_t total = (int64_t)p.per_mat * a.heads * a.batch;
+    if (total >= (int64_t)1 << 31) return SQ_ERR_UNSUPPORTED;
+    p.total_tiles = (uint32_t)total;
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     p.b_is_kn = a.b_is_kn;
     p.causal = a.causal;
@@ -482,7 +511,7 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
                                         C::SMEM_BYTES));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const int groups = (int)std::min<int64_t>(p.total_tiles, sm_count() / CG);
+    const int groups = (int)std::min<int64_t>((int64_t)p.total_tiles, sm_count() / CG);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(groups * CG));
     cfg.blockDim = dim3(C::NUM_THREADS);
