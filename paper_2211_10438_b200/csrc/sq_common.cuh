@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/sq.h"
 
 namespace sq {
@@ -144,6 +146,48 @@ __device__ __forceinline__ float block_reduce(float v, float* red) {
     }
     __syncthreads();
     return red[32];
+}
+
+// ---------------------------------------------------------------------------------------
+// Programmatic dependent launch.  The runtime kernels of the path are launched with the
+// programmatic-stream-serialisation attribute: a kernel may be scheduled while its predecessor
+// in the stream is still draining, runs its set-up (barriers, tensor memory, descriptor and
+// weight prefetch) and then blocks in pdl_wait() until the predecessor has completed and its
+// writes are visible.  No global memory that an earlier kernel produces or still reads may be
+// touched before pdl_wait().  Both instructions are no-ops for ordinary launches.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+inline sq_status launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                            int cluster_x, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    if (cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        return SQ_ERR_CUDA;
+    }
+    return launch_status();
 }
 
 // max for non-negative floats through their (order-preserving) bit patterns

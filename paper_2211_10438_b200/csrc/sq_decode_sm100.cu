@@ -122,6 +122,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     __syncthreads();
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    pdl_launch_dependents();
 
     if (warp == 0) {
         // ============================ TMA producer ============================
@@ -129,10 +130,31 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            // The weights are static, the activations come from the kernel in front (the per-token
+            // quantiser): fill the ring with weight slices first, wait for the predecessor, then
+            // add the activation slices of those stages.
+            int prefetched = 0;
+            bool waited = false;
             for (int64_t u = blockIdx.x; ok && u < p.total_units; u += gridDim.x) {
                 const int ni = (int)(u / p.splits), ks = (int)(u % p.splits);
                 const int kb0 = ks * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                int kb = kb0;
+                if (!waited) {
+                    const int n_pre = min(DEC_STAGES, kb1 - kb0);
+                    for (int i = 0; i < n_pre; ++i) {
+                        mbar_expect_tx(full_bar + i, DEC_STAGE);
+                        tma_load_4d<1>(smem + i * DEC_STAGE, &tmap_w, full_bar + i, (kb0 + i) * BLOCK_K, ni * BLOCK_M, 0, 0);
+                    }
+                    pdl_wait();
+                    for (int i = 0; i < n_pre; ++i)
+                        tma_load_4d<1>(smem + i * DEC_STAGE + W_BYTES, &tmap_x, full_bar + i, (kb0 + i) * BLOCK_K, 0, 0, 0);
+                    prefetched = n_pre;
+                    waited = true;
+                    kb = kb0 + n_pre;
+                    stage = n_pre % DEC_STAGES;
+                    phase = (n_pre == DEC_STAGES) ? 1u : 0u;
+                }
+                for (; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 6))) break;
                     uint8_t* sw = smem + stage * DEC_STAGE;
                     mbar_expect_tx(full_bar + stage, DEC_STAGE);
@@ -141,6 +163,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     if (++stage == DEC_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            (void)prefetched;
         }
     } else if (warp == 1) {
         // ============================ MMA issuer ==============================
@@ -177,6 +200,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         }
     } else {
         // ============================ epilogue (warps 2-5) ====================
+        pdl_wait();  // x_scale and the split-K scratch belong to earlier kernels until here
         const int quarter = warp & 3;           // TMEM lanes this warp may read
         const int ch = quarter * 32 + lane;     // output channel within the tile
         const int et = threadIdx.x - 64;        // 0..127
@@ -312,8 +336,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int grid = (int)std::min<int64_t>(p.total_units, sm_count());
-    decode_gemm_kernel<<<grid, DEC_THREADS, DEC_SMEM, st>>>(mw, mx, p);
-    return launch_status();
+    return launch_pdl(decode_gemm_kernel, dim3((unsigned)grid), dim3(DEC_THREADS), (size_t)DEC_SMEM, st, 1, mw, mx, p);
 }
 
 }  // namespace sq

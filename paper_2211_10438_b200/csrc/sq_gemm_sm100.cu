@@ -295,6 +295,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (CG == 1) __syncthreads(); else cluster_sync_all();  // peers' barriers are live before any remote signal
     tcgen05_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    pdl_wait();               // set-up overlapped the previous kernel's tail; its outputs are visible from here on
+    pdl_launch_dependents();
 
     if (warp == EW) {
         // ============================ TMA producer ============================
@@ -512,23 +514,8 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int groups = (int)std::min<int64_t>((int64_t)p.total_tiles, sm_count() / CG);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(groups * CG));
-    cfg.blockDim = dim3(C::NUM_THREADS);
-    cfg.dynamicSmemBytes = C::SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = CG;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = CG > 1 ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<BLOCK_N, CG, EW>, ma, mb, mc, p) != cudaSuccess) {
-        cudaGetLastError();
-        return SQ_ERR_CUDA;
-    }
-    return launch_status();
+    return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
+                      (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, p);
 }
 
 // Short reductions (few K slices per tile) are bound by draining the accumulators: give them

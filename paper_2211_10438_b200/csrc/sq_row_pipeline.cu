@@ -107,6 +107,10 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
         for (int s = 0; s < stages; ++s) mbar_init(my_full + s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    pdl_wait();               // the producer of X (and of the statistics / absmax word) has completed
+    pdl_launch_dependents();  // the next kernel may be scheduled as this one's CTAs drain
+    if (gt == 0) {
         // prologue: fill the ring
         for (int s = 0; s < stages; ++s) {
             const int64_t r = first + (int64_t)s * stride;
@@ -288,10 +292,9 @@ sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, co
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     const int grid = (int)std::min<int64_t>((M + G - 1) / G, sm_count());
-    kern<<<grid, CTA_THREADS, smem, st>>>(static_cast<const T*>(X), M, (int)C, static_cast<const T*>(gamma),
-                                          static_cast<const T*>(beta), eps, mode, stages, Xq, scale, absmax_word,
-                                          stats, stats_are_input, status);
-    return launch_status();
+    return launch_pdl(kern, dim3((unsigned)grid), dim3(CTA_THREADS), smem, st, 1, static_cast<const T*>(X), M,
+                      (int)C, static_cast<const T*>(gamma), static_cast<const T*>(beta), eps, mode, stages, Xq, scale,
+                      absmax_word, stats, stats_are_input, status);
 }
 
 template <typename T, bool LN>
