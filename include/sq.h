@@ -256,6 +256,16 @@ sq_status sq_softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int
 sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out,
                           void* stream);
 
+/*
+ * Self-test of the bounded-wait machinery that every tensor-core kernel of the library uses
+ * (no counterpart in the paper).  Launches one small CTA that waits, with a budget of
+ * `budget_cycles` SM clock cycles, on an mbarrier that nothing will ever complete; when the
+ * budget runs out the kernel stores SQ_ERR_TIMEOUT | (where << 8) into *status_word and returns
+ * normally -- the same path a real kernel takes if a TMA copy or an MMA never signals.  The
+ * context stays usable.  status_word: device pointer to a zero-initialised uint32.
+ */
+sq_status sq_selftest_bounded_wait(uint32_t* status_word, uint32_t budget_cycles, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

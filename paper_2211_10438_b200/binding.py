@@ -24,7 +24,8 @@ SQ_NOALLOC_MAX_ROWS = 16384
 
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
-           "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc"]
+           "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
+           "sq_selftest_bounded_wait"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -67,6 +68,7 @@ def lib():
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
         L.sq_residual_add.argtypes = [vp, vp, i32, i64, vp, vp]
         L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
+        L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = i32
         _lib = L
@@ -244,3 +246,11 @@ def sq_ln_quant_tensor_noalloc(X, gamma_hat, beta_hat, eps, Xq=None, x_scale=Non
                                             float(eps), _ptr(Xq), _ptr(x_scale), _stream()),
            "sq_ln_quant_tensor_noalloc")
     return Xq, x_scale
+
+
+def sq_selftest_bounded_wait(budget_cycles=200000):
+    """Runs the library's bounded-wait self-test; returns the status word the kernel left
+    (SQ_ERR_TIMEOUT | where << 8 when the wait gave up as designed)."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().sq_selftest_bounded_wait(_ptr(word), int(budget_cycles), _stream()), "sq_selftest_bounded_wait")
+    return int(word.item())

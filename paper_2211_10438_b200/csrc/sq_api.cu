@@ -231,6 +231,12 @@ sq_status sq_softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int
     return softmax_quant_p(scores, dt, n_mat, S, Pq, as_stream(stream));
 }
 
+sq_status sq_selftest_bounded_wait(uint32_t* status_word, uint32_t budget_cycles, void* stream) {
+    if (!status_word) return SQ_ERR_INVALID_ARG;
+    if (budget_cycles > 100000000u) return SQ_ERR_INVALID_ARG;  // a self-test never waits longer than ~50 ms
+    return bounded_wait_selftest(status_word, budget_cycles, as_stream(stream));
+}
+
 sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out, void* stream) {
     if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
     if (n < 0) return SQ_ERR_SHAPE;

@@ -536,6 +536,27 @@ double tiling_cost(const GemmArgs& a, int bn, int cg, int sms) {
 
 }  // namespace
 
+namespace {
+// One warp waits on a barrier that never completes; the bounded wait must give up and report.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint32_t budget) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) tc::mbar_wait(&bar, 0u, &abort_flag, status, 15u, budget);
+    __syncthreads();
+}
+}  // namespace
+
+sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, budget);
+    return launch_status();
+}
+
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
     if (decode_supports(a)) return decode_gemm(a, a.status, a.ws_bytes, st);
     // [K, N]-stored B is limited to one 128-byte swizzle row of N per tile

@@ -63,6 +63,7 @@ struct GemmArgs {
     size_t ws_bytes;      // size of the caller's workspace
 };
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
+sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st);
 
 // Decode-shaped path (M <= 16): swapped operands, split-K with INT32 scratch in the workspace.
 size_t decode_workspace_bytes(int64_t N);

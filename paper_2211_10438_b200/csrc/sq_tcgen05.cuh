@@ -63,14 +63,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the CTA's abort flag + the global status word)
 // if the phase does not complete within the cycle budget or another role already aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status, uint32_t where) {
+                                          uint32_t* status, uint32_t where, uint32_t budget = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
-            if ((unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) {
+            if ((unsigned long long)(clock64() - t0) > (unsigned long long)budget) {
                 *abort_flag = 1u;
                 atomicCAS(status, 0u, ((uint32_t)SQ_ERR_TIMEOUT) | (where << 8));
                 return false;
