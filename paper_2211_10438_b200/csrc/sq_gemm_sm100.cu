@@ -525,15 +525,6 @@ sq_status launch(const GemmArgs& a, cudaStream_t st) {
     return a.K <= 1024 ? launch_ew<BLOCK_N, CG, 8>(a, st) : launch_ew<BLOCK_N, CG, 4>(a, st);
 }
 
-// Relative cost of covering the problem with tiles of (128*cg) x bn on `sms` SMs: full waves
-// of tiles times the tile's MMA time, which is proportional to bn.
-double tiling_cost(const GemmArgs& a, int bn, int cg, int sms) {
-    const int64_t tiles = ((a.M + 128 * cg - 1) / (128 * cg)) * ((a.N + bn - 1) / bn) * a.heads * a.batch;
-    const int64_t groups = sms / cg;
-    const int64_t waves = (tiles + groups - 1) / groups;
-    return (double)waves * bn;
-}
-
 }  // namespace
 
 namespace {
@@ -562,15 +553,9 @@ sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
     // [K, N]-stored B is limited to one 128-byte swizzle row of N per tile
     if (a.b_is_kn || a.N <= 128) return launch<128, 1>(a, st);
     if (a.M <= 128) return launch<256, 1>(a, st);
-    // CTA pairs; pick the tile width that leaves the fewest idle SMs in the last wave
-    const int sms = sm_count();
-    // (narrower tiles move more operand bytes per MAC: 28 KB per 128x192x128 vs 32 KB per 128x256x128)
-    const double c256 = tiling_cost(a, 256, 2, sms), c192 = tiling_cost(a, 192, 2, sms) * 1.10,
-                 c128 = tiling_cost(a, 128, 2, sms) * 1.25;
-    const bool allow192 = a.out_dt != SQ_I8;  // 192 columns are not a whole number of 128-column INT8 store groups
-    if ((c256 <= c192 || !allow192) && c256 <= c128) return launch<256, 2>(a, st);
-    if (allow192 && c192 <= c128) return launch<192, 2>(a, st);
-    return launch<128, 2>(a, st);
+    // CTA pairs with 256 x 256 tiles.  Narrower pair tiles (192, 128 columns) were measured: they
+    // even out the last wave of some shapes but move more operand bytes per MAC and lose overall.
+    return launch<256, 2>(a, st);
 }
 
 }  // namespace sq
