@@ -237,6 +237,27 @@ sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t h
                       const int64_t strideC[3], void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * Fused causal INT8 self-attention (Fig. 6: both BMMs in INT8, softmax in floating point) over
+ * the fused QKV code buffer:
+ *     s[i, j]  = (float)(Q_i . K_j) * alpha_qk                      (INT32 accumulate; fp32 scores)
+ *     p[i, j]  = exp(s[i, j] - max_i) / sum_{j' <= i} exp(s[i, j'] - max_i),   0 for j > i
+ *     P[i, j]  = round(127 * p[i, j])                               (step 1/127)
+ *     out[i,:] = clamp(round(((float)(P_i . V) * alpha_pv) * requant_mul))
+ * i.e. the chain sq_w8a8_bmm -> sq_softmax_quant_p -> sq_w8a8_bmm with the scores kept in fp32
+ * instead of being rounded to a 16-bit type, and without writing the [S, S] score and probability
+ * matrices to memory.  exp and the row sums are not bit-reproducible against another
+ * implementation, so individual P codes (and, through them, output codes) may differ by one
+ * where a value sits on a rounding boundary.  alpha_qk must be positive.
+ * qkv: [B*S, 3*H*d] int8, row-major (Q | K | V column blocks, head h at columns h*d .. of each),
+ * 16-byte aligned; d must be 128 (else SQ_ERR_UNSUPPORTED); S a multiple of 16.
+ * alpha_qk = Delta_q * Delta_k / sqrt(d); alpha_pv = Delta_v / 127; requant_mul: device pointer to
+ * 1 / Delta_attn.  out: [B*S, H*d] int8.  workspace: sq_workspace_bytes(SQ_OP_BMM, ...) bytes.
+ */
+sq_status sq_w8a8_attention(const int8_t* qkv, int64_t B, int64_t H, int64_t S, int64_t d,
+                            float alpha_qk, float alpha_pv, const float* requant_mul,
+                            int8_t* out, void* workspace, size_t ws_bytes, void* stream);
+
+/*
  * Attention plumbing between the two BMMs (Fig. 6 keeps Softmax in floating point):
  * causal softmax over each [S, S] score matrix followed by quantisation of the
  * probabilities with the fixed step 1/127 (softmax output lies in [0, 1]):

@@ -383,13 +383,15 @@ def linear_f64(X, W, b=None):
 # --------------------------------------------------------------------------- #
 # Whole decoder block (Fig. 6), static per-tensor activation steps (O3)
 # --------------------------------------------------------------------------- #
-def decoder_block_static(x, p, B, S, H, d, dtype="f16", eps=1e-5):
+def decoder_block_static(x, p, B, S, H, d, dtype="f16", eps=1e-5, score_dtype=None):
     """One pre-LayerNorm decoder block in the precision mapping of Fig. 6: INT8 for the four
     linear layers and the two attention BMMs, floating point for LayerNorm, softmax, ReLU and
     the residual adds.  `x` is [B*S, H*d] (A-valued float32); `p` holds, per linear
     ("qkv", "out_proj", "fc1", "fc2"), the INT8 weight `Wq`, `w_scale`, `bias`, and the static
     steps `d_ln1, d_q, d_k, d_v, d_attn, d_ln2, d_fc1` plus folded LayerNorm parameters
-    `g1, b1, g2, b2`.  Every intermediate is returned for stage-by-stage comparison."""
+    `g1, b1, g2, b2`.  `score_dtype` is the type the attention scores are held in before the
+    softmax (default: the activation dtype; "f32" when they never leave fp32).  Every intermediate
+    is returned for stage-by-stage comparison."""
     f32 = np.float32
     hid = H * d
     out = {}
@@ -407,7 +409,7 @@ def decoder_block_static(x, p, B, S, H, d, dtype="f16", eps=1e-5):
     v = np.ascontiguousarray(qkv[:, :, 2].transpose(0, 2, 1, 3))
     # scores = Q K^T * (d_q d_k / sqrt(d)), rounded to the activation dtype
     alpha_qk = f32(f32(p["d_q"]) * f32(p["d_k"])) / f32(np.sqrt(f32(d)))
-    _, out["scores"] = w8a8_bmm(q, k, float(alpha_qk), out_dtype=dtype)
+    _, out["scores"] = w8a8_bmm(q, k, float(alpha_qk), out_dtype=score_dtype or dtype)
     # causal softmax in floating point, P quantised with the fixed step 1/127
     Pq = np.empty((B, H, S, S), np.int8)
     for b in range(B):

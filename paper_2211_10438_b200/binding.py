@@ -25,7 +25,7 @@ SQ_NOALLOC_MAX_ROWS = 16384
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
-           "sq_selftest_bounded_wait"]
+           "sq_selftest_bounded_wait", "sq_w8a8_attention"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -69,6 +69,7 @@ def lib():
         L.sq_residual_add.argtypes = [vp, vp, i32, i64, vp, vp]
         L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
         L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
+        L.sq_w8a8_attention.argtypes = [vp, i64, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = i32
         _lib = L
@@ -254,3 +255,11 @@ def sq_selftest_bounded_wait(budget_cycles=200000):
     word = torch.zeros(1, dtype=torch.int32, device="cuda")
     _check(lib().sq_selftest_bounded_wait(_ptr(word), int(budget_cycles), _stream()), "sq_selftest_bounded_wait")
     return int(word.item())
+
+
+def sq_w8a8_attention(qkv, B, H, S, d, alpha_qk, alpha_pv, requant_mul, out, workspace):
+    """Fused causal INT8 attention over the fused QKV code buffer [B*S, 3*H*d] -> out [B*S, H*d] int8."""
+    wp, wn = _ws(workspace)
+    _check(lib().sq_w8a8_attention(_ptr(qkv), B, H, S, d, float(alpha_qk), float(alpha_pv), _ptr(requant_mul),
+                                   _ptr(out), wp, wn, _stream()), "sq_w8a8_attention")
+    return out

@@ -221,6 +221,21 @@ sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t h
     return gemm_i8(a, as_stream(stream));
 }
 
+sq_status sq_w8a8_attention(const int8_t* qkv, int64_t B, int64_t H, int64_t S, int64_t d, float alpha_qk,
+                            float alpha_pv, const float* requant_mul, int8_t* out, void* workspace,
+                            size_t ws_bytes, void* stream) {
+    if (B < 0 || H < 0 || S < 0 || d < 0) return SQ_ERR_SHAPE;
+    if (!(alpha_qk > 0.0f)) return SQ_ERR_INVALID_ARG;  // the row maximum is taken on the integer accumulators
+    if (B == 0 || H == 0 || S == 0) return SQ_OK;
+    if (d != 128) return SQ_ERR_UNSUPPORTED;
+    if (!qkv || !out || !requant_mul) return SQ_ERR_INVALID_ARG;
+    if (S % 16 != 0 || !aligned16(qkv) || !aligned16(out)) return SQ_ERR_ALIGN;
+    if (B * S >= ((int64_t)1 << 31) || B > 65535 || H > 65535) return SQ_ERR_UNSUPPORTED;
+    if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_BMM, S, S, d))) return SQ_ERR_WORKSPACE;
+    return attention_i8(qkv, B, H, S, d, alpha_qk, alpha_pv, requant_mul, out,
+                        reinterpret_cast<uint32_t*>(workspace), as_stream(stream));
+}
+
 sq_status sq_softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_t S, int8_t* Pq,
                              void* stream) {
     if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;

@@ -63,6 +63,8 @@ struct GemmArgs {
     size_t ws_bytes;      // size of the caller's workspace
 };
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
+sq_status attention_i8(const int8_t* qkv, int64_t B, int64_t H, int64_t S, int64_t d, float alpha_qk, float alpha_pv,
+                       const float* requant_mul, int8_t* out, uint32_t* status, cudaStream_t st);
 sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st);
 
 // Decode-shaped path (M <= 16): swapped operands, split-K with INT32 scratch in the workspace.

@@ -130,8 +130,10 @@ class DecoderBlockStatic:
     `lin` maps "qkv" / "out_proj" / "fc1" / "fc2" to PreparedLinear; `steps` holds the calibrated
     static steps d_ln1, d_q, d_k, d_v, d_attn, d_ln2, d_fc1 (python floats)."""
 
-    def __init__(self, lin, steps, B, S, H, d, act_dtype, eps=1e-5):
+    def __init__(self, lin, steps, B, S, H, d, act_dtype, eps=1e-5, fused_attention=None):
         self.lin, self.B, self.S, self.H, self.d, self.dt, self.eps = lin, B, S, H, d, act_dtype, eps
+        # the fused attention kernel covers head dimension 128; otherwise BMM -> softmax -> BMM
+        self.fused_attention = (d == 128) if fused_attention is None else fused_attention
         dev = lin["qkv"].Wq.device
         M, hid, ffn = B * S, H * d, lin["fc1"].Wq.shape[0]
         self.M, self.hid = M, hid
@@ -154,7 +156,7 @@ class DecoderBlockStatic:
         self.x2q, self.f1q = e((M, hid), torch.int8), e((M, ffn), torch.int8)
         self.fc2, self.y = e((M, hid), act_dtype), e((M, hid), act_dtype)
         self.ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid), dev)
-        self.launches_per_step = 11
+        self.launches_per_step = 9 if self.fused_attention else 11
 
     def forward(self, x):
         L, s, B, S, H, d, hid = self.lin, self.s, self.B, self.S, self.H, self.d, self.hid
@@ -163,12 +165,15 @@ class DecoderBlockStatic:
                        x_scale=s["d_ln1"], workspace=self.ws)
         sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
                         requant_mul=self.r_qkv, out=self.qkv)
-        flat = self.qkv.view(-1)
-        sq.sq_w8a8_bmm(flat, flat[hid:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False,
-                       self.alpha_qk, self.scores, (H * S * S, S * S, S), self.ws, causal=True)
-        sq.sq_softmax_quant_p(self.scores, self.P)
-        sq.sq_w8a8_bmm(self.P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
-                       self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn, causal=True)
+        if self.fused_attention:
+            sq.sq_w8a8_attention(self.qkv, B, H, S, d, self.alpha_qk, self.alpha_pv, self.r_attn, self.attn, self.ws)
+        else:
+            flat = self.qkv.view(-1)
+            sq.sq_w8a8_bmm(flat, flat[hid:], B, H, S, S, d, (S * row, d, row), (S * row, d, row), False,
+                           self.alpha_qk, self.scores, (H * S * S, S * S, S), self.ws, causal=True)
+            sq.sq_softmax_quant_p(self.scores, self.P)
+            sq.sq_w8a8_bmm(self.P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
+                           self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn, causal=True)
         sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
                         bias=L["out_proj"].bias, out=self.proj)
         sq.sq_residual_add(x, self.proj, out=self.h)

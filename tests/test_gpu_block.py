@@ -72,7 +72,8 @@ def _oracle_prepare(x, W, bias, ln, B, S, H, d, dtype, alpha=0.5, eps=1e-5):
 def test_decoder_block_static_against_oracle(dtype, B, S, H, d, ffn):
     x, W, bias, ln = _make_block(B, S, H, d, ffn, dtype)
     p = _oracle_prepare(x, W, bias, ln, B, S, H, d, dtype)
-    want = oracle.decoder_block_static(x, p, B, S, H, d, dtype)
+    fused = d == 128  # the pipeline then uses the fused attention kernel, whose scores stay in fp32
+    want = oracle.decoder_block_static(x, p, B, S, H, d, dtype, score_dtype="f32" if fused else None)
 
     tdt = {"f16": torch.float16, "bf16": torch.bfloat16}[dtype]
     lin = {}
@@ -94,7 +95,8 @@ def test_decoder_block_static_against_oracle(dtype, B, S, H, d, ffn):
 
     codes_close("LN1 codes", blk.x1q, want["x1q"], 1e-3)
     codes_close("QKV codes", blk.qkv, want["qkv"], 5e-3)
-    codes_close("P codes", blk.P, want["P"].reshape(B * H, S, S), 2e-2)
+    if not blk.fused_attention:  # the fused attention kernel never materialises P
+        codes_close("P codes", blk.P, want["P"].reshape(B * H, S, S), 2e-2)
     codes_close("attention codes", blk.attn, want["attn"], 2e-2)
     codes_close("FC1 codes", blk.f1q, want["f1q"], 2e-2)
     got = host(y).astype(np.float64)
