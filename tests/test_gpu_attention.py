@@ -27,7 +27,7 @@ def _oracle_attention(qkv, B, H, S, d, alpha_qk, alpha_pv, r, dtype):
     return np.ascontiguousarray(o.transpose(0, 2, 1, 3)).reshape(B * S, H * d), P
 
 
-@pytest.mark.parametrize("B,H,S", [(1, 2, 128), (2, 3, 512), (1, 1, 384), (1, 2, 208), (2, 1, 16), (1, 1, 1024)])
+@pytest.mark.parametrize("B,H,S", [(1, 2, 128), (2, 3, 512), (1, 1, 384), (1, 2, 208), (2, 1, 16), (1, 1, 1024), (1, 2, 2048)])
 def test_fused_attention_against_oracle_chain(B, H, S):
     dtype = "f32"  # the fused kernel never rounds the scores to a 16-bit type
     d = 128

@@ -47,6 +47,18 @@ def test_gemm_all_127_and_identity(ws):
     assert np.array_equal(host(acc), 127 * Xq.astype(np.int32))
 
 
+@pytest.mark.parametrize("M", [130, 16])
+def test_gemm_longest_supported_reduction_hits_the_int32_edge(ws, M):
+    # K = 133120 (the largest multiple of 128 below the 133144 bound), every product = 127 * 127 or -(127 * 127)
+    N, K = 128, 133120
+    X = np.full((M, K), 127, np.int8)
+    W = np.full((N, K), 127, np.int8)
+    W[1::2] = -127
+    acc = host(sq.sq_w8a8_gemm(dev(X), dev(W), None, None, ws, out_dtype=torch.int32))
+    want = np.where(np.arange(N) % 2 == 0, 16129 * K, -16129 * K).astype(np.int64)
+    assert want.max() < 2 ** 31 and np.array_equal(acc.astype(np.int64), np.broadcast_to(want, (M, N)))
+
+
 def test_gemm_run_to_run_identical(ws):
     Xq, Wq = synth.int8_tensor(20, 4, (384, 2048)), synth.int8_tensor(20, 5, (1536, 2048))
     a = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, ws, out_dtype=torch.int32)
