@@ -400,7 +400,8 @@ def main():
         raise SystemExit("device status word = %d: a bounded wait expired" % status)
     gemm_total = sum(sum(v) for v in gemm_s.values())
     achieved = ops_step * args.steps / gemm_total / 1e12
-    peak_tops = 2.0 * peaks["bf16_sustained"]
+    # the timed region is tens of milliseconds at full clocks: the burst figure is the fair denominator
+    peak_tops = 2.0 * peaks["bf16_burst"]
 
     # ---------------- end to end: host buffers in, host result out ----------------
     hx = x_in.cpu().pin_memory()
@@ -440,14 +441,33 @@ def main():
         "gpu_launches": block.launches_per_step * args.steps,
         "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak_tops,
                      "unit": "TOP/s", "frac": achieved / peak_tops,
-                     "peak_source": "2 x %s bf16 sustained (%s); int8:bf16 nominal ratio 2" % (peaks["bf16_sustained"], peaks["source"]),
-                     "frac_of_2x_bf16_burst": achieved / (2 * peaks["bf16_burst"]), "frac_of_nominal_4500": achieved / 4500.0,
+                     "peak_source": "2 x %s bf16 burst (%s); int8:bf16 nominal ratio 2" % (peaks["bf16_burst"], peaks["source"]),
+                     "frac_of_2x_bf16_sustained": achieved / (2 * peaks["bf16_sustained"]), "frac_of_nominal_4500": achieved / 4500.0,
                      "per_gemm_us": {k: statistics.mean(v) * 1e6 for k, v in gemm_s.items()},
                      "traffic": GEMM_DRAM_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": block.gemm_bytes() / 4},
         "offline_setup_s": offline_s,
     }
     if rank == 0 and world == 1 and not args.no_rows:
         out["rows"] = timed_rows(device, peaks)
+        # the same step repeated for ~2 s: what the part sustains under its power cap
+        sampler = ClockSampler(local)
+        sampler.start()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        n_sus = 0
+        e0.record()
+        while time.perf_counter() - t0 < 2.0:
+            for _ in range(200):
+                block.step(x_in, attn_out)
+            n_sus += 200
+            torch.cuda.synchronize()
+        e1.record()
+        torch.cuda.synchronize()
+        sus_s = e0.elapsed_time(e1) * 1e-3
+        sus_tops = ops_step * n_sus / sus_s / 1e12
+        out["rows"]["sustained_step_2s"] = {"TOPS": sus_tops, "ms_per_step": sus_s / n_sus * 1e3, "steps": n_sus,
+                                            "frac_of_2x_bf16_sustained_incl_quantise": sus_tops / (2 * peaks["bf16_sustained"]),
+                                            "clocks": sampler.stop()}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         host = host_model(wl)
