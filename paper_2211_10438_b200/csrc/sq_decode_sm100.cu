@@ -311,9 +311,6 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     p.splits = choose_splits(p.M, p.N, p.num_n, p.num_kb, sm_count());
     if (ws_bytes < decode_workspace_bytes(a.N)) p.splits = 1;  // no scratch: every tile in one unit
-#ifdef SQ_EXP_SPLITS  // measurement build
-    p.splits = SQ_EXP_SPLITS;
-#endif
     p.kb_per_split = (p.num_kb + p.splits - 1) / p.splits;
     p.total_units = (int64_t)p.num_n * p.splits;
     p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
