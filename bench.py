@@ -406,21 +406,20 @@ def main():
     # ---------------- end to end: host buffers in, host result out ----------------
     hx = x_in.cpu().pin_memory()
     ha = attn_out.cpu().pin_memory()
-    hy = torch.empty((block.M, wl.hidden), dtype=torch.bfloat16).pin_memory()
-    dx, da = torch.empty_like(x_in), torch.empty_like(attn_out)
+    hy = [torch.empty((block.M, wl.hidden), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    from paper_2211_10438_b200.pipeline import HostStreamedBlock
+    streamed = HostStreamedBlock(block, wl.hidden)
 
-    def e2e_step():
-        dx.copy_(hx, non_blocking=True)
-        da.copy_(ha, non_blocking=True)
-        y = block.step(dx, da)
-        hy.copy_(y, non_blocking=True)
-
-    for _ in range(3):
-        e2e_step()
+    # every step copies its own inputs up and its own result down; the copies of neighbouring
+    # steps overlap with the kernels, and the timed region ends after the last result has landed
+    for i in range(3):
+        streamed.submit(hx, ha, hy[i & 1])
+    streamed.drain()
     barrier()
     e0.record()
-    for _ in range(args.steps):
-        e2e_step()
+    for i in range(args.steps):
+        streamed.submit(hx, ha, hy[i & 1])
+    streamed.drain()
     e1.record()
     barrier()
     e2e_value, e2e_elapsed = aggregate_replicas(ops_step, args.steps, e0.elapsed_time(e1) * 1e-3, world, max_over_ranks)
@@ -437,7 +436,8 @@ def main():
                    "l2": "working set per step ~0.6 GB (314 MB INT8 weights + activations) exceeds the 126 MB L2; no flush"},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "TOPS", "ms_per_step": e2e_elapsed / args.steps * 1e3,
-                "h2d_bytes_per_step": int(hx.numel() * 2 + ha.numel() * 2), "d2h_bytes_per_step": int(hy.numel() * 2)},
+                "h2d_bytes_per_step": int(hx.numel() * 2 + ha.numel() * 2), "d2h_bytes_per_step": int(hy[0].numel() * 2),
+                "overlap": "copies of steps i+1 / i-1 on two copy streams beside step i's kernels; all inside the timed region"},
         "gpu_launches": block.launches_per_step * args.steps,
         "roofline": {"bound": "tensor", "kernel": "gemm_i8_kernel", "achieved": achieved, "peak": peak_tops,
                      "unit": "TOP/s", "frac": achieved / peak_tops,

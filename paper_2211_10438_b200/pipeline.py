@@ -66,21 +66,22 @@ class LinearBlock:
         self.launches_per_step = 8 if gran != "per_tensor_dynamic" else 12
         self.gemm_events = None  # optional list collecting (start, stop) CUDA events per GEMM
 
-    def _gemm(self, name):
+    def _gemm(self, name, out=None):
         l, b = self.lin[name], self.buf[name]
+        Y = b["Y"] if out is None else out
         ev = None
         if self.gemm_events is not None:
             ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
             ev[0].record()
-        sq.sq_w8a8_gemm(b["Xq"], l.Wq, b["xs"], l.w_scale, self.ws, bias=l.bias, relu=l.relu, out=b["Y"])
+        sq.sq_w8a8_gemm(b["Xq"], l.Wq, b["xs"], l.w_scale, self.ws, bias=l.bias, relu=l.relu, out=Y)
         if ev is not None:
             ev[1].record()
             self.gemm_events.append((name, ev))
-        return b["Y"]
+        return Y
 
-    def step(self, x_in, attn_out):
+    def step(self, x_in, attn_out, out=None):
         """x_in: block input [M, hidden]; attn_out: attention output [M, hidden] (the attention
-        itself is a separate path).  Returns the FC2 output."""
+        itself is a separate path).  Returns the FC2 output (written to `out` when given)."""
         q, o, f1, f2 = (self.lin[n] for n in ("qkv", "out_proj", "fc1", "fc2"))
         b = self.buf
         sq.sq_ln_quant(x_in, q.gamma_hat, q.beta_hat, self.eps, self.gran, Xq=b["qkv"]["Xq"],
@@ -93,7 +94,7 @@ class LinearBlock:
                        x_scale=b["fc1"]["xs"], workspace=self.ws)
         a = self._gemm("fc1")
         sq.sq_quant_act(a, self.gran, Xq=b["fc2"]["Xq"], x_scale=b["fc2"]["xs"], workspace=self.ws)
-        return self._gemm("fc2")
+        return self._gemm("fc2", out=out)
 
     def gemm_ops(self):
         return sum(2 * self.M * l.Wq.shape[0] * l.Wq.shape[1] for l in self.lin.values())
@@ -102,6 +103,53 @@ class LinearBlock:
         """Algorithmic bytes of the four GEMMs: M*K + N*K (INT8) + M*N outputs in the activation dtype."""
         return sum(self.M * l.Wq.shape[1] + l.Wq.shape[0] * l.Wq.shape[1] + 2 * self.M * l.Wq.shape[0]
                    for l in self.lin.values())
+
+
+class HostStreamedBlock:
+    """Runs LinearBlock steps on inputs that live in pinned HOST memory and returns results to
+    pinned host memory, with the copies of neighbouring steps overlapped with the kernels: step
+    i+1's inputs go up on one stream and step i-1's result comes down on another while step i
+    computes.  Two device slots per buffer; events order slot reuse.  All copies of every step
+    are issued and waited for inside whatever region the caller times."""
+
+    def __init__(self, block, hidden):
+        self.block = block
+        dev = block.ws.device
+        M, dt = block.M, block.dt
+        e = lambda: torch.empty((M, hidden), dtype=dt, device=dev)
+        self.dx, self.da, self.dy = [e(), e()], [e(), e()], [e(), e()]
+        self.s_in, self.s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+        ev = lambda: [torch.cuda.Event(), torch.cuda.Event()]
+        self.in_done, self.comp_done, self.out_done = ev(), ev(), ev()
+        self.i = 0
+
+    def submit(self, hx, ha, hy):
+        """Queue one step: hx, ha pinned host inputs, hy pinned host output.  Returns at once; hy
+        is valid after drain() (or after the out_done event of its slot)."""
+        k, first = self.i & 1, self.i < 2
+        comp = torch.cuda.current_stream()
+        with torch.cuda.stream(self.s_in):
+            if not first:
+                self.s_in.wait_event(self.comp_done[k])  # step i-2 has finished reading this slot
+            self.dx[k].copy_(hx, non_blocking=True)
+            self.da[k].copy_(ha, non_blocking=True)
+            self.in_done[k].record(self.s_in)
+        comp.wait_event(self.in_done[k])
+        if not first:
+            comp.wait_event(self.out_done[k])  # step i-2's result has left this slot
+        self.block.step(self.dx[k], self.da[k], out=self.dy[k])
+        self.comp_done[k].record(comp)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.comp_done[k])
+            hy.copy_(self.dy[k], non_blocking=True)
+            self.out_done[k].record(self.s_out)
+        self.i += 1
+
+    def drain(self):
+        """Make the compute stream wait for every queued copy-out."""
+        comp = torch.cuda.current_stream()
+        for k in range(min(self.i, 2)):
+            comp.wait_event(self.out_done[k])
 
 
 def synth_device_activations(M, C, dtype, channels, factors, seed, device="cuda"):

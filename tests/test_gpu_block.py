@@ -121,3 +121,36 @@ def test_decoder_block_is_deterministic():
     a = blk.forward(xd).clone()
     b = blk.forward(xd).clone()
     assert torch.equal(a, b)
+
+
+def test_host_streamed_block_matches_sequential_steps():
+    """Five steps with different pinned host inputs through the overlapped copy/compute path give,
+    byte for byte, what the same LinearBlock gives when stepped one input at a time."""
+    M, hid, ffn = 384, 512, 2048
+    rng = synth.rng_for(41, 1)
+    shapes = {"qkv": (3 * hid, hid), "out_proj": (hid, hid), "fc1": (ffn, hid), "fc2": (hid, ffn)}
+    lin = {}
+    for i, (n, (N, K)) in enumerate(shapes.items()):
+        lin[n] = pl.PreparedLinear(n, dev(synth.int8_tensor(41, 10 + i, (N, K))),
+                                   dev(rng.uniform(1e-4, 1e-3, N).astype(np.float32)),
+                                   dev(synth.bias(41, 20 + i, N, "bf16"), "bf16"), n == "fc1")
+    for n, k in (("qkv", 3), ("fc1", 4)):
+        g, b = synth.ln_params(41, k, hid, "bf16")
+        lin[n].gamma_hat, lin[n].beta_hat = dev(g, "bf16"), dev(b, "bf16")
+    blk = pl.LinearBlock(lin["qkv"], lin["out_proj"], lin["fc1"], lin["fc2"], M, torch.bfloat16)
+    xs = [torch.from_numpy(synth.activations(41, 30 + i, M, hid, "bf16", [3, 77], [40.0, 25.0])).to(torch.bfloat16).pin_memory()
+          for i in range(5)]
+    ats = [torch.from_numpy(synth.activations(41, 40 + i, M, hid, "bf16", [3, 77], [40.0, 25.0])).to(torch.bfloat16).pin_memory()
+           for i in range(5)]
+    want = []
+    for x, a in zip(xs, ats):
+        want.append(blk.step(x.cuda(), a.cuda()).cpu().clone())
+    outs = [torch.empty((M, hid), dtype=torch.bfloat16).pin_memory() for _ in range(5)]
+    st = pl.HostStreamedBlock(blk, hid)
+    for x, a, o in zip(xs, ats, outs):
+        st.submit(x, a, o)
+    st.drain()
+    torch.cuda.synchronize()
+    assert sq.device_status(blk.ws) == 0
+    for o, w in zip(outs, want):
+        assert torch.equal(o.view(torch.int16), w.view(torch.int16))
