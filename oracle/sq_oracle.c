@@ -307,6 +307,28 @@ void sqo_softmax_causal_f64(const float *S, int64_t rows, int64_t cols, int64_t 
     }
 }
 
+/* Softmax of rows that each see a prefix of the keys: row i sees the first
+ * (first + i) of them.  first = 1 is the causal softmax of a prompt; one row
+ * with first = L is the generation stage, where the newest token attends to
+ * all L cached positions.  Same fp32 steps, in the same order, as above. */
+void sqo_softmax_prefix(const float *S, int64_t rows, int64_t cols, int64_t ld, int64_t first,
+                        float *P) {
+    for (int64_t i = 0; i < rows; ++i) {
+        int64_t n = first + i < cols ? first + i : cols;
+        float mx = S[i * ld];
+        for (int64_t j = 1; j < n; ++j)
+            if (S[i * ld + j] > mx) mx = S[i * ld + j];
+        float sum = 0.0f;
+        for (int64_t j = 0; j < n; ++j) {
+            float e = expf(S[i * ld + j] - mx);
+            P[i * cols + j] = e;
+            sum += e;
+        }
+        for (int64_t j = 0; j < n; ++j) P[i * cols + j] = P[i * cols + j] / sum;
+        for (int64_t j = n; j < cols; ++j) P[i * cols + j] = 0.0f;
+    }
+}
+
 /* ------------------------------------------------------------------------- */
 /* fp64 truth: the unquantised linear layer Y = X W^T (+ b), stored W [N, K]. */
 /* ------------------------------------------------------------------------- */

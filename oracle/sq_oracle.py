@@ -367,6 +367,42 @@ def softmax_quant_p(S):
     return requant(P, np.float32(127.0)), P
 
 
+def softmax_prefix(S, first: int):
+    """fp32 softmax where row i sees the first (first + i) keys; first=1 is softmax_causal."""
+    S = _f32(S)
+    P = np.empty_like(S)
+    _lib.sqo_softmax_prefix(_p(S, _f32p), _i64(S.shape[0]), _i64(S.shape[1]), _i64(S.shape[1]),
+                            _i64(first), _p(P, _f32p))
+    return P
+
+
+def kv_decode_attention(q, K, V, lens, alpha_qk: float, alpha_pv: float, out_dtype="f16",
+                        requant_mul=None, score_dtype="f32"):
+    """Generation-stage attention over an INT8 key/value cache (the Discussion's point that
+    quantised activations also shrink the KV cache), in the precision mapping of Fig. 6:
+    INT8 q.K^T -> floating-point softmax -> P_bar = round(127 p) -> INT8 P_bar.V.
+
+    q [B, H, d] INT8: the newest token's query; K, V [B, H, L_max, d] INT8: the cache, of which
+    sequence b holds lens[b] valid positions (the newest token's own k, v included).
+    Returns (out [B, H, d], P_bar list per (b, h)), out = requant or rounded to out_dtype."""
+    q, K, V = _i8(q), _i8(K), _i8(V)
+    B, H, d = q.shape
+    out = np.empty((B, H, d), np.int8 if requant_mul is not None else np.float32)
+    Ps = []
+    for b in range(B):
+        L = int(lens[b])
+        for h in range(H):
+            acc = gemm_i32(q[b, h][None, :], K[b, h, :L])          # [1, L]
+            s = round_to(scale_acc(acc, alpha_qk), score_dtype)
+            p = softmax_prefix(s, L)
+            Pq = requant(p, np.float32(127.0))
+            acc2 = gemm_i32_bt(Pq, V[b, h, :L])                     # [1, d]
+            y = scale_acc(acc2, alpha_pv)
+            out[b, h] = (requant(y, requant_mul) if requant_mul is not None else round_to(y, out_dtype))[0]
+            Ps.append(Pq[0])
+    return out, Ps
+
+
 def linear_f64(X, W, b=None):
     """fp64 truth: Y = X W^T + b with W stored [N, K]."""
     X = np.ascontiguousarray(X, np.float64)

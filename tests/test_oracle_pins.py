@@ -365,3 +365,77 @@ def test_softmax_causal_and_bmm():
     assert np.array_equal(acc2, ref2)
     y = (ref2.astype(np.float32) * np.float32(0.002)) * np.float32(1.5)
     assert np.array_equal(q2, np.clip(np.rint(y), -127, 127).astype(np.int8))
+
+
+# --------------------------------------------------------------------------- #
+# Generation-stage attention over an INT8 KV cache
+# --------------------------------------------------------------------------- #
+def test_softmax_prefix_reduces_to_causal_and_to_library_softmax():
+    rng = np.random.default_rng(43)
+    S = (rng.standard_normal((12, 12)) * 4).astype(np.float32)
+    assert np.array_equal(oracle.softmax_prefix(S, 1), oracle.softmax_causal(S))
+    # one row that sees every key = the last row of the causal softmax = a plain softmax
+    last = oracle.softmax_prefix(S[-1:], 12)
+    assert np.array_equal(last[0], oracle.softmax_causal(S)[-1])
+    ref = torch.softmax(torch.from_numpy(S[-1:]).double(), -1).numpy()
+    assert np.abs(last - ref).max() <= 1e-6
+    # a shorter prefix leaves the tail at zero and still sums to one
+    P5 = oracle.softmax_prefix(S[:1], 5)
+    assert not P5[0, 5:].any() and abs(P5.sum() - 1.0) <= 1e-6
+    # softmax is invariant under a common shift of the scores
+    assert np.abs(oracle.softmax_prefix(S[:1] + 3.0, 12) - oracle.softmax_prefix(S[:1], 12)).max() <= 1e-6
+
+
+def test_kv_decode_attention_is_the_last_row_of_prompt_attention():
+    """Incremental decoding must give what the prompt pass gives for its last token: the same q,
+    the same keys and values, every position visible."""
+    rng = np.random.default_rng(44)
+    B, H, L, d = 2, 3, 37, 16
+    q = rng.integers(-100, 101, (B, H, L, d), dtype=np.int8)
+    K = rng.integers(-100, 101, (B, H, L, d), dtype=np.int8)
+    V = rng.integers(-100, 101, (B, H, L, d), dtype=np.int8)
+    a_qk, a_pv, r = np.float32(0.004), np.float32(0.01 / 127), np.float32(1 / 0.004)
+    _, scores = oracle.w8a8_bmm(q, K, a_qk, out_dtype="f32")
+    want = np.empty((B, H, d), np.int8)
+    for b in range(B):
+        for h in range(H):
+            Pq, _ = oracle.softmax_quant_p(scores[b, h])
+            _, o = oracle.w8a8_bmm(Pq, V[b, h], a_pv, b_is_kn=True, requant_mul=r)
+            want[b, h] = o[-1]
+    got, _ = oracle.kv_decode_attention(q[:, :, -1], K, V, [L, L], a_qk, a_pv, requant_mul=r)
+    assert np.array_equal(got, want)
+    # a shorter valid length ignores everything stored beyond it
+    got_short, _ = oracle.kv_decode_attention(q[:, :, -1], K, V, [20, 9], a_qk, a_pv, requant_mul=r)
+    K2, V2 = K.copy(), V.copy()
+    K2[0, :, 20:], V2[0, :, 20:], K2[1, :, 9:], V2[1, :, 9:] = 99, -99, -99, 99
+    got_short2, _ = oracle.kv_decode_attention(q[:, :, -1], K2, V2, [20, 9], a_qk, a_pv, requant_mul=r)
+    assert np.array_equal(got_short, got_short2) and not np.array_equal(got_short, got)
+
+
+def test_kv_decode_attention_closed_forms_and_error_bound():
+    rng = np.random.default_rng(45)
+    B, H, L, d = 1, 2, 50, 8
+    q = rng.integers(-90, 91, (B, H, d), dtype=np.int8)
+    V = rng.integers(-127, 128, (B, H, L, d), dtype=np.int8)
+    K = rng.integers(-90, 91, (B, H, L, d), dtype=np.int8)
+    a_qk, d_v = np.float32(0.002), np.float32(0.03)
+    a_pv = np.float32(d_v / np.float32(127.0))
+    # one cached position: p = 1, P_bar = 127, out = 127 * v * (d_v / 127)
+    out1, Ps = oracle.kv_decode_attention(q, K, V, [1], a_qk, a_pv, out_dtype="f32")
+    assert all(P[0] == 127 and P.size == 1 for P in Ps)
+    assert np.array_equal(out1, (V[:, :, 0].astype(np.float32) * np.float32(127.0)) * a_pv)
+    # identical keys: uniform p = 1/L, so every P_bar = round(127 / L) and out = P_bar * sum(v) * alpha
+    Ku = np.broadcast_to(K[:, :, :1], K.shape).copy()
+    outu, Ps = oracle.kv_decode_attention(q, Ku, V, [L], a_qk, a_pv, out_dtype="f32")
+    pb = int(np.rint(127.0 / L))
+    assert all((P == pb).all() for P in Ps)
+    assert np.array_equal(outu, (pb * V.astype(np.int64).sum(2)).astype(np.float32) * a_pv)
+    # against the unquantised-probability result in fp64: each P_bar/127 is within 0.5/127 of p
+    out, _ = oracle.kv_decode_attention(q, K, V, [L], a_qk, a_pv, out_dtype="f32")
+    s = np.einsum("bhd,bhld->bhl", q.astype(np.float64), K.astype(np.float64)) * float(a_qk)
+    p = np.exp(s - s.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    truth = np.einsum("bhl,bhld->bhd", p, V.astype(np.float64)) * float(d_v)
+    bound = (0.5 / 127) * np.abs(V.astype(np.float64)).sum(2) * float(d_v)
+    assert np.all(np.abs(out - truth) <= bound * (1 + 1e-5) + 1e-6)
+    assert np.abs(out - truth).max() > 0  # the bound is not vacuous: quantising p does move the result
