@@ -258,6 +258,54 @@ sq_status sq_w8a8_attention(const int8_t* qkv, int64_t B, int64_t H, int64_t S, 
                             int8_t* out, void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * INT8 key/value cache for the generation stage (Section 7, Discussion: quantising activations
+ * also reduces the memory held by the KV cache).  Layout, chosen for the reader below:
+ *     k_cache [B, H, L_max, d]      int8: one key per d-byte row;
+ *     v_cache [B, H, L_max/4, d, 4] int8: the values of four consecutive positions 4g .. 4g+3 of
+ *                                   one channel share a 32-bit word (position 4g+r, channel c at
+ *                                   byte ((g*d + c)*4 + r) of the head's block).
+ * sq_kv_cache_write copies the K and V codes of T tokens per sequence out of the fused QKV code
+ * buffer qkv [B*T, ld] (row b*T + t; Q | K | V column blocks of H*d, head h at columns h*d ..)
+ * to cache positions pos0[b] .. pos0[b] + T - 1 of sequence b.  pos0: device pointer to B int32
+ * (nullable = all zero).  T = prompt length fills the cache after the prompt pass; T = 1 appends
+ * the newest token.  A sequence whose run would leave [0, L_max) is skipped and the device
+ * status word is set (SQ_ERR_SHAPE).  d must be 128; L_max a multiple of 4; ld a multiple of 16;
+ * pointers 16-byte aligned.  workspace: at least 256 bytes, 256-byte aligned; word 0 = device status.
+ */
+sq_status sq_kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T, int64_t H, int64_t d,
+                            const int32_t* pos0, int8_t* k_cache, int8_t* v_cache, int64_t L_max,
+                            void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * Generation-stage attention of the newest token of each sequence over the INT8 cache, in the
+ * precision mapping of Fig. 6 (both products in INT8, softmax in floating point):
+ *     s[j]   = (float)(q . K_j) * alpha_qk                          j < seq_lens[b]
+ *     p[j]   = exp(s[j] - max) / sum_j' exp(s[j'] - max)
+ *     P[j]   = round(127 * p[j])                                    (step 1/127)
+ *     out[:] = ((float)(sum_j P[j] * V_j)) * alpha_pv               -> 16-bit float, or
+ *              clamp(round(that * requant_mul)) -> int8
+ * i.e. what sq_w8a8_attention computes for the last row of a prompt of seq_lens[b] tokens.
+ * exp and the sum are not bit-reproducible against another implementation, so P codes (and
+ * through them output codes) may differ by one where a value sits on a rounding boundary; for a
+ * given shape the result is deterministic.  alpha_qk must be positive.
+ * q: [B, ldq] int8, head h at columns h*d .. (it may point into the QKV code buffer, ldq = 3*H*d);
+ * k_cache / v_cache: as above; seq_lens: device pointer to B int32, the number of valid positions
+ * INCLUDING the newest token (whose k, v the caller has already written); max_len: a host-side
+ * upper bound of seq_lens[] (<= L_max) that sizes shared memory and the split of one sequence
+ * over a thread-block cluster -- a longer sequence is truncated to max_len and the device status
+ * word is set (SQ_ERR_SHAPE); seq_lens[b] <= 0 gives a zero output row.
+ * out: [B, ldo] of out_dt (SQ_I8 needs requant_mul, a device pointer to one fp32; SQ_F16 / SQ_BF16
+ * ignore it).  d must be 128 (else SQ_ERR_UNSUPPORTED), L_max a multiple of 4, ldq a multiple of 16,
+ * q / caches 16-byte aligned; max_len beyond what eight CTAs can hold in shared memory
+ * (about 300 000 positions) is SQ_ERR_UNSUPPORTED.  workspace: >= 256 bytes; word 0 = device status.
+ */
+sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, const int8_t* k_cache, const int8_t* v_cache,
+                                   const int32_t* seq_lens, int64_t B, int64_t H, int64_t d, int64_t L_max,
+                                   int64_t max_len, float alpha_qk, float alpha_pv, const float* requant_mul,
+                                   void* out, sq_dtype out_dt, int64_t ldo, void* workspace, size_t ws_bytes,
+                                   void* stream);
+
+/*
  * Attention plumbing between the two BMMs (Fig. 6 keeps Softmax in floating point):
  * causal softmax over each [S, S] score matrix followed by quantisation of the
  * probabilities with the fixed step 1/127 (softmax output lies in [0, 1]):

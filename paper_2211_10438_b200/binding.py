@@ -14,6 +14,8 @@ LIB_PATH = os.path.join(_HERE, "libsq.so")
 
 # enums of include/sq.h
 SQ_OK = 0
+(SQ_ERR_INVALID_ARG, SQ_ERR_SHAPE, SQ_ERR_ALIGN, SQ_ERR_UNSUPPORTED, SQ_ERR_CUDA, SQ_ERR_TIMEOUT,
+ SQ_ERR_WORKSPACE) = range(1, 8)
 SQ_F16, SQ_BF16, SQ_I8, SQ_I32 = 0, 1, 2, 3
 SQ_PER_TENSOR_STATIC, SQ_PER_TENSOR_DYNAMIC, SQ_PER_TOKEN_DYNAMIC = 0, 1, 2
 SQ_W_PER_TENSOR, SQ_W_PER_CHANNEL = 0, 1
@@ -25,7 +27,7 @@ SQ_NOALLOC_MAX_ROWS = 16384
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
-           "sq_selftest_bounded_wait", "sq_w8a8_attention"]
+           "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -70,6 +72,9 @@ def lib():
         L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
         L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
         L.sq_w8a8_attention.argtypes = [vp, i64, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
+        L.sq_kv_cache_write.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, vp, i64, vp, sz, vp]
+        L.sq_w8a8_decode_attention.argtypes = [vp, i64, vp, vp, vp, i64, i64, i64, i64, i64, f32, f32, vp, vp, i32,
+                                               i64, vp, sz, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = i32
         _lib = L
@@ -262,4 +267,26 @@ def sq_w8a8_attention(qkv, B, H, S, d, alpha_qk, alpha_pv, requant_mul, out, wor
     wp, wn = _ws(workspace)
     _check(lib().sq_w8a8_attention(_ptr(qkv), B, H, S, d, float(alpha_qk), float(alpha_pv), _ptr(requant_mul),
                                    _ptr(out), wp, wn, _stream()), "sq_w8a8_attention")
+    return out
+
+
+def sq_kv_cache_write(qkv, B, T, H, d, pos0, k_cache, v_cache, L_max, workspace):
+    """Copies K and V codes of T tokens per sequence from the QKV code buffer [B*T, 3*H*d] into the
+    INT8 cache at positions pos0[b] .. (pos0: int32 device tensor or None = 0)."""
+    wp, wn = _ws(workspace)
+    _check(lib().sq_kv_cache_write(_ptr(qkv), qkv.stride(0), B, T, H, d, _ptr(pos0), _ptr(k_cache), _ptr(v_cache),
+                                   L_max, wp, wn, _stream()), "sq_kv_cache_write")
+
+
+def sq_w8a8_decode_attention(q, k_cache, v_cache, seq_lens, B, H, d, L_max, max_len, alpha_qk, alpha_pv, workspace,
+                             requant_mul=None, out=None, out_dtype=None):
+    """Attention of each sequence's newest token over the INT8 cache.  q: [B, >= H*d] int8 (row stride
+    taken from the tensor); seq_lens: int32 device tensor [B]; out: [B, H*d] int8 / fp16 / bf16."""
+    if out is None:
+        out = torch.empty((B, H * d), dtype=out_dtype or (torch.int8 if requant_mul is not None else torch.float16),
+                          device=q.device)
+    wp, wn = _ws(workspace)
+    _check(lib().sq_w8a8_decode_attention(_ptr(q), q.stride(0), _ptr(k_cache), _ptr(v_cache), _ptr(seq_lens), B, H, d,
+                                          L_max, max_len, float(alpha_qk), float(alpha_pv), _ptr(requant_mul), _ptr(out),
+                                          _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_decode_attention")
     return out

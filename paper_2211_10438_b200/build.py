@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsq.so")
 SOURCES = ["sq_api.cu", "sq_stream_kernels.cu", "sq_gemm_sm100.cu", "sq_noalloc.cu",
-           "sq_row_pipeline.cu", "sq_decode_sm100.cu", "sq_attention_sm100.cu"]
+           "sq_row_pipeline.cu", "sq_decode_sm100.cu", "sq_attention_sm100.cu", "sq_kv_attention.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
