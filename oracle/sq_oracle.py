@@ -468,3 +468,41 @@ def decoder_block_static(x, p, B, S, H, d, dtype="f16", eps=1e-5, score_dtype=No
                                 out_dtype=dtype)
     out["y"] = round_to(out["h"] + out["fc2"], dtype)
     return out
+
+
+def decoder_block_static_decode(x, p, K_cache, V_cache, ctx, H, d, dtype="f16", eps=1e-5):
+    """Generation stage of decoder_block_static: x [B, H*d] is the newest token of each sequence,
+    K_cache / V_cache [B, H, L_max, d] INT8 hold the codes of the ctx[b] earlier positions.  The
+    token's own k, v codes are stored at position ctx[b] (the caches are updated in place) and its
+    attention runs over ctx[b] + 1 positions with fp32 scores (kv_decode_attention); everything
+    else is the prompt block's arithmetic on one row per sequence."""
+    f32 = np.float32
+    B, hid = x.shape[0], H * d
+    out = {}
+    out["x1q"], _, _ = ln_quant(x, p["g1"], p["b1"], eps, "per_tensor_static", static_scale=p["d_ln1"])
+    acc = gemm_i32(out["x1q"], p["qkv"]["Wq"])
+    y = dequant(acc, p["d_ln1"], p["qkv"]["w_scale"], p["qkv"]["bias"])
+    r = np.concatenate([np.full(hid, f32(1) / f32(p["d_q"]), f32), np.full(hid, f32(1) / f32(p["d_k"]), f32),
+                        np.full(hid, f32(1) / f32(p["d_v"]), f32)])
+    out["qkv"] = requant(y, r)
+    qkv = out["qkv"].reshape(B, 3, H, d)
+    lens = []
+    for b in range(B):
+        K_cache[b, :, int(ctx[b])] = qkv[b, 1]
+        V_cache[b, :, int(ctx[b])] = qkv[b, 2]
+        lens.append(int(ctx[b]) + 1)
+    alpha_qk = f32(f32(p["d_q"]) * f32(p["d_k"])) / f32(np.sqrt(f32(d)))
+    alpha_pv = f32(p["d_v"]) / f32(127.0)
+    o, _ = kv_decode_attention(np.ascontiguousarray(qkv[:, 0]), K_cache, V_cache, lens, float(alpha_qk), float(alpha_pv),
+                               requant_mul=f32(1) / f32(p["d_attn"]))
+    out["attn"] = o.reshape(B, hid)
+    _, out["proj"] = w8a8_linear(out["attn"], p["d_attn"], p["out_proj"]["Wq"], p["out_proj"]["w_scale"],
+                                 bias=p["out_proj"]["bias"], out_dtype=dtype)
+    out["h"] = round_to(_f32(x) + out["proj"], dtype)
+    out["x2q"], _, _ = ln_quant(out["h"], p["g2"], p["b2"], eps, "per_tensor_static", static_scale=p["d_ln2"])
+    _, out["f1q"] = w8a8_linear(out["x2q"], p["d_ln2"], p["fc1"]["Wq"], p["fc1"]["w_scale"], bias=p["fc1"]["bias"],
+                                relu=True, requant_mul=f32(1) / f32(p["d_fc1"]))
+    _, out["fc2"] = w8a8_linear(out["f1q"], p["d_fc1"], p["fc2"]["Wq"], p["fc2"]["w_scale"], bias=p["fc2"]["bias"],
+                                out_dtype=dtype)
+    out["y"] = round_to(out["h"] + out["fc2"], dtype)
+    return out

@@ -38,6 +38,7 @@ struct DecParams {
     const float* w_scale; int w_per_col;
     const void* bias; int bias_is_bf16;
     int relu;
+    const float* requant_mul; int requant_per_col;  // INT8 output: code = round(y * r)
     void* Y; int out_dt; int64_t ldy;
     int32_t* acc;        // [16][N] scratch (splits > 1), zero on entry and on exit
     uint32_t* counters;  // [num_n]   arrivals per tile, zero on entry and on exit
@@ -70,13 +71,16 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
     if (p.bias)
         bs = p.bias_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
                             : __half2float(static_cast<const __half*>(p.bias)[col]);
+    const float rq = p.requant_mul ? __ldg(p.requant_mul + (p.requant_per_col ? col : 0)) : 1.0f;
 #pragma unroll
     for (int t = 0; t < DEC_N; ++t) {
         if (t < p.M) {
             const float xs = __ldg(p.x_scale + (p.x_per_row ? t : 0));
             float v = __fmaf_rn(__int2float_rn(acc[t]), __fmul_rn(xs, ws), bs);
             if (p.relu) v = fmaxf(v, 0.0f);
-            if (p.out_dt == SQ_BF16)
+            if (p.out_dt == SQ_I8)
+                static_cast<int8_t*>(p.Y)[(int64_t)t * p.ldy + col] = (int8_t)(quant_code(v, rq) & 0xffu);
+            else if (p.out_dt == SQ_BF16)
                 static_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.ldy + col] = __float2bfloat16_rn(v);
             else
                 static_cast<__half*>(p.Y)[(int64_t)t * p.ldy + col] = __float2half_rn(v);
@@ -300,8 +304,8 @@ size_t decode_workspace_bytes(int64_t N) {
 }
 
 bool decode_supports(const GemmArgs& a) {
-    return a.M <= DEC_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn && a.requant_mul == nullptr &&
-           a.row_absmax_out == nullptr && a.out_dt != SQ_I8 && a.strideA[2] == a.K && a.strideB[2] == a.K;
+    return a.M <= DEC_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn &&
+           a.row_absmax_out == nullptr && a.strideA[2] == a.K && a.strideB[2] == a.K;
 }
 
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st) {
@@ -317,6 +321,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
     p.bias = a.bias; p.bias_is_bf16 = a.bias_dt == SQ_BF16;
     p.relu = a.relu;
+    p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
     p.Y = a.C; p.out_dt = (int)a.out_dt; p.ldy = a.strideC[2];
     p.acc = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader);
     p.counters = reinterpret_cast<uint32_t*>(p.acc + (size_t)DEC_N * a.N);

@@ -143,6 +143,27 @@ def test_decode_gemm_exact_and_workspace_restored(ws, M, N, K):
     assert not ws[4:].any(), "workspace not handed back zero-filled"
 
 
+@pytest.mark.parametrize("M,N,K,per_col", [(1, 384, 512, True), (16, 1280, 4096, True), (7, 200, 272, False),
+                                           (16, 36864, 1024, True)])
+def test_decode_gemm_requant_int8_out(ws, M, N, K, per_col):
+    """Decode-shaped GEMM with the requantising epilogue (INT8 codes out, as the QKV and FC1
+    projections of a static-step block emit them): byte-exact, the epilogue is fully specified fp32."""
+    Xq, Wq = synth.int8_tensor(26, 1, (M, K)), synth.int8_tensor(26, 2, (N, K))
+    rng = synth.rng_for(26, 3)
+    xs = np.array([0.03], np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = synth.bias(26, 4, N, "f16", std=0.5)
+    r = rng.uniform(5.0, 40.0, N if per_col else 1).astype(np.float32)
+    acc = oracle.gemm_i32(Xq, Wq)
+    want = oracle.requant(oracle.dequant(acc, xs, wsc, bias, relu=True), r)
+    got = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True, requant_mul=dev(r))
+    assert got.dtype == torch.int8
+    assert np.array_equal(host(got), want)
+    assert np.abs(want).max() == 127 and (np.abs(want) < 127).mean() > 0.5  # saturating and non-trivial
+    assert sq.device_status(ws) == 0
+    assert not ws[4:].any()
+
+
 def test_decode_gemm_without_scratch_falls_back_to_single_split():
     M, N, K = 4, 256, 8192
     Xq, Wq = synth.int8_tensor(25, 5, (M, K)), synth.int8_tensor(25, 6, (N, K))

@@ -439,3 +439,35 @@ def test_kv_decode_attention_closed_forms_and_error_bound():
     bound = (0.5 / 127) * np.abs(V.astype(np.float64)).sum(2) * float(d_v)
     assert np.all(np.abs(out - truth) <= bound * (1 + 1e-5) + 1e-6)
     assert np.abs(out - truth).max() > 0  # the bound is not vacuous: quantising p does move the result
+
+
+def test_decode_block_continues_the_prompt_block_exactly():
+    """The generation-stage block fed with the prompt's last token and a cache holding the earlier
+    tokens' k, v codes reproduces the prompt block's last row bit for bit, at every stage."""
+    rng = np.random.default_rng(46)
+    B, S, H, d, ffn = 2, 9, 2, 8, 32
+    hid = H * d
+    x = (rng.standard_normal((B * S, hid)) * 2).astype(np.float16).astype(np.float32)
+    p = {"g1": (1 + 0.1 * rng.standard_normal(hid)).astype(np.float16).astype(np.float32),
+         "b1": (0.1 * rng.standard_normal(hid)).astype(np.float16).astype(np.float32),
+         "g2": (1 + 0.1 * rng.standard_normal(hid)).astype(np.float16).astype(np.float32),
+         "b2": (0.1 * rng.standard_normal(hid)).astype(np.float16).astype(np.float32),
+         "d_ln1": 0.03, "d_q": 0.02, "d_k": 0.02, "d_v": 0.015, "d_attn": 0.012, "d_ln2": 0.03, "d_fc1": 0.02}
+    for n, (N, K) in {"qkv": (3 * hid, hid), "out_proj": (hid, hid), "fc1": (ffn, hid), "fc2": (hid, ffn)}.items():
+        p[n] = {"Wq": rng.integers(-127, 128, (N, K), dtype=np.int8),
+                "w_scale": rng.uniform(5e-4, 2e-3, N).astype(np.float32),
+                "bias": (0.05 * rng.standard_normal(N)).astype(np.float16).astype(np.float32)}
+    prompt = oracle.decoder_block_static(x, p, B, S, H, d, "f16", score_dtype="f32")
+    qkv = prompt["qkv"].reshape(B, S, 3, H, d)
+    L_max = 12
+    Kc = np.zeros((B, H, L_max, d), np.int8)
+    Vc = np.zeros((B, H, L_max, d), np.int8)
+    Kc[:, :, :S - 1] = qkv[:, :S - 1, 1].transpose(0, 2, 1, 3)
+    Vc[:, :, :S - 1] = qkv[:, :S - 1, 2].transpose(0, 2, 1, 3)
+    x_last = x.reshape(B, S, hid)[:, -1]
+    dec = oracle.decoder_block_static_decode(x_last, p, Kc, Vc, [S - 1, S - 1], H, d, "f16")
+    for key in ("x1q", "qkv", "attn", "proj", "h", "x2q", "f1q", "fc2", "y"):
+        want = prompt[key].reshape(B, S, -1)[:, -1]
+        assert np.array_equal(dec[key], want), key
+    assert np.array_equal(Kc[:, :, S - 1], qkv[:, S - 1, 1]) and np.array_equal(Vc[:, :, S - 1], qkv[:, S - 1, 2])
+    assert np.abs(prompt["attn"]).max() > 10 and np.abs(prompt["y"]).max() > 0.5  # not a vacuous comparison
