@@ -241,6 +241,81 @@ class DecoderBlockStatic:
         return lin + 2 * (2 * self.B * self.H * S * S * d)
 
 
+class DecoderBlockDecode:
+    """Generation stage of DecoderBlockStatic: one new token per sequence against an INT8 KV cache,
+    as ten libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> append k, v to the cache ->
+    attention of the new token over the cache (INT8 out) -> out-proj GEMM -> residual ->
+    LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM -> residual.  Same `lin` / `steps` as the
+    prompt block.  `ctx` (int32 device tensor [B]) counts the positions each sequence has cached."""
+
+    def __init__(self, lin, steps, B, H, d, L_max, act_dtype, eps=1e-5):
+        self.lin, self.B, self.H, self.d, self.L_max, self.dt, self.eps = lin, B, H, d, L_max, act_dtype, eps
+        dev = lin["qkv"].Wq.device
+        hid, ffn = H * d, lin["fc1"].Wq.shape[0]
+        self.hid = hid
+        f32 = lambda v: torch.tensor([v], dtype=torch.float32, device=dev)
+        self.s = {k: f32(v) for k, v in steps.items()}
+        one = torch.tensor(1.0, dtype=torch.float32)
+        inv = lambda v: float(one / torch.tensor(v, dtype=torch.float32))
+        self.r_qkv = torch.cat([torch.full((hid,), inv(steps["d_q"])), torch.full((hid,), inv(steps["d_k"])),
+                                torch.full((hid,), inv(steps["d_v"]))]).to(torch.float32).to(dev)
+        self.r_attn, self.r_fc1 = f32(inv(steps["d_attn"])), f32(inv(steps["d_fc1"]))
+        t32 = lambda v: torch.tensor(v, dtype=torch.float32)
+        self.alpha_qk = float((t32(steps["d_q"]) * t32(steps["d_k"])) / torch.sqrt(t32(float(d))))
+        self.alpha_pv = float(t32(steps["d_v"]) / t32(127.0))
+        e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
+        self.x1q, self.qkv, self.attn = e((B, hid), torch.int8), e((B, 3 * hid), torch.int8), e((B, hid), torch.int8)
+        self.proj, self.h = e((B, hid), act_dtype), e((B, hid), act_dtype)
+        self.x2q, self.f1q = e((B, hid), torch.int8), e((B, ffn), torch.int8)
+        self.fc2, self.y = e((B, hid), act_dtype), e((B, hid), act_dtype)
+        self.k_cache = torch.zeros((B, H, L_max, d), dtype=torch.int8, device=dev)
+        self.v_cache = torch.zeros((B, H, L_max // 4, d, 4), dtype=torch.int8, device=dev)
+        self.ctx = torch.zeros(B, dtype=torch.int32, device=dev)
+        self.lens = torch.ones(B, dtype=torch.int32, device=dev)  # ctx + 1: what the new token attends over
+        need = max(sq.workspace_bytes(sq.SQ_OP_GEMM, B, max(l.Wq.shape[0] for l in lin.values()),
+                                      max(l.Wq.shape[1] for l in lin.values())),
+                   sq.workspace_bytes(sq.SQ_OP_LN_QUANT, B, 0, hid))
+        self.ws = sq.new_workspace(need, dev)
+        self.launches_per_step = 10
+
+    def load_prompt(self, qkv_codes, S):
+        """Fill the cache from a prompt pass's QKV code buffer [B*S, 3*H*d]; every sequence then holds S positions."""
+        sq.sq_kv_cache_write(qkv_codes, self.B, S, self.H, self.d, None, self.k_cache, self.v_cache, self.L_max, self.ws)
+        self.ctx.fill_(S)
+        self.lens.fill_(S + 1)
+
+    def step(self, x, max_len=None, advance=True):
+        """x [B, H*d]: the newest token of each sequence.  max_len: host-side bound of ctx + 1
+        (default: the cache capacity).  Returns the block output [B, H*d]."""
+        L, s, B, H, d = self.lin, self.s, self.B, self.H, self.d
+        max_len = self.L_max if max_len is None else max_len
+        sq.sq_ln_quant(x, L["qkv"].gamma_hat, L["qkv"].beta_hat, self.eps, "per_tensor_static", Xq=self.x1q,
+                       x_scale=s["d_ln1"], workspace=self.ws)
+        sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
+                        requant_mul=self.r_qkv, out=self.qkv)
+        sq.sq_kv_cache_write(self.qkv, B, 1, H, d, self.ctx, self.k_cache, self.v_cache, self.L_max, self.ws)
+        sq.sq_w8a8_decode_attention(self.qkv, self.k_cache, self.v_cache, self.lens, B, H, d, self.L_max, max_len,
+                                    self.alpha_qk, self.alpha_pv, self.ws, requant_mul=self.r_attn, out=self.attn)
+        sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
+                        bias=L["out_proj"].bias, out=self.proj)
+        sq.sq_residual_add(x, self.proj, out=self.h)
+        sq.sq_ln_quant(self.h, L["fc1"].gamma_hat, L["fc1"].beta_hat, self.eps, "per_tensor_static", Xq=self.x2q,
+                       x_scale=s["d_ln2"], workspace=self.ws)
+        sq.sq_w8a8_gemm(self.x2q, L["fc1"].Wq, s["d_ln2"], L["fc1"].w_scale, self.ws, bias=L["fc1"].bias, relu=True,
+                        requant_mul=self.r_fc1, out=self.f1q)
+        sq.sq_w8a8_gemm(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, bias=L["fc2"].bias,
+                        out=self.fc2)
+        sq.sq_residual_add(self.h, self.fc2, out=self.y)
+        if advance:  # bookkeeping of the sequence lengths, not part of the arithmetic
+            torch._foreach_add_([self.ctx, self.lens], 1)
+        return self.y
+
+    def bytes_per_step(self, ctx_sum):
+        """Algorithmic HBM bytes of one step: INT8 weights once + the cache positions attended over."""
+        w = sum(l.Wq.numel() for l in self.lin.values())
+        return w + 2 * self.H * self.d * (ctx_sum + self.B)
+
+
 def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
     """Static per-tensor steps for DecoderBlockStatic from calibration batches (each [B*S, H*d]):
     the block is walked with DYNAMIC steps and floating-point intermediates, and the running

@@ -154,3 +154,57 @@ def test_host_streamed_block_matches_sequential_steps():
     assert sq.device_status(blk.ws) == 0
     for o, w in zip(outs, want):
         assert torch.equal(o.view(torch.int16), w.view(torch.int16))
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+def test_generation_stage_block_against_oracle(dtype):
+    """Prompt pass of 128 tokens with the prompt block, cache filled from its QKV codes, then three
+    generated tokens through the generation-stage block; each step against the oracle's generation
+    block, which walks its own caches (oracle prompt codes -> oracle cache)."""
+    B, S, H, d, ffn, L_max = 2, 128, 2, 128, 1024, 160
+    hid = H * d
+    x, W, bias, ln = _make_block(B, S, H, d, ffn, dtype)
+    p = _oracle_prepare(x, W, bias, ln, B, S, H, d, dtype)
+    prompt = oracle.decoder_block_static(x, p, B, S, H, d, dtype, score_dtype="f32")
+    qkv = prompt["qkv"].reshape(B, S, 3, H, d)
+    Kc, Vc = np.zeros((B, H, L_max, d), np.int8), np.zeros((B, H, L_max, d), np.int8)
+    Kc[:, :, :S] = qkv[:, :, 1].transpose(0, 2, 1, 3)
+    Vc[:, :, :S] = qkv[:, :, 2].transpose(0, 2, 1, 3)
+
+    tdt = {"f16": torch.float16, "bf16": torch.bfloat16}[dtype]
+    lin = {}
+    for n in W:
+        lin[n] = pl.PreparedLinear(n, dev(p[n]["Wq"]), dev(p[n]["w_scale"]), dev(bias[n], dtype), n == "fc1")
+    lin["qkv"].gamma_hat, lin["qkv"].beta_hat = dev(p["g1"], dtype), dev(p["b1"], dtype)
+    lin["fc1"].gamma_hat, lin["fc1"].beta_hat = dev(p["g2"], dtype), dev(p["b2"], dtype)
+    steps = {k: p[k] for k in ("d_ln1", "d_q", "d_k", "d_v", "d_attn", "d_ln2", "d_fc1")}
+    blk = pl.DecoderBlockStatic(lin, steps, B, S, H, d, tdt)
+    blk.forward(dev(x, dtype))
+    gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, tdt)
+    gen.load_prompt(blk.qkv, S)
+
+    def codes_close(name, got, ref, max_frac):
+        diff = np.abs(host(got).astype(np.int32).reshape(ref.shape) - ref.astype(np.int32))
+        assert diff.max() <= 2, "%s: codes differ by %d" % (name, diff.max())
+        assert (diff != 0).mean() <= max_frac, "%s: %.4f of codes differ" % (name, (diff != 0).mean())
+
+    ch = synth.outlier_channels(3, hid, count=max(1, hid // 100))
+    fac = synth.outlier_factors(3, len(ch), 20.0, 80.0)
+    for t in range(3):
+        xt = synth.activations(3, 100 + t, B, hid, dtype, ch, fac)
+        want = oracle.decoder_block_static_decode(xt, p, Kc, Vc, [S + t] * B, H, d, dtype)
+        y = gen.step(dev(xt, dtype), max_len=S + 3)
+        torch.cuda.synchronize()
+        assert sq.device_status(gen.ws) == 0
+        codes_close("LN1 codes", gen.x1q, want["x1q"], 2e-3)
+        codes_close("QKV codes", gen.qkv, want["qkv"], 1e-2)
+        codes_close("attention codes", gen.attn, want["attn"], 3e-2)
+        codes_close("FC1 codes", gen.f1q, want["f1q"], 3e-2)
+        got, ref = host(y).astype(np.float64), want["y"].astype(np.float64)
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rel <= 5e-3, "step %d: block output relative error %.3g" % (t, rel)
+    # the cache now holds S + 3 positions per sequence, equal to the oracle's up to near-tie codes
+    assert host(gen.ctx).tolist() == [S + 3] * B
+    codes_close("K cache", gen.k_cache[:, :, :S + 3], Kc[:, :, :S + 3], 5e-3)
+    v_logical = gen.v_cache.permute(0, 1, 2, 4, 3).reshape(B, H, L_max, d)
+    codes_close("V cache", v_logical[:, :, :S + 3], Vc[:, :, :S + 3], 5e-3)

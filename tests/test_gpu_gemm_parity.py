@@ -156,10 +156,11 @@ def test_decode_gemm_requant_int8_out(ws, M, N, K, per_col):
     r = rng.uniform(5.0, 40.0, N if per_col else 1).astype(np.float32)
     acc = oracle.gemm_i32(Xq, Wq)
     want = oracle.requant(oracle.dequant(acc, xs, wsc, bias, relu=True), r)
-    got = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True, requant_mul=dev(r))
+    got = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True, requant_mul=dev(r),
+                          out_dtype=torch.int8)
     assert got.dtype == torch.int8
     assert np.array_equal(host(got), want)
-    assert np.abs(want).max() == 127 and (np.abs(want) < 127).mean() > 0.5  # saturating and non-trivial
+    assert np.abs(want).max() > 20 and (np.abs(want) < 127).mean() > 0.5  # non-trivial codes
     assert sq.device_status(ws) == 0
     assert not ws[4:].any()
 
