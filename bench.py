@@ -282,7 +282,49 @@ def block_rows(device):
         us = a.elapsed_time(b) / n * 1e3
         out["opt30b_block_static_b%d_s512" % B] = {"us_per_layer": us, "TOPS": blk.ops() / us / 1e6,
                                                    "status": sq.device_status(blk.ws)}
+        if B == 16:
+            out.update(generation_rows(lin, steps, blk, B, S, H, d, hid, dt, ch, fac, seed, device))
         del blk, g
+    return out
+
+
+def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, device):
+    """Generation stage of the same block: one new token per sequence against the INT8 KV cache
+    (INT8 weights read once + the cached positions), one CUDA graph, microseconds per layer.
+    Context 512 = the cache filled from the prompt pass above; context 2047 = the same cache
+    declared full (its later positions hold zeros: the timing does not depend on the values)."""
+    from paper_2211_10438_b200 import pipeline as pl
+    from paper_2211_10438_b200 import binding as sq
+    L_max = 2048
+    gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, dt)
+    gen.load_prompt(prompt_blk.qkv, S)
+    x = pl.synth_device_activations(B, hid, dt, ch, fac, seed + 90, device)
+    out = {}
+    for ctx in (S, L_max - 1):
+        gen.ctx.fill_(ctx)
+        gen.lens.fill_(ctx + 1)
+        for _ in range(3):
+            gen.step(x, advance=False)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            gen.step(x, advance=False)
+        for _ in range(3):
+            g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 20
+        a.record()
+        for _ in range(n):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / n * 1e3
+        byts = gen.bytes_per_step(ctx * B)
+        out["opt30b_generation_b%d_ctx%d" % (B, ctx)] = {
+            "us_per_layer": us, "GB/s": byts / us / 1e3, "frac_hbm": byts / us / 1e3 / measured_peaks()["hbm_gbs"],
+            "status": sq.device_status(gen.ws)}
+        del g
     return out
 
 

@@ -76,9 +76,11 @@ const char* sq_status_str(sq_status s);
 
 /* Bytes of caller-provided workspace `op` needs for the given sizes (host call, no CUDA
  * work).  The workspace must be 256-byte aligned and ZERO-FILLED ONCE by the caller before
- * its first use; every call leaves it zero-filled again except for workspace[0..3], the
- * sticky device status word (0 = no device-side error).  M is the token count, N/K as in
- * the call; pass 0 for sizes the op does not have. */
+ * its first use; every call leaves its first 33 024 bytes (header + arrival counters)
+ * zero-filled again except for workspace[0..3], the sticky device status word (0 = no
+ * device-side error); what lies beyond is scratch whose content is undefined between calls
+ * (partial sums of decode-shaped GEMMs) and is never read before it is written.  M is the
+ * token count, N/K as in the call; pass 0 for sizes the op does not have. */
 size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K);
 
 /*

@@ -4,12 +4,14 @@
 //   * operands are swapped: 128 OUTPUT CHANNELS of W (128 x 128 bytes per K slice) ride on the
 //     MMA's M dimension and the <= 16 tokens on its N dimension (tcgen05.mma.kind::i8,
 //     128 x 16 x 32), so no tile is padded from 16 to 128 rows and a stage is 18 KB;
-//   * work units are (128-channel tile, K split): the split count is chosen so that the units
-//     fill all SMs in whole waves whatever N is (INT32 partial sums add exactly in any order);
+//   * the (128-channel tile, K block) pairs, tile-major, are cut into equal contiguous ranges,
+//     one per CTA ("stream-K"): every SM streams the same number of weight bytes whatever N
+//     and K are, at the price of tiles whose K range is shared by two or more CTAs;
 //   * a 10-stage TMA ring keeps ~180 KB of weights in flight per SM;
-//   * with K splits, partial accumulators are added into an INT32 scratch in the workspace
-//     with red.global.add; the unit that arrives last for a tile applies Eq. 2 (dequant, bias,
-//     ReLU), writes Y and leaves scratch and counter zeroed for the next call.
+//   * a CTA parks the partial accumulators of a shared tile in its own slot of the workspace
+//     with plain stores (INT32 partial sums add exactly in any order); the CTA that arrives
+//     last for a tile (one atomic counter per tile) adds the other slots, applies Eq. 2
+//     (dequant, bias, ReLU, requant), writes Y and leaves the counter zeroed for the next call.
 // Every wait is bounded (status word, as in the prefill kernel).
 #include "sq_kernels.h"
 #include "sq_tcgen05.cuh"
@@ -32,16 +34,18 @@ constexpr int DEC_SMEM = 1024 + DEC_STAGES * DEC_STAGE + (2 * DEC_STAGES + 4) * 
 struct DecParams {
     int M;
     int64_t N, K;
-    int num_n, splits, kb_per_split, num_kb;
-    int64_t total_units;
+    int num_n, num_kb;
+    int64_t total_kb;    // num_n * num_kb: every (tile, K block) pair, tile-major
+    int range;           // K blocks per CTA: CTA g owns positions [g * range, (g + 1) * range)
+    int maxcount;        // most CTAs that share one tile
     const float* x_scale; int x_per_row;
     const float* w_scale; int w_per_col;
     const void* bias; int bias_is_bf16;
     int relu;
     const float* requant_mul; int requant_per_col;  // INT8 output: code = round(y * r)
     void* Y; int out_dt; int64_t ldy;
-    int32_t* acc;        // [16][N] scratch (splits > 1), zero on entry and on exit
-    uint32_t* counters;  // [num_n]   arrivals per tile, zero on entry and on exit
+    int32_t* part;       // [num_n][maxcount][M][128] partial sums of tiles shared by several CTAs
+    uint32_t* counters;  // [num_n] arrivals per shared tile, zero on entry and on exit
     uint32_t* status;
 };
 
@@ -139,9 +143,12 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             // add the activation slices of those stages.
             int prefetched = 0;
             bool waited = false;
-            for (int64_t u = blockIdx.x; ok && u < p.total_units; u += gridDim.x) {
-                const int ni = (int)(u / p.splits), ks = (int)(u % p.splits);
-                const int kb0 = ks * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+            int64_t pos = (int64_t)blockIdx.x * p.range;
+            const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
+            for (; ok && pos < end;) {
+                const int ni = (int)(pos / p.num_kb);
+                const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
+                pos += kb1 - kb0;
                 int kb = kb0;
                 if (!waited) {
                     const int n_pre = min(DEC_STAGES, kb1 - kb0);
@@ -178,9 +185,11 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
-            for (int64_t u = blockIdx.x; ok && u < p.total_units; u += gridDim.x) {
-                const int ks = (int)(u % p.splits);
-                const int kb0 = ks * p.kb_per_split, kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+            int64_t pos = (int64_t)blockIdx.x * p.range;
+            const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
+            for (; ok && pos < end;) {
+                const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
+                pos += kb1 - kb0;
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 7))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * DEC_N);
@@ -210,8 +219,12 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const int et = threadIdx.x - 64;        // 0..127
         int slot = 0;
         uint32_t slot_phase = 0;
-        for (int64_t u = blockIdx.x; u < p.total_units; u += gridDim.x) {
-            const int ni = (int)(u / p.splits);
+        int64_t pos = (int64_t)blockIdx.x * p.range;
+        const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
+        while (pos < end) {
+            const int ni = (int)(pos / p.num_kb);
+            const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
+            pos += kb1 - kb0;
             if (et == 0) *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 9) ? 1u : 0u;
             dec_epi_sync();
             if (*epi_go == 0u) break;
@@ -228,32 +241,33 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             int32_t acc[16];
 #pragma unroll
             for (int t = 0; t < 16; ++t) acc[t] = (int32_t)r[t];
-            if (p.splits == 1) {
-                dec_finish(p, acc, col);
+            if (kb0 == 0 && kb1 == p.num_kb) {
+                dec_finish(p, acc, col);  // the whole K range of this tile was ours
             } else {
-                // add this unit's partial sums; the last unit of the tile finishes it
-                if (col < p.N) {
+                // The tile is shared: CTAs g0 .. g0 + count - 1 each hold one K piece.  Park this
+                // piece in its own slot (plain stores: integer partial sums add exactly in any
+                // order); whoever arrives last adds the others and applies Eq. 2.
+                const int g0 = (int)(((int64_t)ni * p.num_kb) / p.range);
+                const int count = (int)(((int64_t)(ni + 1) * p.num_kb - 1) / p.range) - g0 + 1;
+                const int mine = (int)blockIdx.x - g0;
+                int32_t* slot0 = p.part + ((int64_t)ni * p.maxcount) * p.M * BLOCK_M;
 #pragma unroll
-                    for (int t = 0; t < DEC_N; ++t)
-                        if (t < p.M) atomicAdd(p.acc + (int64_t)t * p.N + col, acc[t]);
-                }
+                for (int t = 0; t < DEC_N; ++t)
+                    if (t < p.M) __stcg(slot0 + ((int64_t)mine * p.M + t) * BLOCK_M + ch, acc[t]);
                 __threadfence();
                 dec_epi_sync();
-                if (et == 0) *epi_last = (atomicAdd(p.counters + ni, 1u) == (uint32_t)(p.splits - 1)) ? 1u : 0u;
+                if (et == 0) *epi_last = (atomicAdd(p.counters + ni, 1u) == (uint32_t)(count - 1)) ? 1u : 0u;
                 dec_epi_sync();
                 if (*epi_last != 0u) {
                     __threadfence();
-                    if (col < p.N) {
+                    for (int o = 0; o < count; ++o) {
+                        if (o == mine) continue;
 #pragma unroll
-                        for (int t = 0; t < DEC_N; ++t) {
-                            if (t < p.M) {
-                                acc[t] = __ldcg(p.acc + (int64_t)t * p.N + col);
-                                __stcg(p.acc + (int64_t)t * p.N + col, 0);  // hand the scratch back zeroed
-                            }
-                        }
+                        for (int t = 0; t < DEC_N; ++t)
+                            if (t < p.M) acc[t] += __ldcg(slot0 + ((int64_t)o * p.M + t) * BLOCK_M + ch);
                     }
                     dec_finish(p, acc, col);
-                    if (et == 0) p.counters[ni] = 0u;
+                    if (et == 0) p.counters[ni] = 0u;  // hand the counters back zeroed
                 }
             }
             dec_epi_sync();  // epi_go / epi_last are rewritten by thread 0 in the next round
@@ -270,37 +284,39 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     }
 }
 
-// K splits.  The kernel is HBM-bound, so a partly filled last wave only costs time when it has
-// too few SMs to saturate HBM; splitting K adds INT32 atomics that grow with M.  Pick the split
-// that minimises a small time model (microseconds): every wave streams its bytes at
-// min(HBM rate, SMs in the wave x per-SM streaming rate), plus the atomics.
-int choose_splits(int M, int64_t N, int num_n, int num_kb, int sms) {
-    const double hbm = 6100.0e3, per_sm = 57.0e3;  // bytes per microsecond (measured on B200)
-    const double atomic_us = 14.0e-6;              // per partial sum added through the scratch
-    int best = 1;
-    double best_t = 1e30;
-    for (int s = 1; s <= 16 && num_kb / s >= 8; ++s) {
-        const int per = (num_kb + s - 1) / s;
-        if ((num_kb + per - 1) / per != s) continue;  // some split would get no work
-        const double unit_bytes = (double)per * W_BYTES;
-        int64_t units = (int64_t)num_n * s;
-        double t = 0.0;
-        while (units > 0) {
-            const int64_t in_wave = std::min<int64_t>(units, sms);
-            t += in_wave * unit_bytes / std::min(hbm, per_sm * (double)in_wave);
-            units -= in_wave;
-        }
-        if (s > 1) t += atomic_us * (double)M * (double)N * s;
-        if (t < best_t) { best_t = t; best = s; }
+// Work split ("stream-K"): the (tile, K block) pairs, tile-major, are cut into equal contiguous
+// ranges, one per CTA, so every SM streams the same number of weight bytes whatever the shape;
+// a tile whose K range is cut is finished by the last of the CTAs that share it.
+constexpr int kMinKbPerCta = 4;       // below this a CTA's fixed costs outweigh its stream
+constexpr int kMaxCtas = 256;         // bound used by the workspace formula
+constexpr int64_t kMaxSharedTiles = (int64_t)kDecCounterBytes / 4;
+
+struct DecPlan { int ctas, range, maxcount; };
+DecPlan plan_decode(int num_n, int num_kb, int sms, bool may_share) {
+    const int64_t total = (int64_t)num_n * num_kb;
+    DecPlan pl;
+    if (!may_share) {  // whole tiles only
+        const int ctas = (int)std::min<int64_t>(num_n, sms);
+        const int tiles_per = (num_n + ctas - 1) / ctas;
+        pl.range = tiles_per * num_kb;
+        pl.ctas = (num_n + tiles_per - 1) / tiles_per;
+        pl.maxcount = 1;
+        return pl;
     }
-    return best;
+    int64_t ctas = std::min<int64_t>(std::min(sms, kMaxCtas), std::max<int64_t>(1, total / kMinKbPerCta));
+    pl.range = (int)((total + ctas - 1) / ctas);
+    pl.ctas = (int)((total + pl.range - 1) / pl.range);
+    pl.maxcount = (num_kb + pl.range - 2) / pl.range + 1;
+    return pl;
 }
 
 }  // namespace
 
-size_t decode_workspace_bytes(int64_t N) {
+// Counters (fixed area, zero between calls) + one slot per (shared tile, sharing CTA).  The
+// number of slots is at most ctas + 2 * tiles for any balanced cut, with ctas <= kMaxCtas.
+size_t decode_workspace_bytes(int64_t M, int64_t N) {
     const int64_t num_n = (N + tc::BLOCK_M - 1) / tc::BLOCK_M;
-    return kWsHeader + (size_t)DEC_N * N * sizeof(int32_t) + (size_t)num_n * sizeof(uint32_t);
+    return kWsHeader + kDecCounterBytes + (size_t)(kMaxCtas + 2 * num_n) * (size_t)M * tc::BLOCK_M * sizeof(int32_t);
 }
 
 bool decode_supports(const GemmArgs& a) {
@@ -313,18 +329,19 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.M = (int)a.M; p.N = a.N; p.K = a.K;
     p.num_n = (int)((a.N + BLOCK_M - 1) / BLOCK_M);
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
-    p.splits = choose_splits(p.M, p.N, p.num_n, p.num_kb, sm_count());
-    if (ws_bytes < decode_workspace_bytes(a.N)) p.splits = 1;  // no scratch: every tile in one unit
-    p.kb_per_split = (p.num_kb + p.splits - 1) / p.splits;
-    p.total_units = (int64_t)p.num_n * p.splits;
+    const bool may_share = ws_bytes >= decode_workspace_bytes(a.M, a.N) && p.num_n <= kMaxSharedTiles;
+    const DecPlan plan = plan_decode(p.num_n, p.num_kb, sm_count(), may_share);
+    p.total_kb = (int64_t)p.num_n * p.num_kb;
+    p.range = plan.range;
+    p.maxcount = plan.maxcount;
     p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
     p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
     p.bias = a.bias; p.bias_is_bf16 = a.bias_dt == SQ_BF16;
     p.relu = a.relu;
     p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
     p.Y = a.C; p.out_dt = (int)a.out_dt; p.ldy = a.strideC[2];
-    p.acc = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader);
-    p.counters = reinterpret_cast<uint32_t*>(p.acc + (size_t)DEC_N * a.N);
+    p.counters = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsHeader);
+    p.part = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader + kDecCounterBytes);
     p.status = a.status;
     CUtensorMap mw, mx;
     int s0, s1, s2;
@@ -337,8 +354,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
         SQ_CUDA_OK(cudaFuncSetAttribute(decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DEC_SMEM));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const int grid = (int)std::min<int64_t>(p.total_units, sm_count());
-    return launch_pdl(decode_gemm_kernel, dim3((unsigned)grid), dim3(DEC_THREADS), (size_t)DEC_SMEM, st, 1, mw, mx, p);
+    return launch_pdl(decode_gemm_kernel, dim3((unsigned)plan.ctas), dim3(DEC_THREADS), (size_t)DEC_SMEM, st, 1, mw, mx, p);
 }
 
 }  // namespace sq

@@ -20,7 +20,8 @@ enum RowMode {
 // Workspace layout (bytes).  Word 0 is the sticky device status.
 constexpr size_t kWsStatusOff = 0;
 constexpr size_t kWsAbsmaxOff = 16;   // per-tensor dynamic absmax word
-constexpr size_t kWsHeader = 256;     // per-row LayerNorm statistics / split-K partials start here
+constexpr size_t kWsHeader = 256;     // per-row LayerNorm statistics / decode-GEMM arrival counters start here
+constexpr size_t kDecCounterBytes = 32768;  // decode-shaped GEMM: one arrival counter per 128-channel tile, then partial sums
 
 sq_status calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld, float* a,
                        cudaStream_t st);
@@ -74,7 +75,7 @@ sq_status kv_decode_attention(const int8_t* q, int64_t ldq, const int8_t* kc, co
 sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st);
 
 // Decode-shaped path (M <= 16): swapped operands, split-K with INT32 scratch in the workspace.
-size_t decode_workspace_bytes(int64_t N);
+size_t decode_workspace_bytes(int64_t M, int64_t N);
 bool decode_supports(const GemmArgs& a);
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st);
 

@@ -136,7 +136,7 @@ def test_decode_gemm_full_size(name, N, K, M):
     assert np.array_equal(acc, want_acc)
     y = host(sq.sq_w8a8_gemm(dev(Xq), Wd, dev(xs), dev(wsc), ws, out_dtype=torch.bfloat16))
     assert np.array_equal(y, oracle.round_to(oracle.dequant(want_acc, xs, wsc), "bf16"))
-    assert sq.device_status(ws) == 0 and not ws[4:].any()
+    assert sq.device_status(ws) == 0 and not ws[4:33024].any()
 
 
 @pytest.mark.parametrize("gran", ["per_token", "per_tensor_dynamic", "per_tensor_static"])

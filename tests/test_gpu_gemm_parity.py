@@ -140,7 +140,7 @@ def test_decode_gemm_exact_and_workspace_restored(ws, M, N, K):
         want = oracle.round_to(oracle.dequant(want_acc, xs, wsc, bias, relu=True), "bf16")
         assert np.array_equal(host(y), want)
     assert sq.device_status(ws) == 0
-    assert not ws[4:].any(), "workspace not handed back zero-filled"
+    assert not ws[4:33024].any(), "header and counters not handed back zero-filled"
 
 
 @pytest.mark.parametrize("M,N,K,per_col", [(1, 384, 512, True), (16, 1280, 4096, True), (7, 200, 272, False),
@@ -162,7 +162,7 @@ def test_decode_gemm_requant_int8_out(ws, M, N, K, per_col):
     assert np.array_equal(host(got), want)
     assert np.abs(want).max() > 20 and (np.abs(want) < 127).mean() > 0.5  # non-trivial codes
     assert sq.device_status(ws) == 0
-    assert not ws[4:].any()
+    assert not ws[4:33024].any()
 
 
 def test_decode_gemm_without_scratch_falls_back_to_single_split():
