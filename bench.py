@@ -147,6 +147,8 @@ def timed_rows(device, peaks):
     rows = {}
 
     def t(fn, n=10):
+        torch.cuda.synchronize()
+        time.sleep(0.2)  # let the clocks recover from the previous row: every row starts from idle
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
@@ -174,7 +176,27 @@ def timed_rows(device, peaks):
     rows["ln_quant_per_token_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
     s = t(lambda: sq.sq_calib_absmax(x, a))
     rows["calib_absmax_16384x20480"] = {"GB/s": 2 * M * C / s / 1e9, "frac_hbm": 2 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    # the other two activation granularities of Table 2: one step for the whole tensor, given
+    # (static, 3 B/element) or found by a first pass over the tensor (dynamic, 5 B/element here:
+    # 671 MB does not stay in L2 between the passes)
+    xs1 = torch.full((1,), 0.05, dtype=torch.float32, device=device)
+    s = t(lambda: sq.sq_quant_act(x, "per_tensor_static", Xq=Xq, x_scale=xs1, workspace=ws))
+    rows["quant_act_per_tensor_static_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    s = t(lambda: sq.sq_quant_act(x, "per_tensor_dynamic", Xq=Xq, x_scale=xs1, workspace=ws))
+    rows["quant_act_per_tensor_dynamic_16384x20480"] = {"GB/s": 5 * M * C / s / 1e9, "frac_hbm": 5 * M * C / s / 1e9 / peaks["hbm_gbs"],
+                                                        "us": s * 1e6}
     del x, Xq
+    # offline: fold the smoothing factors into the largest MT-NLG weight and quantise it per output
+    # channel (81920 x 20480 bf16, 3.4 GB in, 1.7 GB out)
+    Nw, Kw = 81920, 20480
+    Wb = torch.randn((Nw, Kw), device=device, dtype=torch.bfloat16)
+    sm = torch.rand(Kw, device=device) + 0.5
+    Wq8 = torch.empty((Nw, Kw), dtype=torch.int8, device=device)
+    wsc = torch.empty(Nw, dtype=torch.float32, device=device)
+    s = t(lambda: sq.sq_quant_weight(Wb, sm, "per_channel", Wq=Wq8, w_scale=wsc, workspace=ws), n=5)
+    rows["quant_weight_fold_81920x20480"] = {"GB/s": 3 * Nw * Kw / s / 1e9, "frac_hbm": 3 * Nw * Kw / s / 1e9 / peaks["hbm_gbs"],
+                                             "ms": s * 1e3}
+    del Wb, Wq8
     # generation-stage attention over an INT8 KV cache, GPT-3-175B heads (96 x 128), context up to
     # 2048 with a seeded length mix (uniform in [1024, 2048]); the newest token's k, v are appended
     # by sq_kv_cache_write inside the timed call.  Cache sizes 0.8 / 3.2 GB exceed L2.
@@ -269,6 +291,7 @@ def block_rows(device):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             blk.forward(x)
+        time.sleep(0.2)  # start from idle clocks, like every other row
         for _ in range(3):
             g.replay()
         torch.cuda.synchronize()
@@ -309,6 +332,7 @@ def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, 
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             gen.step(x, advance=False)
+        time.sleep(0.2)
         for _ in range(3):
             g.replay()
         torch.cuda.synchronize()
