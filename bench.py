@@ -199,7 +199,7 @@ def timed_rows(device, peaks):
     del Wb, Wq8
     # generation-stage attention over an INT8 KV cache, GPT-3-175B heads (96 x 128), context up to
     # 2048 with a seeded length mix (uniform in [1024, 2048]); the newest token's k, v are appended
-    # by sq_kv_cache_write inside the timed call.  Cache sizes 0.8 / 3.2 GB exceed L2.
+    # by the attention kernel itself.  Cache sizes 0.8 / 3.2 GB exceed L2.
     H, D, L = 96, 128, 2048
     gen = torch.Generator(device=device)
     gen.manual_seed(0x5EED0400)
@@ -208,13 +208,12 @@ def timed_rows(device, peaks):
         vc = torch.randint(-100, 101, (Bk, H, L // 4, D, 4), dtype=torch.int8, device=device, generator=gen)
         qkv = torch.randint(-100, 101, (Bk, 3 * H * D), dtype=torch.int8, device=device, generator=gen)
         lens = torch.randint(L // 2, L + 1, (Bk,), dtype=torch.int32, device=device, generator=gen)
-        pos = lens - 1
         out = torch.empty((Bk, H * D), dtype=torch.int8, device=device)
         r = torch.tensor([1000.0], device=device)
 
-        def call():
-            sq.sq_kv_cache_write(qkv, Bk, 1, H, D, pos, kc, vc, L, ws)
-            sq.sq_w8a8_decode_attention(qkv, kc, vc, lens, Bk, H, D, L, L, 0.0009, 0.01 / 127, ws, requant_mul=r, out=out)
+        def call():  # one launch: the kernel takes the newest k, v from the QKV rows and appends them itself
+            sq.sq_w8a8_decode_attention(qkv, kc, vc, lens, Bk, H, D, L, L, 0.0009, 0.01 / 127, ws, requant_mul=r, out=out,
+                                        k_new=qkv[:, H * D:], v_new=qkv[:, 2 * H * D:])
         s = t(call)
         byts = 2 * H * D * int(lens.sum().item()) + 4 * Bk * H * D  # cache read + q, k, v, out rows
         rows["kv_decode_attention_gpt3_b%d_ctx1024-2048" % Bk] = {

@@ -292,16 +292,24 @@ sq_status sq_kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T,
  * given shape the result is deterministic.  alpha_qk must be positive.
  * q: [B, ldq] int8, head h at columns h*d .. (it may point into the QKV code buffer, ldq = 3*H*d);
  * k_cache / v_cache: as above; seq_lens: device pointer to B int32, the number of valid positions
- * INCLUDING the newest token (whose k, v the caller has already written); max_len: a host-side
- * upper bound of seq_lens[] (<= L_max) that sizes shared memory and the split of one sequence
- * over a thread-block cluster -- a longer sequence is truncated to max_len and the device status
- * word is set (SQ_ERR_SHAPE); seq_lens[b] <= 0 gives a zero output row.
+ * INCLUDING the newest token.  k_new / v_new (both NULL, or both given): [B, ld_new] int8 rows
+ * holding the newest token's k and v codes (head h at columns h*d ..; they may point into the
+ * QKV code buffer).  When NULL the caller has already written them to the cache
+ * (sq_kv_cache_write with T = 1).  When given, position seq_lens[b] - 1 of the cache is NOT read:
+ * its key and value are taken from these rows, and the kernel stores them at that position
+ * for the steps to come -- one launch less per generated token; the result is the same.
+ * max_len: a host-side upper bound of seq_lens[] (<= L_max) that sizes shared memory and the
+ * split of one sequence over a thread-block cluster -- a longer sequence is truncated to max_len
+ * and the device status word is set (SQ_ERR_SHAPE); seq_lens[b] <= 0 gives a zero output row
+ * (and appends nothing).
  * out: [B, ldo] of out_dt (SQ_I8 needs requant_mul, a device pointer to one fp32; SQ_F16 / SQ_BF16
- * ignore it).  d must be 128 (else SQ_ERR_UNSUPPORTED), L_max a multiple of 4, ldq a multiple of 16,
- * q / caches 16-byte aligned; max_len beyond what eight CTAs can hold in shared memory
- * (about 300 000 positions) is SQ_ERR_UNSUPPORTED.  workspace: >= 256 bytes; word 0 = device status.
+ * ignore it).  d must be 128 (else SQ_ERR_UNSUPPORTED), L_max a multiple of 4, ldq and ld_new
+ * multiples of 16, q / k_new / v_new / caches 16-byte aligned; max_len beyond what eight CTAs can
+ * hold in shared memory (about 300 000 positions) is SQ_ERR_UNSUPPORTED.  workspace: >= 256 bytes;
+ * word 0 = device status.
  */
-sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, const int8_t* k_cache, const int8_t* v_cache,
+sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, int8_t* k_cache, int8_t* v_cache,
+                                   const int8_t* k_new, const int8_t* v_new, int64_t ld_new,
                                    const int32_t* seq_lens, int64_t B, int64_t H, int64_t d, int64_t L_max,
                                    int64_t max_len, float alpha_qk, float alpha_pv, const float* requant_mul,
                                    void* out, sq_dtype out_dt, int64_t ldo, void* workspace, size_t ws_bytes,

@@ -73,8 +73,8 @@ def lib():
         L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
         L.sq_w8a8_attention.argtypes = [vp, i64, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
         L.sq_kv_cache_write.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, vp, i64, vp, sz, vp]
-        L.sq_w8a8_decode_attention.argtypes = [vp, i64, vp, vp, vp, i64, i64, i64, i64, i64, f32, f32, vp, vp, i32,
-                                               i64, vp, sz, vp]
+        L.sq_w8a8_decode_attention.argtypes = [vp, i64, vp, vp, vp, vp, i64, vp, i64, i64, i64, i64, i64, f32, f32, vp,
+                                               vp, i32, i64, vp, sz, vp]
         for name in EXPORTS[2:]:
             getattr(L, name).restype = i32
         _lib = L
@@ -279,14 +279,19 @@ def sq_kv_cache_write(qkv, B, T, H, d, pos0, k_cache, v_cache, L_max, workspace)
 
 
 def sq_w8a8_decode_attention(q, k_cache, v_cache, seq_lens, B, H, d, L_max, max_len, alpha_qk, alpha_pv, workspace,
-                             requant_mul=None, out=None, out_dtype=None):
+                             requant_mul=None, out=None, out_dtype=None, k_new=None, v_new=None):
     """Attention of each sequence's newest token over the INT8 cache.  q: [B, >= H*d] int8 (row stride
-    taken from the tensor); seq_lens: int32 device tensor [B]; out: [B, H*d] int8 / fp16 / bf16."""
+    taken from the tensor); seq_lens: int32 device tensor [B]; out: [B, H*d] int8 / fp16 / bf16.
+    k_new / v_new: [B, >= H*d] int8 rows of the newest token when it is not in the cache yet (same
+    row stride for both); the kernel then appends them itself."""
+    if k_new is not None and k_new.stride(0) != v_new.stride(0):
+        raise ValueError("k_new and v_new must share one row stride")
     if out is None:
         out = torch.empty((B, H * d), dtype=out_dtype or (torch.int8 if requant_mul is not None else torch.float16),
                           device=q.device)
     wp, wn = _ws(workspace)
-    _check(lib().sq_w8a8_decode_attention(_ptr(q), q.stride(0), _ptr(k_cache), _ptr(v_cache), _ptr(seq_lens), B, H, d,
+    _check(lib().sq_w8a8_decode_attention(_ptr(q), q.stride(0), _ptr(k_cache), _ptr(v_cache), _ptr(k_new), _ptr(v_new),
+                                          k_new.stride(0) if k_new is not None else 0, _ptr(seq_lens), B, H, d,
                                           L_max, max_len, float(alpha_qk), float(alpha_pv), _ptr(requant_mul), _ptr(out),
                                           _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_decode_attention")
     return out

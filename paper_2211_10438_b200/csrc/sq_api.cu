@@ -251,7 +251,8 @@ sq_status sq_kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T,
                           as_stream(stream));
 }
 
-sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, const int8_t* k_cache, const int8_t* v_cache,
+sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, int8_t* k_cache, int8_t* v_cache,
+                                   const int8_t* k_new, const int8_t* v_new, int64_t ld_new,
                                    const int32_t* seq_lens, int64_t B, int64_t H, int64_t d, int64_t L_max,
                                    int64_t max_len, float alpha_qk, float alpha_pv, const float* requant_mul, void* out,
                                    sq_dtype out_dt, int64_t ldo, void* workspace, size_t ws_bytes, void* stream) {
@@ -261,11 +262,13 @@ sq_status sq_w8a8_decode_attention(const int8_t* q, int64_t ldq, const int8_t* k
     if (B == 0 || H == 0) return SQ_OK;
     if (d != 128) return SQ_ERR_UNSUPPORTED;
     if (!q || !k_cache || !v_cache || !seq_lens || !out || (out_dt == SQ_I8 && !requant_mul)) return SQ_ERR_INVALID_ARG;
-    if (max_len > L_max || max_len == 0 || ldq < H * d || ldo < H * d) return SQ_ERR_SHAPE;
+    if ((k_new == nullptr) != (v_new == nullptr)) return SQ_ERR_INVALID_ARG;
+    if (max_len > L_max || max_len == 0 || ldq < H * d || ldo < H * d || (k_new && ld_new < H * d)) return SQ_ERR_SHAPE;
     if (L_max % 4 != 0 || ldq % 16 != 0 || !aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache)) return SQ_ERR_ALIGN;
+    if (k_new && (ld_new % 16 != 0 || !aligned16(k_new) || !aligned16(v_new))) return SQ_ERR_ALIGN;
     if (B > 65535 || H > 65535 || L_max >= ((int64_t)1 << 31)) return SQ_ERR_UNSUPPORTED;
     if (!ws_ok(workspace, ws_bytes, kWsHeader)) return SQ_ERR_WORKSPACE;
-    return kv_decode_attention(q, ldq, k_cache, v_cache, seq_lens, B, H, L_max, max_len, alpha_qk, alpha_pv, requant_mul,
+    return kv_decode_attention(q, ldq, k_cache, v_cache, k_new, v_new, ld_new, seq_lens, B, H, L_max, max_len, alpha_qk, alpha_pv, requant_mul,
                                out, out_dt, ldo, reinterpret_cast<uint32_t*>(workspace), as_stream(stream));
 }
 

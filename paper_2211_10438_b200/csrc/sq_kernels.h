@@ -68,7 +68,8 @@ sq_status attention_i8(const int8_t* qkv, int64_t B, int64_t H, int64_t S, int64
                        const float* requant_mul, int8_t* out, uint32_t* status, cudaStream_t st);
 sq_status kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T, int64_t H, const int32_t* pos0, int8_t* kc,
                          int8_t* vc, int64_t lmax, uint32_t* status, cudaStream_t st);
-sq_status kv_decode_attention(const int8_t* q, int64_t ldq, const int8_t* kc, const int8_t* vc, const int32_t* lens,
+sq_status kv_decode_attention(const int8_t* q, int64_t ldq, int8_t* kc, int8_t* vc, const int8_t* k_new,
+                              const int8_t* v_new, int64_t ld_new, const int32_t* lens,
                               int64_t B, int64_t H, int64_t lmax, int64_t max_len, float alpha_qk, float alpha_pv,
                               const float* requant_mul, void* out, sq_dtype out_dt, int64_t ldo, uint32_t* status,
                               cudaStream_t st);

@@ -92,8 +92,11 @@ __device__ __forceinline__ float ex2_approx(float x) {
 struct KvParams {
     const int8_t* q;        // [B, ldq]; head h at columns h*128 ..
     int64_t ldq;
-    const int8_t* kc;       // [B, H, lmax, 128]
-    const int8_t* vc;       // [B, H, lmax/4, 128, 4]
+    int8_t* kc;             // [B, H, lmax, 128]
+    int8_t* vc;             // [B, H, lmax/4, 128, 4]
+    const int8_t* k_new;    // nullable: [B, ld_new] k / v codes of the newest token, not yet cached;
+    const int8_t* v_new;    // head h at columns h*128 ..
+    int64_t ld_new;
     const int32_t* lens;    // [B]
     int64_t lmax;
     int H;
@@ -166,7 +169,12 @@ kv_decode_attention_kernel(const KvParams p) {
     const int chunk = ((len + C - 1) / C + KV_TILE - 1) / KV_TILE * KV_TILE;
     const int key0 = (int)crank * chunk;
     const int n = max(0, min(len - key0, chunk));
-    const int nt = (n + KV_TILE - 1) / KV_TILE;
+    // With k_new / v_new the newest position (len - 1) is not in the cache yet: the CTA that owns
+    // it takes its key and value from the new rows, stores them for later steps, and streams only
+    // the positions before it.
+    const bool owns_new = p.k_new != nullptr && n > 0 && key0 + n == len;
+    const int nc = owns_new ? n - 1 : n;  // positions of this CTA that come from the cache
+    const int nt = (nc + KV_TILE - 1) / KV_TILE;
     const int ntw = nt > w ? (nt - w + KV_WARPS - 1) / KV_WARPS : 0;  // tiles of this warp, per operand
     const int total = 2 * ntw;                                        // K tiles, then V tiles
     const size_t base = (((size_t)b * p.H + h) * (size_t)p.lmax + (size_t)key0) * KV_D;
@@ -177,7 +185,7 @@ kv_decode_attention_kernel(const KvParams p) {
     auto issue = [&](int u) {  // lane 0: start the copy of this warp's u-th tile
         const bool is_v = u >= ntw;
         const int t = w + KV_WARPS * (is_v ? u - ntw : u);
-        const int rows = min(KV_TILE, n - KV_TILE * t);
+        const int rows = min(KV_TILE, nc - KV_TILE * t);
         const uint32_t bytes = is_v ? (uint32_t)((rows + 3) / 4) * 4u * KV_D : (uint32_t)rows * KV_D;
         const int8_t* src = (is_v ? p.vc : p.kc) + base + (size_t)t * KV_TILE_BYTES;
         const int slot = u % KV_STAGES;
@@ -201,7 +209,7 @@ kv_decode_attention_kernel(const KvParams p) {
     for (int u = 0; u < ntw; ++u) {
         if (!(ok = wait_tile(u))) break;
         const int t = w + KV_WARPS * u;
-        const int rows = min(KV_TILE, n - KV_TILE * t);
+        const int rows = min(KV_TILE, nc - KV_TILE * t);
         const uint8_t* row = my_ring + (size_t)(u % KV_STAGES) * KV_TILE_BYTES + lane * KV_D;
         int acc = 0;
 #pragma unroll
@@ -220,6 +228,23 @@ kv_decode_attention_kernel(const KvParams p) {
         }
         __syncwarp();
         if (lane == 0 && u + KV_STAGES < total) issue(u + KV_STAGES);
+    }
+    const size_t new_off = (size_t)b * p.ld_new + (size_t)h * KV_D;
+    if (owns_new && w == 0) {  // score of the newest position from its own key row
+        int acc = 0;
+        if (lane < KV_D / 16) {
+            const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k_new + new_off) + lane);
+            const uint4 qv = *reinterpret_cast<const uint4*>(q_s + lane * 16);
+            acc = __dp4a((int)kv.x, (int)qv.x, acc);
+            acc = __dp4a((int)kv.y, (int)qv.y, acc);
+            acc = __dp4a((int)kv.z, (int)qv.z, acc);
+            acc = __dp4a((int)kv.w, (int)qv.w, acc);
+            // and the key row goes into the cache for the steps to come
+            *reinterpret_cast<uint4*>(p.kc + ((((size_t)b * p.H + h) * (size_t)p.lmax + (size_t)(len - 1)) * KV_D) + lane * 16) = kv;
+        }
+        acc = __reduce_add_sync(0xffffffffu, acc);
+        if (lane == 0) scores[nc] = acc;
+        vmax = max(vmax, acc);
     }
     vmax = __reduce_max_sync(0xffffffffu, vmax);
     if (lane == 0) wred[w] = (uint32_t)vmax;
@@ -254,15 +279,16 @@ kv_decode_attention_kernel(const KvParams p) {
     float l = 0.0f;
     for (int r = 0; r < C; ++r) l += __uint_as_float(ld_cluster_u32(x_sum, (uint32_t)r));  // rank order
     const float k127 = __fdiv_rn(127.0f, l);  // P = round(127 * e / l)
-    for (int g = tid; g < nt * (KV_TILE / 4); g += KV_THREADS) {  // four positions per word; zero beyond n
+    for (int g = tid; g < nt * (KV_TILE / 4); g += KV_THREADS) {  // four positions per word; zero beyond nc
         uint32_t c[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int j = 4 * g + e;
-            c[e] = j < n ? quant_code<false>(ex[j], k127) : 0u;  // e <= l: the code cannot exceed 127
+            c[e] = j < nc ? quant_code<false>(ex[j], k127) : 0u;  // e <= l: the code cannot exceed 127
         }
         pbar[g] = pack4(c[0], c[1], c[2], c[3]);
     }
+    const int p_new = owns_new ? (int)(quant_code<false>(ex[nc], k127) & 0xffu) : 0;
     __syncthreads();
 
     // ---- phase 2: partial outputs; lane owns channels 4*lane .. 4*lane+3 ----
@@ -270,7 +296,7 @@ kv_decode_attention_kernel(const KvParams p) {
     for (int u = ntw; ok && u < total; ++u) {
         if (!(ok = wait_tile(u))) break;
         const int t = w + KV_WARPS * (u - ntw);
-        const int ng = (min(KV_TILE, n - KV_TILE * t) + 3) / 4;
+        const int ng = (min(KV_TILE, nc - KV_TILE * t) + 3) / 4;
         const uint8_t* tile = my_ring + (size_t)(u % KV_STAGES) * KV_TILE_BYTES + lane * 16;
         const uint32_t* pw = pbar + t * (KV_TILE / 4);
 #pragma unroll 4
@@ -284,6 +310,17 @@ kv_decode_attention_kernel(const KvParams p) {
         }
         __syncwarp();
         if (lane == 0 && u + KV_STAGES < total) issue(u + KV_STAGES);
+    }
+    if (owns_new) {
+        const int pos = len - 1;
+        if (w == 0) {  // the newest position's share of the output, from its own value row
+            const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.v_new + new_off) + lane);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) o[k] += p_new * (int)(int8_t)((vw >> (8 * k)) & 0xffu);
+        }
+        // value row -> cache: channel tid, byte (pos % 4) of its 4-position word
+        p.vc[(((size_t)b * p.H + h) * (size_t)p.lmax + (size_t)(pos & ~3)) * KV_D + (size_t)tid * 4 + (pos & 3)] =
+            __ldg(p.v_new + new_off + tid);
     }
     *reinterpret_cast<int4*>(wpart + w * KV_D + 4 * lane) = make_int4(o[0], o[1], o[2], o[3]);
     __syncthreads();
@@ -379,12 +416,14 @@ int kv_choose_cluster(int64_t B, int64_t H, int64_t max_len) {
     return c;
 }
 
-sq_status kv_decode_attention(const int8_t* q, int64_t ldq, const int8_t* kc, const int8_t* vc, const int32_t* lens,
+sq_status kv_decode_attention(const int8_t* q, int64_t ldq, int8_t* kc, int8_t* vc, const int8_t* k_new,
+                              const int8_t* v_new, int64_t ld_new, const int32_t* lens,
                               int64_t B, int64_t H, int64_t lmax, int64_t max_len, float alpha_qk, float alpha_pv,
                               const float* requant_mul, void* out, sq_dtype out_dt, int64_t ldo, uint32_t* status,
                               cudaStream_t st) {
     KvParams p;
     p.q = q; p.ldq = ldq; p.kc = kc; p.vc = vc; p.lens = lens; p.lmax = lmax;
+    p.k_new = k_new; p.v_new = v_new; p.ld_new = ld_new;
     p.H = (int)H; p.max_len = (int)max_len;
     p.cluster = kv_choose_cluster(B, H, max_len);
     p.cap = (int)(((max_len + p.cluster - 1) / p.cluster + KV_TILE - 1) / KV_TILE * KV_TILE);

@@ -243,8 +243,8 @@ class DecoderBlockStatic:
 
 class DecoderBlockDecode:
     """Generation stage of DecoderBlockStatic: one new token per sequence against an INT8 KV cache,
-    as ten libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> append k, v to the cache ->
-    attention of the new token over the cache (INT8 out) -> out-proj GEMM -> residual ->
+    as nine libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> attention of the new token over
+    the cache, which also appends its k, v (INT8 out) -> out-proj GEMM -> residual ->
     LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM -> residual.  Same `lin` / `steps` as the
     prompt block.  `ctx` (int32 device tensor [B]) counts the positions each sequence has cached."""
 
@@ -276,7 +276,7 @@ class DecoderBlockDecode:
                                       max(l.Wq.shape[1] for l in lin.values())),
                    sq.workspace_bytes(sq.SQ_OP_LN_QUANT, B, 0, hid))
         self.ws = sq.new_workspace(need, dev)
-        self.launches_per_step = 10
+        self.launches_per_step = 9
 
     def load_prompt(self, qkv_codes, S):
         """Fill the cache from a prompt pass's QKV code buffer [B*S, 3*H*d]; every sequence then holds S positions."""
@@ -293,9 +293,10 @@ class DecoderBlockDecode:
                        x_scale=s["d_ln1"], workspace=self.ws)
         sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
                         requant_mul=self.r_qkv, out=self.qkv)
-        sq.sq_kv_cache_write(self.qkv, B, 1, H, d, self.ctx, self.k_cache, self.v_cache, self.L_max, self.ws)
+        hid = self.hid  # the attention kernel takes the new k, v rows from the QKV buffer and caches them
         sq.sq_w8a8_decode_attention(self.qkv, self.k_cache, self.v_cache, self.lens, B, H, d, self.L_max, max_len,
-                                    self.alpha_qk, self.alpha_pv, self.ws, requant_mul=self.r_attn, out=self.attn)
+                                    self.alpha_qk, self.alpha_pv, self.ws, requant_mul=self.r_attn, out=self.attn,
+                                    k_new=self.qkv[:, hid:], v_new=self.qkv[:, 2 * hid:])
         sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
                         bias=L["out_proj"].bias, out=self.proj)
         sq.sq_residual_add(x, self.proj, out=self.h)

@@ -213,3 +213,50 @@ def test_decode_attention_continues_the_prompt_kernel():
     last = out_prompt.view(B, S, H * D)[:, -1].int()
     d = (last - out_dec.int()).abs()
     assert int(d.max()) <= 2 and float((d != 0).float().mean()) <= 2e-2
+
+
+@pytest.mark.parametrize("B,H,lens,L_max", [(2, 3, [37, 5], 64), (3, 1, [1, 2, 4], 8), (1, 2, [2048], 2048),
+                                            (1, 3, [1997], 2048), (2, 2, [700, 33], 1024), (4, 40, [513, 512, 100, 261], 640)])
+def test_decode_attention_appends_the_newest_token_itself(B, H, lens, L_max):
+    """With k_new / v_new the newest position is NOT in the cache: it holds junk there.  The kernel
+    must give the result of the pre-appended path and leave the cache as a separate append would."""
+    L = max(lens)
+    q = synth.int8_tensor(68, L, (B, H, D), lo=-100, hi=100)
+    K = synth.int8_tensor(68, L + 1, (B, H, L, D), lo=-100, hi=100)
+    V = synth.int8_tensor(68, L + 2, (B, H, L, D), lo=-100, hi=100)
+    alpha_qk, alpha_pv = np.float32(0.0009), np.float32(0.01 / 127)
+    r = np.array([1.0 / 0.0008], np.float32)
+    want, _ = oracle.kv_decode_attention(q, K, V, lens, alpha_qk, alpha_pv, requant_mul=r)
+    # the newest token's rows, laid out like a QKV code buffer [B, 3*H*d]; junk at its cache position
+    qkv = np.zeros((B, 3, H, D), np.int8)
+    Kj, Vj = K.copy(), V.copy()
+    for b in range(B):
+        qkv[b, 0], qkv[b, 1], qkv[b, 2] = q[b], K[b, :, lens[b] - 1], V[b, :, lens[b] - 1]
+        Kj[b, :, lens[b] - 1] = 113
+        Vj[b, :, lens[b] - 1] = -113
+    kc_np, vc_np = _cache_layout(Kj, Vj, L_max)
+    kc, vc = dev(kc_np), dev(vc_np)
+    qd = dev(qkv.reshape(B, 3 * H * D))
+    ws = sq.new_workspace(256)
+    hid = H * D
+    out = sq.sq_w8a8_decode_attention(qd, kc, vc, dev(np.asarray(lens, np.int32)), B, H, D, L_max, L, alpha_qk, alpha_pv, ws,
+                                      requant_mul=dev(r), k_new=qd[:, hid:], v_new=qd[:, 2 * hid:])
+    torch.cuda.synchronize()
+    assert sq.device_status(ws) == 0
+    diff = np.abs(host(out).reshape(B, H, D).astype(np.int32) - want.astype(np.int32))
+    assert diff.max() <= 2 and (diff != 0).mean() <= 1e-2
+    # and byte for byte what the pre-appended path gives on the true cache
+    kt, vt = _cache_layout(K, V, L_max)
+    ref = sq.sq_w8a8_decode_attention(qd, dev(kt), dev(vt), dev(np.asarray(lens, np.int32)), B, H, D, L_max, L, alpha_qk,
+                                      alpha_pv, ws, requant_mul=dev(r))
+    assert torch.equal(out, ref)
+    # the cache now holds the true rows at the newest positions, everything else untouched
+    want_k, want_v = _cache_layout(K, V, L_max)
+    got_k, got_v = host(kc), host(vc)
+    for b in range(B):
+        n = lens[b]
+        assert np.array_equal(got_k[b, :, :n], want_k[b, :, :n])
+        g = (n + 3) // 4
+        logical = got_v[b].transpose(0, 1, 3, 2).reshape(H, L_max, D)   # [H, L_max/4, 4, d] -> positions
+        assert np.array_equal(logical[:, :n], V[b, :, :n])
+        assert np.array_equal(got_k[b, :, n:], kc_np[b, :, n:]) and g >= 1
