@@ -20,6 +20,7 @@
 #include <climits>
 
 #include "sq_common.cuh"
+#include "sq_bulk.cuh"
 #include "sq_kernels.h"
 
 namespace sq {
@@ -33,39 +34,9 @@ constexpr int KV_WARPS = 4;
 constexpr int KV_THREADS = KV_WARPS * 32;
 constexpr int KV_STAGES = 4;                 // ring stages per warp
 constexpr int KV_MAX_CLUSTER = 8;
-constexpr uint32_t kWaitCycles = 2000000000u;
 constexpr float kLog2e = 1.4426950408889634f;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity))
-        if ((++spins & 63u) == 0u && (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) return false;
-    return true;
-}
-// contiguous global -> shared copy; both addresses 16-byte aligned, bytes a multiple of 16
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
+using namespace bulk;
 __device__ __forceinline__ uint32_t cluster_rank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -432,13 +403,12 @@ sq_status kv_decode_attention(const int8_t* q, int64_t ldq, int8_t* kc, int8_t* 
     p.requant_mul = requant_mul; p.out = out; p.out_dt = (int)out_dt; p.ldo = ldo; p.status = status;
     const size_t smem = kv_smem_bytes(p.cap);
     if (smem > 227 * 1024) return SQ_ERR_UNSUPPORTED;
-    static bool attr_set = false;  // per process; the value is the same for every call
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kv_decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess) {
-            cudaGetLastError();
-            return SQ_ERR_CUDA;
-        }
-        attr_set = true;
+    static bool attr_set[64] = {false};  // per device
+    int dev = 0;
+    SQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        SQ_CUDA_OK(cudaFuncSetAttribute(kv_decode_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     return launch_pdl(kv_decode_attention_kernel, dim3((unsigned)p.cluster, (unsigned)H, (unsigned)B), dim3(KV_THREADS), smem, st,
                       p.cluster, p);

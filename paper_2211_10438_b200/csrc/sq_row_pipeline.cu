@@ -17,6 +17,7 @@
 // The kernel is instruction-issue sensitive (about 11 instructions per element at 3 bytes of
 // HBM traffic per element), hence the single-FMA rounding and byte-permute packing.
 #include "sq_common.cuh"
+#include "sq_bulk.cuh"
 #include "sq_kernels.h"
 
 namespace sq {
@@ -24,38 +25,8 @@ namespace sq {
 namespace {
 
 constexpr int CTA_THREADS = 512;
-constexpr uint32_t kWaitCycles = 2000000000u;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    uint32_t spins = 0;
-    while (!mbar_try_wait(bar, parity))
-        if ((++spins & 63u) == 0u && (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) return false;
-    return true;
-}
-// one row: global -> shared, completion counted in bytes on `bar` (addresses 16-byte aligned)
-__device__ __forceinline__ void bulk_load_row(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
+using namespace bulk;
 template <int GROUP>
 __device__ __forceinline__ void group_sync(int g) {
     if (GROUP == CTA_THREADS) __syncthreads();
@@ -116,7 +87,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
             const int64_t r = first + (int64_t)s * stride;
             if (r < M) {
                 mbar_expect_tx(my_full + s, (uint32_t)row_bytes);
-                bulk_load_row(my_rows + (size_t)s * row_bytes, X + r * C, (uint32_t)row_bytes, my_full + s);
+                bulk_load(my_rows + (size_t)s * row_bytes, X + r * C, (uint32_t)row_bytes, my_full + s);
             }
         }
     }
@@ -165,7 +136,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 const int64_t nxt = row + (int64_t)stages * stride;
                 if (nxt < M) {
                     mbar_expect_tx(my_full + s, (uint32_t)row_bytes);
-                    bulk_load_row(my_rows + (size_t)s * row_bytes, X + nxt * C, (uint32_t)row_bytes, my_full + s);
+                    bulk_load(my_rows + (size_t)s * row_bytes, X + nxt * C, (uint32_t)row_bytes, my_full + s);
                 }
             }
             refilled = true;
