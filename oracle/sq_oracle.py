@@ -93,6 +93,23 @@ def row_absmax(X):
     return m
 
 
+def clip_count(T: int, clip_frac: float) -> int:
+    """Number of tokens a clipping fraction sets aside: clip_frac * T rounded to the nearest integer."""
+    return int(np.floor(float(clip_frac) * T + 0.5))
+
+
+def clipped_absmax(token_absmax, n_clip: int):
+    """Calibration of a static step with the largest tokens set aside (Section 5.2: for GLM-130B
+    the top 2 % of tokens are clipped when the static step sizes are calibrated).  Of the T
+    per-token absolute maxima (row_absmax over every calibration token), the n_clip largest are
+    dropped and the largest of the rest is returned; the static step is step_size() of it.
+    n_clip = 0 is the plain maximum; at least one token is always kept."""
+    a = np.sort(np.ascontiguousarray(token_absmax, np.float32).reshape(-1))  # library sort, ascending
+    T = a.size
+    k = max(0, min(int(n_clip), T - 1))
+    return np.float32(a[T - 1 - k])
+
+
 def smooth_scales(act_absmax, w_absmax, alpha: float):
     """Eq. 4: s_j = max|X_j|^alpha / max|W_j|^(1-alpha)."""
     if not (0.0 <= alpha <= 1.0):

@@ -471,3 +471,31 @@ def test_decode_block_continues_the_prompt_block_exactly():
         assert np.array_equal(dec[key], want), key
     assert np.array_equal(Kc[:, :, S - 1], qkv[:, S - 1, 1]) and np.array_equal(Vc[:, :, S - 1], qkv[:, S - 1, 2])
     assert np.abs(prompt["attn"]).max() > 10 and np.abs(prompt["y"]).max() > 0.5  # not a vacuous comparison
+
+
+# --------------------------------------------------------------------------- #
+# Static-step calibration with the largest tokens clipped
+# --------------------------------------------------------------------------- #
+def test_clipped_absmax_pins():
+    rng = np.random.default_rng(47)
+    v = np.arange(1, 101, dtype=np.float32)
+    rng.shuffle(v)
+    assert oracle.clip_count(100, 0.02) == 2 and oracle.clip_count(100, np.float32(0.02)) == 2
+    assert oracle.clip_count(65536, 0.02) == 1311 and oracle.clip_count(7, 0.0) == 0
+    assert oracle.clipped_absmax(v, 0) == 100.0                   # nothing clipped: the plain maximum
+    assert oracle.clipped_absmax(v, 2) == 98.0                    # the two largest of 100 tokens set aside
+    assert oracle.clipped_absmax(v, 50) == 50.0
+    assert oracle.clipped_absmax(v, 100) == 1.0 and oracle.clipped_absmax(v, 1000) == 1.0   # never empties the set
+    assert oracle.clipped_absmax(np.array([5, 5, 5, 1], np.float32), 1) == 5.0              # ties
+    x = np.abs(rng.standard_normal(4099)).astype(np.float32) * 7
+    for k in (0, 4, 82, 1230):
+        want = np.partition(x, x.size - 1 - k)[x.size - 1 - k]    # library selection
+        assert oracle.clipped_absmax(x, k) == want
+        assert oracle.clipped_absmax(rng.permutation(x), k) == want
+        assert (x > want).sum() <= k                               # at most k tokens lie above the result
+    # on the outlier-token model, clipping the few huge tokens shrinks the static step a lot
+    X = rng.standard_normal((1000, 64)).astype(np.float32)
+    X[::100] *= 50.0                                               # 1 % of the tokens are outliers
+    ta = oracle.row_absmax(X)
+    assert oracle.clipped_absmax(ta, oracle.clip_count(1000, 0.02)) < 0.1 * oracle.clipped_absmax(ta, 0)
+    assert oracle.clipped_absmax(ta, 0) == oracle.calib_absmax(X).max()
