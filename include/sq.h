@@ -98,6 +98,23 @@ sq_status sq_calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols
                           float* absmax_inout, void* stream);
 
 /*
+ * Calibration of a per-tensor STATIC step with the largest tokens set aside (Section 5.2: for
+ * GLM-130B the top 2 % of tokens are clipped when the static step sizes are calibrated).
+ * sq_token_absmax: token_absmax[t] = max_j |X[t, j]| for the M tokens of one calibration batch
+ * (X: [M, C] of dtype dt, row stride ld elements; C and ld multiples of 8, X 16-byte aligned);
+ * the caller lays the batches' results side by side in one [T] array.
+ * sq_clipped_absmax: of those T values the n_clip largest are dropped (at least one value is
+ * always kept) and the largest of the rest is written to absmax_out[0]; step_out (nullable)
+ * receives the step size max(absmax, 1e-5) / 127 of Eq. 1.  n_clip = 0 gives the plain maximum.
+ * The selection is exact (radix selection on the bit patterns; values must be >= 0, which
+ * sq_token_absmax guarantees).  T < 2^32.
+ */
+sq_status sq_token_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, int64_t ld, float* token_absmax,
+                          void* stream);
+sq_status sq_clipped_absmax(const float* token_absmax, int64_t T, int64_t n_clip, float* absmax_out,
+                            float* step_out, void* stream);
+
+/*
  * Smoothing factor, Eq. 4:  s_j = max|X_j|^alpha / max|W_j|^(1-alpha),  j < C.
  * act_absmax, w_absmax: [C] fp32 (both floored at 1e-5 so that s_j is finite and
  * non-zero); alpha in [0, 1] else SQ_ERR_INVALID_ARG; s_out: [C] fp32.  The powers are

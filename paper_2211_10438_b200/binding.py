@@ -27,7 +27,8 @@ SQ_NOALLOC_MAX_ROWS = 16384
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
-           "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention"]
+           "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention",
+           "sq_token_absmax", "sq_clipped_absmax"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -72,6 +73,8 @@ def lib():
         L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
         L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
         L.sq_w8a8_attention.argtypes = [vp, i64, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
+        L.sq_token_absmax.argtypes = [vp, i32, i64, i64, i64, vp, vp]
+        L.sq_clipped_absmax.argtypes = [vp, i64, i64, vp, vp, vp]
         L.sq_kv_cache_write.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, vp, i64, vp, sz, vp]
         L.sq_w8a8_decode_attention.argtypes = [vp, i64, vp, vp, vp, vp, i64, vp, i64, i64, i64, i64, i64, f32, f32, vp,
                                                vp, i32, i64, vp, sz, vp]
@@ -295,3 +298,21 @@ def sq_w8a8_decode_attention(q, k_cache, v_cache, seq_lens, B, H, d, L_max, max_
                                           L_max, max_len, float(alpha_qk), float(alpha_pv), _ptr(requant_mul), _ptr(out),
                                           _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_decode_attention")
     return out
+
+
+def sq_token_absmax(X, out=None):
+    """Per-token absolute maximum of a calibration batch [M, C] -> fp32 [M]."""
+    M, C = X.shape
+    if out is None:
+        out = torch.empty(M, dtype=torch.float32, device=X.device)
+    _check(lib().sq_token_absmax(_ptr(X), _DT[X.dtype], M, C, X.stride(0), _ptr(out), _stream()), "sq_token_absmax")
+    return out
+
+
+def sq_clipped_absmax(token_absmax, n_clip):
+    """Largest of the per-token maxima after the n_clip largest have been set aside -> (absmax[1], step[1])."""
+    a = torch.empty(1, dtype=torch.float32, device=token_absmax.device)
+    s = torch.empty(1, dtype=torch.float32, device=token_absmax.device)
+    _check(lib().sq_clipped_absmax(_ptr(token_absmax), token_absmax.numel(), int(n_clip), _ptr(a), _ptr(s), _stream()),
+           "sq_clipped_absmax")
+    return a, s

@@ -81,6 +81,26 @@ sq_status sq_calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols
     return calib_absmax(X, dt, rows, cols, ld, absmax_inout, as_stream(stream));
 }
 
+sq_status sq_token_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, int64_t ld, float* out,
+                          void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (M < 0 || C < 0 || ld < C) return SQ_ERR_SHAPE;
+    if (M == 0) return SQ_OK;
+    if (!X || !out) return SQ_ERR_INVALID_ARG;
+    if (C % 8 != 0 || ld % 8 != 0 || !aligned16(X)) return SQ_ERR_ALIGN;
+    if (M >= ((int64_t)1 << 34)) return SQ_ERR_UNSUPPORTED;
+    return token_absmax(X, dt, M, C, ld, out, as_stream(stream));
+}
+
+sq_status sq_clipped_absmax(const float* vals, int64_t T, int64_t n_clip, float* absmax_out,
+                            float* step_out, void* stream) {
+    if (T < 0 || n_clip < 0) return SQ_ERR_SHAPE;
+    if (T == 0) return SQ_ERR_SHAPE;  // no token to take a maximum of
+    if (!vals || !absmax_out) return SQ_ERR_INVALID_ARG;
+    if (T >= ((int64_t)1 << 32)) return SQ_ERR_UNSUPPORTED;
+    return clipped_absmax(vals, T, n_clip, absmax_out, step_out, as_stream(stream));
+}
+
 sq_status sq_smooth_scales(const float* act_absmax, const float* w_absmax, int64_t C, float alpha,
                            float* s_out, float* s_inv_out, void* stream) {
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return SQ_ERR_INVALID_ARG;

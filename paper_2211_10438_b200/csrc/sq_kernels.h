@@ -25,6 +25,9 @@ constexpr size_t kDecCounterBytes = 32768;  // decode-shaped GEMM: one arrival c
 
 sq_status calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld, float* a,
                        cudaStream_t st);
+sq_status token_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, int64_t ld, float* out, cudaStream_t st);
+sq_status clipped_absmax(const float* token_absmax, int64_t T, int64_t n_clip, float* absmax_out, float* step_out,
+                         cudaStream_t st);
 sq_status smooth_scales(const float* ax, const float* aw, int64_t C, float alpha, float* s, float* s_inv,
                         cudaStream_t st);
 sq_status fold_ln_weight(const void* g, const void* b, sq_dtype dt, const float* s, int64_t C,

@@ -115,6 +115,88 @@ sq_status calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, i
 }
 
 // =======================================================================================
+// Static-step calibration with the largest tokens set aside (Section 5.2: the top 2 % of tokens
+// are clipped when the static step sizes are calibrated for GLM-130B): per-token |max| of every
+// calibration token, then the exact (n_clip + 1)-th largest of them.
+// =======================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+token_absmax_kernel(const T* __restrict__ X, int64_t M, int64_t C, int64_t ld, float* __restrict__ out) {
+    // one warp per token; packed |x| / max on 16-bit pairs is exact
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= M) return;
+    const uint4* src = reinterpret_cast<const uint4*>(X + row * ld);
+    const int64_t nvec = C / 8;
+    uint4 m = make_uint4(0u, 0u, 0u, 0u);
+    for (int64_t v = lane; v < nvec; v += 32) {
+        const uint4 x = __ldcs(src + v);
+        m.x = Act<T>::absmax2(m.x, x.x); m.y = Act<T>::absmax2(m.y, x.y);
+        m.z = Act<T>::absmax2(m.z, x.z); m.w = Act<T>::absmax2(m.w, x.w);
+    }
+    float f[8];
+    unpack8<T>(m, f);
+    float r = fmaxf(fmaxf(fmaxf(f[0], f[1]), fmaxf(f[2], f[3])), fmaxf(fmaxf(f[4], f[5]), fmaxf(f[6], f[7])));
+    r = warp_max(r);
+    if (lane == 0) out[row] = r;
+}
+
+// Exact selection among T non-negative floats: their bit patterns order like the values, so four
+// passes of an 8-bit histogram (most significant byte first) pin the pattern of the element of
+// descending rank k.  One CTA; T is a calibration set's token count (10^4 .. 10^7).
+__global__ void __launch_bounds__(1024)
+select_rank_kernel(const float* __restrict__ vals, int64_t T, int64_t k, float* __restrict__ absmax_out,
+                   float* __restrict__ step_out) {
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t s_prefix, s_k;
+    const uint32_t* u = reinterpret_cast<const uint32_t*>(vals);
+    if (threadIdx.x == 0) { s_prefix = 0u; s_k = (uint32_t)k; }
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const uint32_t mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+        if (threadIdx.x < 256) hist[threadIdx.x] = 0u;
+        __syncthreads();
+        const uint32_t prefix = s_prefix;
+        for (int64_t i = threadIdx.x; i < T; i += blockDim.x) {
+            const uint32_t x = u[i];
+            if ((x & mask) == prefix) atomicAdd(&hist[(x >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t kk = s_k, bin = 255u;
+            for (;; --bin) {  // from the largest byte down; the counts of this pass sum to more than kk
+                if (hist[bin] > kk || bin == 0u) break;
+                kk -= hist[bin];
+            }
+            s_k = kk;
+            s_prefix = prefix | (bin << shift);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const float a = __uint_as_float(s_prefix);
+        absmax_out[0] = a;
+        if (step_out) step_out[0] = step_size(a);
+    }
+}
+
+sq_status token_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, int64_t ld, float* out, cudaStream_t st) {
+    const unsigned grid = (unsigned)((M + 7) / 8);
+    if (dt == SQ_F16)
+        token_absmax_kernel<__half><<<grid, 256, 0, st>>>(static_cast<const __half*>(X), M, C, ld, out);
+    else
+        token_absmax_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(X), M, C, ld, out);
+    return launch_status();
+}
+
+sq_status clipped_absmax(const float* token_absmax, int64_t T, int64_t n_clip, float* absmax_out, float* step_out,
+                         cudaStream_t st) {
+    const int64_t k = std::max<int64_t>(0, std::min<int64_t>(n_clip, T - 1));  // at least one token is kept
+    select_rank_kernel<<<1, 1024, 0, st>>>(token_absmax, T, k, absmax_out, step_out);
+    return launch_status();
+}
+
+// =======================================================================================
 // Eq. 4 and the LayerNorm fold of Eq. 3 (tiny, offline)
 // =======================================================================================
 __global__ void smooth_scales_kernel(const float* __restrict__ ax, const float* __restrict__ aw,

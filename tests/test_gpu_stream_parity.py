@@ -214,3 +214,51 @@ def test_residual_add(dtype):
     b = synth.to_dtype_f32(rng.standard_normal(4096 * 3).astype(np.float32), dtype)
     out = sq.sq_residual_add(dev(a, dtype), dev(b, dtype))
     assert np.array_equal(host(out), oracle.round_to(a + b, dtype))
+
+
+# --------------------------------------------------------------------------- #
+# Static-step calibration with the largest tokens set aside (Section 5.2)
+# --------------------------------------------------------------------------- #
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M,C", [(1, 8), (37, 520), (512, 7168), (4099, 64)])
+def test_token_absmax_exact(dtype, M, C):
+    ch = synth.outlier_channels(7, C, count=max(1, C // 100))
+    x = synth.activations(7, M, M, C, dtype, ch, synth.outlier_factors(7, len(ch), 20.0, 80.0))
+    got = sq.sq_token_absmax(dev(x, dtype))
+    assert np.array_equal(host(got), oracle.row_absmax(x))
+
+
+@pytest.mark.parametrize("T,n_clip", [(1, 0), (1, 5), (100, 2), (4099, 0), (4099, 82), (65536, 1311), (65536, 65535),
+                                      (300000, 6000)])
+def test_clipped_absmax_exact(T, n_clip):
+    rng = synth.rng_for(7, T + n_clip)
+    v = np.abs(rng.standard_normal(T)).astype(np.float32) * 9
+    v[rng.integers(0, T, max(1, T // 50))] *= 40.0       # a few huge tokens
+    if T > 10:
+        v[3], v[7] = v[5], v[5]                           # ties
+        v[1] = 0.0
+    a, s = sq.sq_clipped_absmax(dev(v), n_clip)
+    want = oracle.clipped_absmax(v, n_clip)
+    assert host(a)[0] == want
+    assert host(s)[0] == oracle.step_size(float(want))
+
+
+def test_clipped_static_step_end_to_end():
+    """Four calibration batches -> per-token maxima side by side -> the top 2 % set aside -> static step;
+    quantising with that step saturates exactly the tokens that were set aside (and no others)."""
+    C, Mb = 512, 256
+    batches = [synth.activations(7, 50 + i, Mb, C, "f16", [5], [1.0]) for i in range(4)]
+    for b in batches:
+        b[::64] *= 30.0                                    # 1.6 % of the tokens are huge
+    ta = torch.empty(4 * Mb, dtype=torch.float32, device="cuda")
+    for i, b in enumerate(batches):
+        sq.sq_token_absmax(dev(b, "f16"), out=ta[i * Mb:(i + 1) * Mb])
+    n_clip = oracle.clip_count(4 * Mb, 0.02)
+    a, step = sq.sq_clipped_absmax(ta, n_clip)
+    allx = np.concatenate(batches)
+    want = oracle.clipped_absmax(oracle.row_absmax(allx), n_clip)
+    assert host(a)[0] == want
+    q, _ = oracle.quant_act(allx, "per_tensor_static", static_scale=float(host(step)[0]))
+    saturated_rows = (np.abs(q) == 127).any(1) & (oracle.row_absmax(allx) > want)
+    assert saturated_rows.sum() == (oracle.row_absmax(allx) > want).sum() <= n_clip
+    assert want < 0.2 * oracle.row_absmax(allx).max()
