@@ -64,7 +64,7 @@ size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K) {
     switch (op) {
         case SQ_OP_LN_QUANT: return kWsHeader + (size_t)(M > 0 ? M : 0) * 2 * sizeof(float);
         case SQ_OP_GEMM:  // decode-shaped calls keep split-K partial sums in the workspace
-            return (M > 0 && M <= 16 && N > 0) ? decode_workspace_bytes(M, N) : kWsHeader;
+            return (M > 0 && M <= 64 && N > 0) ? decode_workspace_bytes(M, N) : kWsHeader;
         case SQ_OP_QUANT_ACT:
         case SQ_OP_QUANT_WEIGHT:
         case SQ_OP_BMM: return kWsHeader;

@@ -23,13 +23,18 @@ namespace {
 using namespace tc;
 
 constexpr int DEC_THREADS = 192;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
-constexpr int DEC_N = 16;             // tokens per MMA (N dimension)
+constexpr int DEC_MAX_N = 64;         // most tokens this kernel takes
 constexpr int W_BYTES = BLOCK_M * BLOCK_K;  // 16 KB of weights per stage
-constexpr int X_BYTES = DEC_N * BLOCK_K;    // 2 KB of activations per stage
-constexpr int DEC_STAGE = W_BYTES + X_BYTES;
-constexpr int DEC_STAGES = 10;
-constexpr int DEC_TMEM_COLS = 32;     // two accumulator slots of 16 columns
-constexpr int DEC_SMEM = 1024 + DEC_STAGES * DEC_STAGE + (2 * DEC_STAGES + 4) * 8 + 64;
+// DN = tokens per MMA (its N dimension): 16, 32 or 64.  A stage holds 16 KB of weights and
+// DN * 128 bytes of activations; the ring is as deep as shared memory allows (10 / 10 / 9 stages).
+template <int DN>
+struct DecCfg {
+    static constexpr int X_BYTES = DN * BLOCK_K;
+    static constexpr int STAGE = W_BYTES + X_BYTES;
+    static constexpr int STAGES = DN <= 32 ? 10 : 9;
+    static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
+    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 4) * 8 + 64;
+};
 
 struct DecParams {
     int M;
@@ -61,12 +66,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 __device__ __forceinline__ void dec_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
 // Eq. 2 for one output channel (this thread) and all tokens, then the stores.
-__device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&acc)[16], int64_t col) {
+template <int DN>
+__device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&acc)[DN], int64_t col) {
     if (col >= p.N) return;
     if (p.out_dt == SQ_I32) {
         int32_t* y = static_cast<int32_t*>(p.Y);
 #pragma unroll
-        for (int t = 0; t < DEC_N; ++t)
+        for (int t = 0; t < DN; ++t)
             if (t < p.M) y[(int64_t)t * p.ldy + col] = acc[t];
         return;
     }
@@ -77,7 +83,7 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
                             : __half2float(static_cast<const __half*>(p.bias)[col]);
     const float rq = p.requant_mul ? __ldg(p.requant_mul + (p.requant_per_col ? col : 0)) : 1.0f;
 #pragma unroll
-    for (int t = 0; t < DEC_N; ++t) {
+    for (int t = 0; t < DN; ++t) {
         if (t < p.M) {
             const float xs = __ldg(p.x_scale + (p.x_per_row ? t : 0));
             float v = __fmaf_rn(__int2float_rn(acc[t]), __fmul_rn(xs, ws), bs);
@@ -92,9 +98,12 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
     }
 }
 
+template <int DN>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                    const DecParams p) {
+    constexpr int DEC_N = DN, DEC_STAGE = DecCfg<DN>::STAGE, DEC_STAGES = DecCfg<DN>::STAGES;
+    constexpr int DEC_TMEM_COLS = DecCfg<DN>::TMEM_COLS;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + DEC_STAGES * DEC_STAGE);
@@ -229,20 +238,23 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             dec_epi_sync();
             if (*epi_go == 0u) break;
             tcgen05_fence_after();
-            uint32_t r[16];
-            tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(slot * DEC_N), r);
-            tmem_ld_wait();
+            int32_t acc[DEC_N];
+#pragma unroll
+            for (int c0 = 0; c0 < DEC_N; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(slot * DEC_N + c0), r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int t = 0; t < 16; ++t) acc[c0 + t] = (int32_t)r[t];
+            }
             tcgen05_fence_before();
             mbar_arrive(tmem_empty + slot);  // slot drained into registers
             slot ^= 1;
             if (slot == 0) slot_phase ^= 1u;
 
             const int64_t col = (int64_t)ni * BLOCK_M + ch;
-            int32_t acc[16];
-#pragma unroll
-            for (int t = 0; t < 16; ++t) acc[t] = (int32_t)r[t];
             if (kb0 == 0 && kb1 == p.num_kb) {
-                dec_finish(p, acc, col);  // the whole K range of this tile was ours
+                dec_finish<DEC_N>(p, acc, col);  // the whole K range of this tile was ours
             } else {
                 // The tile is shared: CTAs g0 .. g0 + count - 1 each hold one K piece.  Park this
                 // piece in its own slot (plain stores: integer partial sums add exactly in any
@@ -266,7 +278,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                         for (int t = 0; t < DEC_N; ++t)
                             if (t < p.M) acc[t] += __ldcg(slot0 + ((int64_t)o * p.M + t) * BLOCK_M + ch);
                     }
-                    dec_finish(p, acc, col);
+                    dec_finish<DEC_N>(p, acc, col);
                     if (et == 0) p.counters[ni] = 0u;  // hand the counters back zeroed
                 }
             }
@@ -310,6 +322,22 @@ DecPlan plan_decode(int num_n, int num_kb, int sms, bool may_share) {
     return pl;
 }
 
+template <int DN>
+sq_status launch_decode(const GemmArgs& a, const DecParams& p, int ctas, cudaStream_t st) {
+    CUtensorMap mw, mx;
+    int s0, s1, s2;
+    if (!make_map(&mw, a.B, 1, a.K, a.N, 1, 1, a.K, 0, 0, BLOCK_K, BLOCK_M, &s0, &s1, &s2)) return SQ_ERR_CUDA;
+    if (!make_map(&mx, a.A, 1, a.K, a.M, 1, 1, a.K, 0, 0, BLOCK_K, DN, &s0, &s1, &s2)) return SQ_ERR_CUDA;
+    static bool attr_set[64] = {false};  // per instantiation and device
+    int dev = 0;
+    SQ_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        SQ_CUDA_OK(cudaFuncSetAttribute(decode_gemm_kernel<DN>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<DN>::SMEM));
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    return launch_pdl(decode_gemm_kernel<DN>, dim3((unsigned)ctas), dim3(DEC_THREADS), (size_t)DecCfg<DN>::SMEM, st, 1, mw, mx, p);
+}
+
 }  // namespace
 
 // Counters (fixed area, zero between calls) + one slot per (shared tile, sharing CTA).  The
@@ -319,9 +347,17 @@ size_t decode_workspace_bytes(int64_t M, int64_t N) {
     return kWsHeader + kDecCounterBytes + (size_t)(kMaxCtas + 2 * num_n) * (size_t)M * tc::BLOCK_M * sizeof(int32_t);
 }
 
+// Up to 32 tokens the activation slices are a small addition to the weight stream and this kernel
+// always wins.  At 33..64 tokens they are half as many bytes again, which a single SM's copy
+// rate does not absorb (measured 0.67-0.75 of HBM); the 128 x 256-tile prefill kernel is then
+// faster whenever its N / 256 tiles fill most of the machine, and slower when they do not
+// (N = 12288: 48 tiles, 0.58 against 0.71 here).
 bool decode_supports(const GemmArgs& a) {
-    return a.M <= DEC_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn &&
-           a.row_absmax_out == nullptr && a.strideA[2] == a.K && a.strideB[2] == a.K;
+    if (!(a.M <= DEC_MAX_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn && a.row_absmax_out == nullptr &&
+          a.strideA[2] == a.K && a.strideB[2] == a.K))
+        return false;
+    if (a.M <= 32) return true;
+    return (a.N + 255) / 256 <= (int64_t)(sm_count() * 2) / 3;
 }
 
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st) {
@@ -343,18 +379,9 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.counters = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsHeader);
     p.part = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader + kDecCounterBytes);
     p.status = a.status;
-    CUtensorMap mw, mx;
-    int s0, s1, s2;
-    if (!make_map(&mw, a.B, 1, a.K, a.N, 1, 1, a.K, 0, 0, BLOCK_K, BLOCK_M, &s0, &s1, &s2)) return SQ_ERR_CUDA;
-    if (!make_map(&mx, a.A, 1, a.K, a.M, 1, 1, a.K, 0, 0, BLOCK_K, DEC_N, &s0, &s1, &s2)) return SQ_ERR_CUDA;
-    static bool attr_set[64] = {false};
-    int dev = 0;
-    SQ_CUDA_OK(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(decode_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DEC_SMEM));
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
-    }
-    return launch_pdl(decode_gemm_kernel, dim3((unsigned)plan.ctas), dim3(DEC_THREADS), (size_t)DEC_SMEM, st, 1, mw, mx, p);
+    if (a.M <= 16) return launch_decode<16>(a, p, plan.ctas, st);
+    if (a.M <= 32) return launch_decode<32>(a, p, plan.ctas, st);
+    return launch_decode<64>(a, p, plan.ctas, st);
 }
 
 }  // namespace sq

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def ws():
-    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 16, 65536, 32768))  # decode scratch is the largest
+    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 64, 65536, 32768))  # decode scratch is the largest
     yield w
     assert sq.device_status(w) == 0, "a device-side wait timed out"
 
@@ -120,7 +120,8 @@ def test_gemm_strided_output(ws):
 
 # decode-shaped calls (M <= 16): swapped operands, K splits with INT32 scratch in the workspace
 DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
-                 (16, 36864, 1024), (2, 4096, 49152)]
+                 (16, 36864, 1024), (2, 4096, 49152),
+                 (17, 512, 512), (32, 1280, 4096), (33, 200, 272), (64, 12288, 6144), (48, 136, 12288), (64, 36864, 1024)]
 
 
 @pytest.mark.parametrize("M,N,K", DECODE_SHAPES)
@@ -144,7 +145,7 @@ def test_decode_gemm_exact_and_workspace_restored(ws, M, N, K):
 
 
 @pytest.mark.parametrize("M,N,K,per_col", [(1, 384, 512, True), (16, 1280, 4096, True), (7, 200, 272, False),
-                                           (16, 36864, 1024, True)])
+                                           (16, 36864, 1024, True), (40, 1280, 4096, True), (64, 200, 272, False)])
 def test_decode_gemm_requant_int8_out(ws, M, N, K, per_col):
     """Decode-shaped GEMM with the requantising epilogue (INT8 codes out, as the QKV and FC1
     projections of a static-step block emit them): byte-exact, the epilogue is fully specified fp32."""
