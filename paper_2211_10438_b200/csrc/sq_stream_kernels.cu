@@ -564,6 +564,8 @@ sq_status softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_
 template <typename T>
 __global__ void residual_add_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b,
                                     int64_t nvec, uint4* __restrict__ out) {
+    pdl_wait();  // a and b come from the kernels in front
+    pdl_launch_dependents();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec;
          i += (int64_t)gridDim.x * blockDim.x) {
         float fa[8], fb[8];
@@ -581,10 +583,10 @@ sq_status residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, voi
     const int64_t nvec = n / 8;
     const unsigned grid = (unsigned)std::min<int64_t>((nvec + 255) / 256, 8LL * sm_count());
     if (dt == SQ_F16)
-        residual_add_kernel<__half><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, nvec, (uint4*)out);
-    else
-        residual_add_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const uint4*)a, (const uint4*)b, nvec, (uint4*)out);
-    return launch_status();
+        return launch_pdl(residual_add_kernel<__half>, dim3(grid), dim3(256), 0, st, 1, (const uint4*)a, (const uint4*)b, nvec,
+                          (uint4*)out);
+    return launch_pdl(residual_add_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, 1, (const uint4*)a, (const uint4*)b,
+                      nvec, (uint4*)out);
 }
 
 }  // namespace sq
