@@ -193,3 +193,73 @@ def test_mtnlg_calibration_stream_and_alphas():
         Wq, wsc = sq.sq_quant_weight(dev(W, "bf16"), dev(s), "per_channel")
         oq, osc = oracle.quant_weight(W, s, "per_channel")  # same s on both sides
         assert np.array_equal(host(Wq), oq) and np.array_equal(host(wsc), osc)
+
+
+def test_generation_attention_gpt3_shape_sampled_heads():
+    """The KV-cache attention row exactly as bench.py launches it (96 heads x 128, batch 16, context
+    lengths uniform in [1024, 2048], the kernel appending the newest token itself); 10 sampled
+    (sequence, head) pairs go through the oracle, and the whole cache is checked for the append."""
+    B, H, L, D = 16, 96, 2048, 128
+    rng = synth.rng_for(40, 1)
+    K = synth.int8_tensor(40, 2, (B, H, L, D), lo=-100, hi=100)
+    V = synth.int8_tensor(40, 3, (B, H, L, D), lo=-100, hi=100)
+    qkv = synth.int8_tensor(40, 4, (B, 3, H, D), lo=-100, hi=100)
+    lens = rng.integers(L // 2, L + 1, B).astype(np.int32)
+    for b in range(B):  # the newest token's true k, v; the cache holds junk at that position
+        K[b, :, lens[b] - 1], V[b, :, lens[b] - 1] = qkv[b, 1], qkv[b, 2]
+    Kj, Vj = K.copy(), V.copy()
+    for b in range(B):
+        Kj[b, :, lens[b] - 1], Vj[b, :, lens[b] - 1] = 99, -99
+    kc = dev(Kj)
+    vc = dev(np.ascontiguousarray(Vj.reshape(B, H, L // 4, 4, D).transpose(0, 1, 2, 4, 3)))
+    qd = dev(qkv.reshape(B, 3 * H * D))
+    a_qk, a_pv = np.float32(0.0009), np.float32(0.01 / 127)
+    r = np.array([1000.0], np.float32)
+    ws = sq.new_workspace(256)
+    out = sq.sq_w8a8_decode_attention(qd, kc, vc, dev(lens), B, H, D, L, L, a_qk, a_pv, ws, requant_mul=dev(r),
+                                      k_new=qd[:, H * D:], v_new=qd[:, 2 * H * D:])
+    torch.cuda.synchronize()
+    assert sq.device_status(ws) == 0
+    got = host(out).reshape(B, H, D).astype(np.int32)
+    pairs = {(int(b), int(h)) for b, h in zip(rng.integers(0, B, 10), rng.integers(0, H, 10))}
+    ndiff = ntot = 0
+    for b, h in sorted(pairs):
+        want, _ = oracle.kv_decode_attention(qkv[b:b + 1, 0, h:h + 1], K[b:b + 1, h:h + 1], V[b:b + 1, h:h + 1], [lens[b]],
+                                             a_qk, a_pv, requant_mul=r)
+        d = np.abs(got[b, h] - want[0, 0].astype(np.int32))
+        assert d.max() <= 2
+        ndiff += int((d != 0).sum())
+        ntot += d.size
+    assert ndiff / ntot <= 2e-2
+    # the append: every sequence's newest position now holds its true k and v, nothing else moved
+    gk = host(kc)
+    gv = host(vc).transpose(0, 1, 2, 4, 3).reshape(B, H, L, D)
+    assert np.array_equal(gk, K) and np.array_equal(gv, V)
+
+
+def test_fused_attention_opt30b_shape_sampled_heads():
+    """Fused prompt attention at the block benchmark's shape (56 heads x 128, S = 512, batch 16):
+    8 sampled (sequence, head) pairs through the oracle's unfused chain with fp32 scores."""
+    B, H, S, D = 16, 56, 512, 128
+    qkv = synth.int8_tensor(41, 1, (B * S, 3 * H * D), lo=-100, hi=100)
+    a_qk, a_pv = np.float32(0.0009), np.float32(0.01 / 127)
+    r = np.array([1.0 / 0.004], np.float32)
+    ws = sq.new_workspace(256)
+    out = torch.empty((B * S, H * D), dtype=torch.int8, device="cuda")
+    sq.sq_w8a8_attention(dev(qkv), B, H, S, D, a_qk, a_pv, dev(r), out, ws)
+    torch.cuda.synchronize()
+    assert sq.device_status(ws) == 0
+    got = host(out).reshape(B, S, H, D).astype(np.int32)
+    v5 = qkv.reshape(B, S, 3, H, D)
+    rng = synth.rng_for(41, 2)
+    ndiff = ntot = 0
+    for b, h in zip(rng.integers(0, B, 8), rng.integers(0, H, 8)):
+        q, k, v = (np.ascontiguousarray(v5[b, :, i, h]) for i in range(3))
+        _, scores = oracle.w8a8_bmm(q[None], k[None], float(a_qk), out_dtype="f32")
+        P, _ = oracle.softmax_quant_p(scores[0])
+        _, o = oracle.w8a8_bmm(P[None], v[None], float(a_pv), b_is_kn=True, requant_mul=r)
+        d = np.abs(got[b, :, h] - o[0].astype(np.int32))
+        assert d.max() <= 2
+        ndiff += int((d != 0).sum())
+        ntot += d.size
+    assert ndiff / ntot <= 5e-3
