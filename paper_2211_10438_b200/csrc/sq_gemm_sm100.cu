@@ -74,7 +74,29 @@ struct Params {
     int c_tma;  // C leaves through TMA stores (needs 16-byte aligned base and strides)
     int c_slot_row, c_slot_head, c_slot_batch;
     uint32_t* status;
+    // K split of the last, partly filled wave of tiles (plain GEMMs only; split == 1: none).
+    // Units [0, full_tiles) are whole tiles; unit full_tiles + t * split + i is K piece i of tile
+    // full_tiles + t.  A piece parks its INT32 accumulators in its slot of `part`; the CTA that
+    // arrives last for a tile (per CTA of a pair: `counters`) adds the others and runs the epilogue.
+    uint32_t full_tiles, total_units;
+    int split, kb_per_piece;
+    int32_t* part;
+    uint32_t* counters;
 };
+
+// unit id -> tile and K-block range; piece < 0 for a whole tile (kb1 is then the tile's own count)
+__device__ __forceinline__ void unit_of(uint32_t u, const Params& p, uint32_t& tile, int& kb0, int& kb1, int& piece) {
+    if (u < p.full_tiles) {
+        tile = u; kb0 = 0; kb1 = -1; piece = -1;
+        return;
+    }
+    const uint32_t r = u - p.full_tiles;
+    const uint32_t t = r / (uint32_t)p.split;
+    piece = (int)(r - t * (uint32_t)p.split);
+    tile = p.full_tiles + t;
+    kb0 = piece * p.kb_per_piece;
+    kb1 = min(p.num_kb, kb0 + p.kb_per_piece);
+}
 
 // tile id -> (batch*heads index, m tile, n tile).  Within one matrix, tiles are visited in
 // bands of G m-tiles so that the CTAs running at the same time share A and B tiles in L2.
@@ -119,12 +141,15 @@ __device__ __forceinline__ int tile_num_kb(const Params& p, int mi, int tile_m) 
 // conflict-free 16-byte writes) and one lane issues a TMA store, which also clips the M and N
 // tails.  If C is not 16-byte aligned the rows are written directly instead.
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N>
+// FIX: this CTA arrived last for a K-split tile: the other pieces' partial sums (fix_count slots,
+// fix_stride ints apart, fix_base already at this thread's row) are added to the accumulators first.
+template <int BLOCK_N, bool FIX = false>
 __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
                                               uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
                                               int h, int64_t c_off, const float* s_wscale,
                                               const float* s_bias, const float* s_requant, int lane,
-                                              int cc_begin, int cc_end) {
+                                              int cc_begin, int cc_end, const int32_t* fix_base = nullptr,
+                                              int fix_count = 0, int fix_mine = 0, size_t fix_stride = 0) {
     const bool row_ok = row < p.M;
     float xs = p.alpha;
     if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
@@ -140,6 +165,21 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
         uint32_t r[32];
         tmem_ld32(taddr + cc * 32, r);  // warp-collective: executed by every lane
         tmem_ld_wait();
+        if (FIX) {
+            for (int o = 0; o < fix_count; ++o) {
+                if (o == fix_mine) continue;
+                // slot layout [4-column group][row][4]: a thread's 16 bytes, a warp's 512 contiguous bytes
+                const int4* src = reinterpret_cast<const int4*>(fix_base + (size_t)o * fix_stride) + (size_t)(cc * 8) * BLOCK_M;
+                int4 t[8];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) t[v] = __ldcg(src + (size_t)v * BLOCK_M);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    r[4 * v] += (uint32_t)t[v].x; r[4 * v + 1] += (uint32_t)t[v].y;
+                    r[4 * v + 2] += (uint32_t)t[v].z; r[4 * v + 3] += (uint32_t)t[v].w;
+                }
+            }
+        }
         const int64_t ncols = p.N - (col0 + cc * 32);  // valid columns in this chunk
         // ---- Eq. 2 on the chunk; w[] receives the packed output words ----
         uint32_t w[32];
@@ -268,6 +308,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tmem_empty + 2);
     volatile uint32_t* abort_flag = tmem_holder + 1;
     volatile uint32_t* epi_go = tmem_holder + 2;
+    volatile uint32_t* epi_last = tmem_holder + 3;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = CG == 1 ? 0 : (int)cluster_ctarank();  // 0 = even CTA: issues the MMAs
@@ -304,17 +345,20 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (uint32_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
+            for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
+                uint32_t tile;
+                int kb0, kb1, piece;
+                unit_of(u, p, tile, kb0, kb1, piece);
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
-                const int tile_kb = tile_num_kb(p, mi, BLOCK_M * CG);
+                if (piece < 0) kb1 = tile_num_kb(p, mi, BLOCK_M * CG);
                 const int b = bh / p.heads, h = bh - b * p.heads;
                 int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
                 ca[p.a_slot_row] = (mi * CG + rank) * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
                 cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
                 const int b_row0 = ni * BLOCK_N + rank * C::B_ROWS;  // this CTA's share of the B tile
-                for (int kb = 0; kb < tile_kb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
                     uint8_t* sa = stage_base + stage * C::STAGE_BYTES;
                     uint8_t* sb = sa + C::A_BYTES;
@@ -344,15 +388,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
-            for (uint32_t tile = first_tile; ok && tile < p.total_tiles; tile += tile_step) {
+            for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
+                uint32_t tile;
+                int kb0, kb1, piece;
+                unit_of(u, p, tile, kb0, kb1, piece);
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
-                const int tile_kb = tile_num_kb(p, mi, BLOCK_M * CG);
+                if (piece < 0) kb1 = tile_num_kb(p, mi, BLOCK_M * CG);
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
-                for (int kb = 0; kb < tile_kb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 3))) break;
                     tcgen05_fence_after();
                     const uint32_t sa = smem_u32(stage_base + stage * C::STAGE_BYTES);
@@ -361,7 +408,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         const uint64_t adesc = make_smem_desc(sa + k * UMMA_K, 16);
                         const uint64_t bdesc = make_smem_desc(sb + k * b_kstep, p.b_is_kn ? 16384u : 16u);
-                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc, (kb | k) != 0 ? 1u : 0u);
+                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit<CG>(empty_bar + stage);  // frees the stage (in both CTAs) once these MMAs retire
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -382,7 +429,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int quarter = warp & 3, half = warp >> 2;
         int slot = 0;
         uint32_t slot_phase = 0;
-        for (uint32_t tile = first_tile; tile < p.total_tiles; tile += tile_step) {
+        for (uint32_t u = first_tile; u < p.total_units; u += tile_step) {
+            uint32_t tile;
+            int kb0, kb1, piece;
+            unit_of(u, p, tile, kb0, kb1, piece);
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
             if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -420,8 +470,39 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int g_split = EW == 8 ? (groups + 1) / 2 : groups;
             const int cc_begin = half == 0 ? 0 : g_split * cps;
             const int cc_end = half == 0 ? min(g_split * cps, BLOCK_N / 32) : BLOCK_N / 32;
-            epilogue_slot<BLOCK_N>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
-                                   c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
+            if (EW == 8 || piece < 0) {  // (the eight-warp configuration serves short reductions: never split)
+                epilogue_slot<BLOCK_N>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
+                                       c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
+            } else {
+                // K piece of a split tile: park the accumulators, then see who is last
+                constexpr size_t kTileInts = (size_t)BLOCK_M * BLOCK_N;
+                const uint32_t rem = tile - p.full_tiles;
+                // slot layout [4-column group][row of this CTA][4]: a thread stores 16 bytes, a warp 512 contiguous bytes
+                int32_t* tile_slots = p.part + ((size_t)rem * p.split * CG + rank) * kTileInts +
+                                      (size_t)(quarter * 32 + lane) * 4;  // piece 0, this CTA, this row
+                int32_t* mine = tile_slots + (size_t)piece * CG * kTileInts;
+                for (int cc = cc_begin; cc < cc_end; ++cc) {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + cc * 32, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        __stcg(reinterpret_cast<int4*>(mine) + (size_t)(cc * 8 + v) * BLOCK_M,
+                               make_int4((int)r[4 * v], (int)r[4 * v + 1], (int)r[4 * v + 2], (int)r[4 * v + 3]));
+                }
+                __threadfence();
+                epi_bar_sync<C::EPI_THREADS>();
+                if (et == 0)
+                    *epi_last = atomicAdd(p.counters + rem * CG + rank, 1u) == (uint32_t)(p.split - 1) ? 1u : 0u;
+                epi_bar_sync<C::EPI_THREADS>();
+                if (*epi_last != 0u) {
+                    __threadfence();
+                    epilogue_slot<BLOCK_N, true>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b,
+                                                 h, c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end,
+                                                 tile_slots, p.split, piece, (size_t)CG * kTileInts);
+                    if (et == 0) p.counters[rem * CG + rank] = 0u;  // hand the counter back zeroed
+                }
+            }
 
             // accumulator slot drained: hand it back to the MMA warp (in the even CTA)
             tcgen05_fence_before();
@@ -447,6 +528,38 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // ------------------------------------------------------------------------------------
 // Host side: tensor maps + launch
 // ------------------------------------------------------------------------------------
+// K split of the last wave.  With T tiles on G resident CTA groups the last R = T mod G tiles keep
+// only part of the machine busy.  Cutting each of them into s K pieces spreads them over up to
+// R * s groups, at the price of parking and re-reading INT32 partial sums (128 KB per CTA and
+// piece, which a single SM reads at only ~50 GB/s).  Measured on B200: it pays for long
+// reductions only (a 256 x 256 tile of K = 20480 takes 66 us: 156 -> 144 us on 2048 x 5120 x 20480,
+// 291 -> 271 us on 2048 x 7168 x 28672), loses for K = 5120 (tile 16 us) at every s, and loses badly
+// when the pieces need more than one round.  Hence: K >= 12288, s in {4, 3, 2} with R * s <= G
+// and at least 16 K blocks per piece.
+struct SplitPlan { uint32_t full; int split; int kb_per_piece; };
+inline SplitPlan plan_split(int64_t total_tiles, int num_kb, int groups, int64_t K, int tile_m, int tile_n) {
+    SplitPlan pl{(uint32_t)total_tiles, 1, num_kb};
+    (void)tile_m; (void)tile_n;
+    if (groups <= 0 || total_tiles <= 0 || K < 12288) return pl;
+    const int64_t R = total_tiles % groups;
+    if (R == 0) return pl;
+    for (int s = 4; s >= 2; --s) {
+        const int per = (num_kb + s - 1) / s;
+        if (R * s > groups || per < 16 || (num_kb + per - 1) / per != s) continue;
+        pl.split = s;
+        pl.kb_per_piece = per;
+        pl.full = (uint32_t)(total_tiles - R);
+        break;
+    }
+    return pl;
+}
+template <int BLOCK_N, int CG>
+inline size_t split_workspace_bytes(const SplitPlan& pl, int64_t total_tiles) {
+    if (pl.split <= 1) return kWsHeader;
+    return kWsHeader + kDecCounterBytes +
+           (size_t)(total_tiles - pl.full) * pl.split * CG * BLOCK_M * BLOCK_N * sizeof(int32_t);
+}
+
 template <int BLOCK_N, int CG, int EW>
 sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     using C = Cfg<BLOCK_N, CG, EW>;
@@ -513,7 +626,21 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
                                         C::SMEM_BYTES));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const int groups = (int)std::min<int64_t>((int64_t)p.total_tiles, sm_count() / CG);
+    // K split of the last wave: plain GEMMs only, and only with the scratch it needs
+    p.full_tiles = p.total_tiles; p.total_units = p.total_tiles; p.split = 1; p.kb_per_piece = p.num_kb;
+    p.part = nullptr; p.counters = nullptr;
+    if (EW == 4 && a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn) {
+        const SplitPlan pl = plan_split(p.total_tiles, p.num_kb, sm_count() / CG, a.K, BLOCK_M * CG, BLOCK_N);
+        if (pl.split > 1 && (p.total_tiles - pl.full) * CG <= kDecCounterBytes / 4 &&
+            a.ws_bytes >= split_workspace_bytes<BLOCK_N, CG>(pl, p.total_tiles)) {
+            p.full_tiles = pl.full; p.split = pl.split; p.kb_per_piece = pl.kb_per_piece;
+            p.total_units = pl.full + (p.total_tiles - pl.full) * (uint32_t)pl.split;
+            char* ws = reinterpret_cast<char*>(a.status);
+            p.counters = reinterpret_cast<uint32_t*>(ws + kWsHeader);
+            p.part = reinterpret_cast<int32_t*>(ws + kWsHeader + kDecCounterBytes);
+        }
+    }
+    const int groups = (int)std::min<int64_t>((int64_t)p.total_units, sm_count() / CG);
     return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
                       (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, p);
 }
@@ -546,6 +673,17 @@ __global__ void bounded_wait_selftest_kernel(uint32_t* status, uint32_t budget) 
 sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st) {
     bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, budget);
     return launch_status();
+}
+
+// Scratch a plain GEMM of this shape can use for the K split of its last wave (the tile
+// configuration follows gemm_i8's dispatch); with less the split is simply not taken.
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 128 || N <= 128 || K <= 1024) return kWsHeader;  // only the CTA-pair configuration splits
+    const int64_t tiles = ((M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * ((N + 255) / 256);
+    if (tiles >= (int64_t)1 << 31) return kWsHeader;
+    const int num_kb = (int)((K + BLOCK_K - 1) / BLOCK_K);
+    const SplitPlan pl = plan_split(tiles, num_kb, sm_count() / 2, K, 2 * BLOCK_M, 256);
+    return split_workspace_bytes<256, 2>(pl, tiles);
 }
 
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {

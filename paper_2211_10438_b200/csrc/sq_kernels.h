@@ -67,6 +67,7 @@ struct GemmArgs {
     size_t ws_bytes;      // size of the caller's workspace
 };
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);  // scratch for the K split of the last wave
 sq_status attention_i8(const int8_t* qkv, int64_t B, int64_t H, int64_t S, int64_t d, float alpha_qk, float alpha_pv,
                        const float* requant_mul, int8_t* out, uint32_t* status, cudaStream_t st);
 sq_status kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T, int64_t H, const int32_t* pos0, int8_t* kc,

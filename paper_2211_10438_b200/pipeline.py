@@ -59,9 +59,8 @@ class LinearBlock:
             self.buf[n] = dict(Xq=torch.empty((M, K), dtype=torch.int8, device=dev),
                                xs=torch.empty(ns, dtype=torch.float32, device=dev),
                                Y=torch.empty((M, N), dtype=act_dtype, device=dev))
-        need = max(sq.workspace_bytes(sq.SQ_OP_GEMM, M, max(l.Wq.shape[0] for l in self.lin.values()),
-                                      max(l.Wq.shape[1] for l in self.lin.values())),
-                   sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, 0))
+        need = max([sq.workspace_bytes(sq.SQ_OP_GEMM, M, l.Wq.shape[0], l.Wq.shape[1]) for l in self.lin.values()] +
+                   [sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, 0)])
         self.ws = sq.new_workspace(need, dev)
         self.launches_per_step = 8 if gran != "per_tensor_dynamic" else 12
         self.gemm_events = None  # optional list collecting (start, stop) CUDA events per GEMM
@@ -203,7 +202,9 @@ class DecoderBlockStatic:
         self.attn, self.proj, self.h = e((M, hid), torch.int8), e((M, hid), act_dtype), e((M, hid), act_dtype)
         self.x2q, self.f1q = e((M, hid), torch.int8), e((M, ffn), torch.int8)
         self.fc2, self.y = e((M, hid), act_dtype), e((M, hid), act_dtype)
-        self.ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid), dev)
+        need = max([sq.workspace_bytes(sq.SQ_OP_GEMM, M, l.Wq.shape[0], l.Wq.shape[1]) for l in lin.values()] +
+                   [sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid)])
+        self.ws = sq.new_workspace(need, dev)
         self.launches_per_step = 9 if self.fused_attention else 11
 
     def forward(self, x):
@@ -272,9 +273,8 @@ class DecoderBlockDecode:
         self.v_cache = torch.zeros((B, H, L_max // 4, d, 4), dtype=torch.int8, device=dev)
         self.ctx = torch.zeros(B, dtype=torch.int32, device=dev)
         self.lens = torch.ones(B, dtype=torch.int32, device=dev)  # ctx + 1: what the new token attends over
-        need = max(sq.workspace_bytes(sq.SQ_OP_GEMM, B, max(l.Wq.shape[0] for l in lin.values()),
-                                      max(l.Wq.shape[1] for l in lin.values())),
-                   sq.workspace_bytes(sq.SQ_OP_LN_QUANT, B, 0, hid))
+        need = max([sq.workspace_bytes(sq.SQ_OP_GEMM, B, l.Wq.shape[0], l.Wq.shape[1]) for l in lin.values()] +
+                   [sq.workspace_bytes(sq.SQ_OP_LN_QUANT, B, 0, hid)])
         self.ws = sq.new_workspace(need, dev)
         self.launches_per_step = 9
 

@@ -118,6 +118,33 @@ def test_gemm_strided_output(ws):
     assert np.all(got[:, N:] == -7.0)  # nothing written beyond the N columns
 
 
+# long reductions whose tile count leaves a partly filled last wave: with the recommended workspace
+# the tiles of that wave are cut along K (2 .. 4 pieces) and meet in the workspace; without it they are not
+SPLIT_SHAPES = [(512, 4096, 12288), (2048, 5120, 20480), (300, 2304, 16400), (2048, 7168, 28672), (520, 1000, 12304),
+                (256, 20480, 12288)]
+
+
+@pytest.mark.parametrize("M,N,K", SPLIT_SHAPES)
+def test_gemm_last_wave_k_split_is_exact(M, N, K):
+    Xq, Wq = synth.int8_tensor(27, 1, (M, K)), synth.int8_tensor(27, 2, (N, K))
+    rng = synth.rng_for(27, 3)
+    xs = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = synth.bias(27, 4, N, "f16", std=0.5)
+    need = sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K)
+    big, small = sq.new_workspace(need), sq.new_workspace(256)
+    want_acc = oracle.gemm_i32(Xq, Wq)
+    want = oracle.round_to(oracle.dequant(want_acc, xs, wsc, bias, relu=True), "f16")
+    Xd, Wd = dev(Xq), dev(Wq)
+    for ws in (big, small, big):  # the second use of `big` must find its counters zeroed by the first
+        acc = sq.sq_w8a8_gemm(Xd, Wd, None, None, ws, out_dtype=torch.int32)
+        assert np.array_equal(host(acc), want_acc)
+        y = sq.sq_w8a8_gemm(Xd, Wd, dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True, out_dtype=torch.float16)
+        assert np.array_equal(host(y), want)
+        assert sq.device_status(ws) == 0
+    assert not big[4:33024].any(), "header and counters not handed back zero-filled"
+
+
 # decode-shaped calls (M <= 16): swapped operands, K splits with INT32 scratch in the workspace
 DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
                  (16, 36864, 1024), (2, 4096, 49152),
