@@ -22,7 +22,9 @@
 // keys above the diagonal are masked by selecting -inf as the exponent argument (no branches).
 // Measured: time = 5.2 us per CTA + 2.05 us per (key tile, pass) over 296 resident CTAs; backing
 // the waiting lanes off with nanosleep, or prefetching TMEM chunks into a second register buffer,
-// was slower.
+// was slower, and a persistent variant (two CTAs per SM walking a list of tiles, one TMEM
+// allocation and barrier set-up per CTA) took the same time: the per-tile cost is the serial
+// load -> first MMA -> ... -> epilogue latency of a tile, not the launch of its CTA.
 // Every wait is bounded and reports through the status word.
 #include "sq_kernels.h"
 #include "sq_tcgen05.cuh"
