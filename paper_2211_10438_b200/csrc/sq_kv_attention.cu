@@ -365,22 +365,12 @@ kv_cache_write_kernel(const int8_t* __restrict__ qkv, int64_t ld, int B, int T, 
     }
 }
 
-int sm_count_kv() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    }
-    return n;
-}
-
 }  // namespace
 
 // Cluster width: enough CTAs to fill the machine a few times over, each keeping a worthwhile
 // number of keys, and a score buffer that fits in shared memory.
 int kv_choose_cluster(int64_t B, int64_t H, int64_t max_len) {
-    const int64_t want = 4LL * sm_count_kv();
+    const int64_t want = 4LL * sm_count();
     int c = 1;
     while (c < KV_MAX_CLUSTER && B * H * c < want && max_len / (2 * c) >= 256) c *= 2;
     while (c < KV_MAX_CLUSTER && kv_smem_bytes((int)(((max_len + c - 1) / c + KV_TILE - 1) / KV_TILE * KV_TILE)) > 200 * 1024) c *= 2;
