@@ -499,3 +499,48 @@ def test_clipped_absmax_pins():
     ta = oracle.row_absmax(X)
     assert oracle.clipped_absmax(ta, oracle.clip_count(1000, 0.02)) < 0.1 * oracle.clipped_absmax(ta, 0)
     assert oracle.clipped_absmax(ta, 0) == oracle.calib_absmax(X).max()
+
+
+def test_decoder_block_static_tracks_the_float_block():
+    """The W8A8 block (static steps taken from the float block's own maxima) stays within a few
+    per cent of the same block computed in fp64 with library routines -- a dropped residual, a
+    transposed weight, a missing 1/sqrt(d) or a wrong mask would be off by far more."""
+    rng = np.random.default_rng(48)
+    B, S, H, d, ffn = 2, 24, 2, 16, 64
+    hid = H * d
+    f16 = lambda a: a.astype(np.float16).astype(np.float32)
+    x = f16(rng.standard_normal((B * S, hid)))
+    g1, b1 = f16(1 + 0.1 * rng.standard_normal(hid)), f16(0.1 * rng.standard_normal(hid))
+    g2, b2 = f16(1 + 0.1 * rng.standard_normal(hid)), f16(0.1 * rng.standard_normal(hid))
+    shapes = {"qkv": (3 * hid, hid), "out_proj": (hid, hid), "fc1": (ffn, hid), "fc2": (hid, ffn)}
+    p = {"g1": g1, "b1": b1, "g2": g2, "b2": b2}
+    Wf, bias = {}, {}
+    for n, (N, K) in shapes.items():
+        W = f16(rng.standard_normal((N, K)) / np.sqrt(K))
+        Wq, ws = oracle.quant_weight(W, None, "per_channel")
+        bias[n] = f16(0.05 * rng.standard_normal(N))
+        p[n] = {"Wq": Wq, "w_scale": ws, "bias": bias[n]}
+        Wf[n] = torch.from_numpy(Wq.astype(np.float64) * ws[:, None].astype(np.float64))  # the weights the block really uses
+    # the float block, fp64, library routines
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    X = t(x)
+    ln1 = torch.nn.functional.layer_norm(X, (hid,), t(g1), t(b1), 1e-5)
+    qkv = ln1 @ Wf["qkv"].T + t(bias["qkv"])
+    q, k, v = (qkv[:, i * hid:(i + 1) * hid].reshape(B, S, H, d).permute(0, 2, 1, 3) for i in range(3))
+    sc = q @ k.transpose(-1, -2) / np.sqrt(d)
+    sc = sc + torch.full((S, S), float("-inf"), dtype=torch.float64).triu(1)
+    att = (torch.softmax(sc, -1) @ v).permute(0, 2, 1, 3).reshape(B * S, hid)
+    h = X + att @ Wf["out_proj"].T + t(bias["out_proj"])
+    ln2 = torch.nn.functional.layer_norm(h, (hid,), t(g2), t(b2), 1e-5)
+    f1 = torch.relu(ln2 @ Wf["fc1"].T + t(bias["fc1"]))
+    y = h + f1 @ Wf["fc2"].T + t(bias["fc2"])
+    step = lambda a: float(a.abs().max()) / 127.0
+    p.update(d_ln1=step(ln1), d_q=step(qkv[:, :hid]), d_k=step(qkv[:, hid:2 * hid]), d_v=step(qkv[:, 2 * hid:]),
+             d_attn=step(att), d_ln2=step(ln2), d_fc1=step(f1))
+    out = oracle.decoder_block_static(x, p, B, S, H, d, "f16")
+    rel = lambda a, b: float(np.linalg.norm(np.asarray(a, np.float64) - b.numpy()) / np.linalg.norm(b.numpy()))
+    assert rel(out["h"], h) < 0.02
+    assert rel(out["y"], y) < 0.03
+    assert rel(out["attn"].astype(np.float64) * p["d_attn"], att) < 0.06
+    # and the error is not zero: the block does quantise
+    assert rel(out["y"], y) > 1e-4
