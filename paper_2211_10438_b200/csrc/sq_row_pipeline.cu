@@ -48,10 +48,15 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int g, int gw
 }
 
 // EXACT: the row has exactly GROUP * V vectors, so no per-vector bounds checks are needed.
-template <typename T, int GROUP, int V, bool LN, bool EXACT>
+// MUL (never together with LN): every element is first multiplied by a per-column fp32 factor --
+// s_j when weights are folded (Eq. 3), 1/s_j for an activation whose producer cannot absorb it.
+// The factors live in shared memory for the CTA's lifetime, in the space LayerNorm's parameters
+// would take (4 bytes per column either way).
+template <typename T, int GROUP, int V, bool LN, bool EXACT, bool MUL = false>
 __global__ void __launch_bounds__(CTA_THREADS, 1)
 row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__ gamma,
-                const T* __restrict__ beta, float eps, int mode, int stages, int8_t* __restrict__ Xq,
+                const T* __restrict__ beta, const float* __restrict__ col_mul, float eps, int mode, int stages,
+                int8_t* __restrict__ Xq,
                 float* __restrict__ scale, float* __restrict__ absmax_word, float* __restrict__ stats,
                 int stats_are_input, uint32_t* __restrict__ status) {
     constexpr int G = CTA_THREADS / GROUP;  // rows in flight per CTA
@@ -61,7 +66,8 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     const int nvec = C >> 3;
     uint8_t* s_gamma = smem;                                   // [C] T   (LN only)
     uint8_t* s_beta = smem + (LN ? row_bytes : 0);             // [C] T   (LN only)
-    uint8_t* s_rows = smem + (LN ? 2 * row_bytes : 0);         // [G][stages][C] T
+    const float* s_mul = reinterpret_cast<const float*>(smem); // [C] fp32 (MUL only)
+    uint8_t* s_rows = smem + ((LN || MUL) ? 2 * row_bytes : 0);  // [G][stages][C] T
     uint64_t* full = reinterpret_cast<uint64_t*>(s_rows + (size_t)G * stages * row_bytes);  // [G][stages]
     float* s_red = reinterpret_cast<float*>(full + G * stages);                             // [G][3][NW]
 
@@ -90,6 +96,10 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 bulk_load(my_rows + (size_t)s * row_bytes, X + r * C, (uint32_t)row_bytes, my_full + s);
             }
         }
+    }
+    if (MUL) {
+        const float4* m4 = reinterpret_cast<const float4*>(col_mul);
+        for (int v = tid; v < 2 * nvec; v += CTA_THREADS) reinterpret_cast<float4*>(smem)[v] = __ldg(m4 + v);
     }
     if (LN) {  // parameters: global -> shared once per CTA
         const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
@@ -198,6 +208,22 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                     }
                 }
             }
+        } else if (MUL) {
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const int v = gt + i * GROUP;
+                if (EXACT || v < nvec) {
+                    const float4 m0 = reinterpret_cast<const float4*>(s_mul)[2 * v];
+                    const float4 m1 = reinterpret_cast<const float4*>(s_mul)[2 * v + 1];
+                    float* f = y[i];
+                    f[0] = __fmul_rn(f[0], m0.x); f[1] = __fmul_rn(f[1], m0.y);
+                    f[2] = __fmul_rn(f[2], m0.z); f[3] = __fmul_rn(f[3], m0.w);
+                    f[4] = __fmul_rn(f[4], m1.x); f[5] = __fmul_rn(f[5], m1.y);
+                    f[6] = __fmul_rn(f[6], m1.z); f[7] = __fmul_rn(f[7], m1.w);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(f[k]));
+                }
+            }
         } else if (mode == ROW_DYNAMIC || mode == ROW_ABSMAX_ONLY) {
             uint32_t pm = 0u;  // packed running max of |x|: exact in fp16/bf16
 #pragma unroll
@@ -241,20 +267,20 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     (void)parity;
 }
 
-template <typename T, int GROUP, int V, bool LN, bool EXACT = false>
-sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, const void* beta, float eps,
+template <typename T, int GROUP, int V, bool LN, bool EXACT = false, bool MUL = false>
+sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, const void* beta, const float* col_mul, float eps,
                       int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats, int stats_are_input,
                       uint32_t* status, cudaStream_t st) {
     constexpr int G = CTA_THREADS / GROUP;
     const size_t row_bytes = (size_t)C * 2;
-    const size_t fixed = (LN ? 2 * row_bytes : 0) + 2048 /*barriers + reduction scratch*/;
+    const size_t fixed = ((LN || MUL) ? 2 * row_bytes : 0) + 2048 /*barriers + reduction scratch*/;
     const size_t budget = 220 * 1024;
     if (budget < fixed + G * row_bytes) return SQ_ERR_UNSUPPORTED;
     int stages = (int)((budget - fixed) / (G * row_bytes));
     stages = std::min(stages, 8);
-    const size_t smem = (LN ? 2 * row_bytes : 0) + (size_t)G * stages * row_bytes + (size_t)G * stages * 8 +
+    const size_t smem = ((LN || MUL) ? 2 * row_bytes : 0) + (size_t)G * stages * row_bytes + (size_t)G * stages * 8 +
                         (size_t)G * 3 * (GROUP / 32) * 4 + (size_t)G * 4 + 128;
-    auto kern = row_pipe_kernel<T, GROUP, V, LN, EXACT>;
+    auto kern = row_pipe_kernel<T, GROUP, V, LN, EXACT, MUL>;
     static bool attr_set[64] = {false};
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
@@ -264,7 +290,7 @@ sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, co
     }
     const int grid = (int)std::min<int64_t>((M + G - 1) / G, sm_count());
     return launch_pdl(kern, dim3((unsigned)grid), dim3(CTA_THREADS), smem, st, 1, static_cast<const T*>(X), M,
-                      (int)C, static_cast<const T*>(gamma), static_cast<const T*>(beta), eps, mode, stages, Xq, scale,
+                      (int)C, static_cast<const T*>(gamma), static_cast<const T*>(beta), col_mul, eps, mode, stages, Xq, scale,
                       absmax_word, stats, stats_are_input, status);
 }
 
@@ -274,11 +300,11 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
                         int stats_are_input, uint32_t* status, cudaStream_t st) {
     const int64_t nvec = C / 8;
 #define SQ_PIPE(GROUP, V)                                                                                  \
-    return launch_pipe<T, GROUP, V, LN>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,    \
+    return launch_pipe<T, GROUP, V, LN>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale, absmax_word, stats, \
                                         stats_are_input, status, st)
 #define SQ_PIPE_EXACT(GROUP, V)                                                                            \
     if (nvec == (GROUP) * (V))                                                                             \
-        return launch_pipe<T, GROUP, V, LN, true>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, \
+        return launch_pipe<T, GROUP, V, LN, true>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale, absmax_word, \
                                                   stats, stats_are_input, status, st)
     // the hidden sizes of the model shapes this library is benchmarked on divide evenly
     SQ_PIPE_EXACT(64, 10);   // 5120
@@ -297,15 +323,35 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
 #undef SQ_PIPE
 }
 
+// Column-multiplier variant (weights folded with s, activations scaled by 1/s): the generic ladder
+// only -- these calls are offline or rare, so the bounds-check-free instantiations are not built.
+template <typename T>
+sq_status dispatch_pipe_mul(const void* X, int64_t M, int64_t C, const float* col_mul, int mode, int8_t* Xq,
+                            float* scale, float* absmax_word, uint32_t* status, cudaStream_t st) {
+    const int64_t nvec = C / 8;
+#define SQ_PIPE(GROUP, V)                                                                                       \
+    return launch_pipe<T, GROUP, V, false, false, true>(X, M, C, nullptr, nullptr, col_mul, 0.f, mode, Xq, scale, \
+                                                        absmax_word, nullptr, 0, status, st)
+    if (nvec <= 64 * 10) SQ_PIPE(64, 10);    // C <= 5120
+    if (nvec <= 128 * 10) SQ_PIPE(128, 10);  // C <= 10240
+    if (nvec <= 256 * 10) SQ_PIPE(256, 10);  // C <= 20480
+    SQ_PIPE(512, 8);                         // C <= 32768
+#undef SQ_PIPE
+}
+
 }  // namespace
 
 bool row_pipeline_supports(int64_t M, int64_t C, bool has_col_mul) {
-    return !has_col_mul && M > 0 && C % 8 == 0 && C / 8 <= 512 * 8;
+    (void)has_col_mul;  // both plain and column-multiplied rows are served
+    return M > 0 && C % 8 == 0 && C / 8 <= 512 * 8;
 }
 
-sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma, const void* beta,
-                       float eps, bool ln, int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats,
-                       int stats_are_input, uint32_t* status, cudaStream_t st) {
+sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul, const void* gamma,
+                       const void* beta, float eps, bool ln, int mode, int8_t* Xq, float* scale, float* absmax_word,
+                       float* stats, int stats_are_input, uint32_t* status, cudaStream_t st) {
+    if (col_mul != nullptr && !ln)
+        return dt == SQ_F16 ? dispatch_pipe_mul<__half>(X, M, C, col_mul, mode, Xq, scale, absmax_word, status, st)
+                            : dispatch_pipe_mul<__nv_bfloat16>(X, M, C, col_mul, mode, Xq, scale, absmax_word, status, st);
     if (dt == SQ_F16)
         return ln ? dispatch_pipe<__half, true>(X, M, C, gamma, beta, eps, mode, Xq, scale, absmax_word, stats,
                                                 stats_are_input, status, st)
