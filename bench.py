@@ -189,6 +189,15 @@ def timed_rows(device, peaks):
     rows["quant_act_per_tensor_dynamic_16384x20480"] = {"GB/s": 5 * M * C / s / 1e9, "frac_hbm": 5 * M * C / s / 1e9 / peaks["hbm_gbs"],
                                                         "us": s * 1e6}
     del x, Xq
+    # the widest activation of the configurations: MT-NLG's FC2 input, 16384 x 81920 (4.0 GB per launch)
+    Mw, Cw = 16384, 81920
+    xw = torch.randn((Mw, Cw), device=device, dtype=torch.bfloat16)
+    Xw = torch.empty((Mw, Cw), dtype=torch.int8, device=device)
+    xsw = torch.empty(Mw, dtype=torch.float32, device=device)
+    s = t(lambda: sq.sq_quant_act(xw, "per_token", Xq=Xw, x_scale=xsw, workspace=ws), n=5)
+    rows["quant_act_per_token_16384x81920"] = {"GB/s": 3 * Mw * Cw / s / 1e9, "frac_hbm": 3 * Mw * Cw / s / 1e9 / peaks["hbm_gbs"],
+                                               "us": s * 1e6}
+    del xw, Xw
     # offline: fold the smoothing factors into the largest MT-NLG weight and quantise it per output
     # channel (81920 x 20480 bf16, 3.4 GB in, 1.7 GB out)
     Nw, Kw = 81920, 20480

@@ -36,7 +36,7 @@ sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const floa
                     const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
                     float* scale, float* absmax_word, float* stats, int stats_are_input,
                     cudaStream_t st);
-bool row_pipeline_supports(int64_t M, int64_t C, bool has_col_mul);
+bool row_pipeline_supports(int64_t M, int64_t C, bool ln, bool has_col_mul);
 sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul, const void* gamma,
                        const void* beta, float eps, bool ln, int mode, int8_t* Xq, float* scale, float* absmax_word,
                        float* stats, int stats_are_input, uint32_t* status, cudaStream_t st);

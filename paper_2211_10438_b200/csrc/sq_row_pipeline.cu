@@ -157,9 +157,15 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
         }
 
         float m = 0.0f;
-        float y[V][8];
+        // LayerNorm and the column multiplier change the values and keep them as fp32; the plain
+        // quantiser keeps the packed 16-bit row (half the registers: rows of up to 81 920 elements
+        // fit) and unpacks a vector only when it is rounded.
+        constexpr bool FP32_ROW = LN || MUL;
+        float y[FP32_ROW ? V : 1][8];
+        if (FP32_ROW) {
 #pragma unroll
-        for (int i = 0; i < V; ++i) unpack8<T>(raw[i], y[i]);
+            for (int i = 0; i < V; ++i) unpack8<T>(raw[i], y[FP32_ROW ? i : 0]);
+        }
         if (LN) {
             float mu, rstd;
             if (stats_are_input) {
@@ -169,7 +175,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 float sum = 0.0f;
 #pragma unroll
                 for (int i = 0; i < V; ++i) {  // zero-filled vectors add nothing
-                    const float* f = y[i];
+                    const float* f = y[FP32_ROW ? i : 0];
                     sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
                 }
                 mu = group_reduce<false, GROUP>(sum, red, g, gwarp, lane) / (float)C;
@@ -180,7 +186,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                     if (EXACT || gt + i * GROUP < nvec) {
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            const float d = y[i][k] - mu;
+                            const float d = y[FP32_ROW ? i : 0][k] - mu;
                             ss = fmaf(d, d, ss);
                         }
                     }
@@ -202,8 +208,8 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                     unpack8<T>(reinterpret_cast<const uint4*>(s_beta)[v], be);
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        const float t = __fmaf_rn(__fmaf_rn(y[i][k], rstd, shift), ga[k], be[k]);
-                        y[i][k] = t;
+                        const float t = __fmaf_rn(__fmaf_rn(y[FP32_ROW ? i : 0][k], rstd, shift), ga[k], be[k]);
+                        y[FP32_ROW ? i : 0][k] = t;
                         m = fmaxf(m, fabsf(t));
                     }
                 }
@@ -215,7 +221,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 if (EXACT || v < nvec) {
                     const float4 m0 = reinterpret_cast<const float4*>(s_mul)[2 * v];
                     const float4 m1 = reinterpret_cast<const float4*>(s_mul)[2 * v + 1];
-                    float* f = y[i];
+                    float* f = y[FP32_ROW ? i : 0];
                     f[0] = __fmul_rn(f[0], m0.x); f[1] = __fmul_rn(f[1], m0.y);
                     f[2] = __fmul_rn(f[2], m0.z); f[3] = __fmul_rn(f[3], m0.w);
                     f[4] = __fmul_rn(f[4], m1.x); f[5] = __fmul_rn(f[5], m1.y);
@@ -252,13 +258,29 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 const int v = gt + i * GROUP;
-                if (EXACT || v < nvec) qrow[v] = quant8<true>(y[i], inv);
+                if (EXACT || v < nvec) {
+                    if (FP32_ROW) {
+                        qrow[v] = quant8<true>(y[FP32_ROW ? i : 0], inv);
+                    } else {
+                        float f[8];
+                        unpack8<T>(raw[i], f);
+                        qrow[v] = quant8<true>(f, inv);
+                    }
+                }
             }
         } else {  // |y| <= absmax by construction: |y * inv| < 127.5, no clamp needed
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 const int v = gt + i * GROUP;
-                if (EXACT || v < nvec) qrow[v] = quant8<false>(y[i], inv);
+                if (EXACT || v < nvec) {
+                    if (FP32_ROW) {
+                        qrow[v] = quant8<false>(y[FP32_ROW ? i : 0], inv);
+                    } else {
+                        float f[8];
+                        unpack8<T>(raw[i], f);
+                        qrow[v] = quant8<false>(f, inv);
+                    }
+                }
             }
         }
         if (++s == stages) { s = 0; parity ^= 1u; }
@@ -319,7 +341,13 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
     if (nvec <= 128 * 10) SQ_PIPE(128, 10);  // C <= 10240
     if (nvec <= 256 * 8) SQ_PIPE(256, 8);    // C <= 16384  (12288)
     if (nvec <= 256 * 10) SQ_PIPE(256, 10);  // C <= 20480
-    SQ_PIPE(512, 8);                         // C <= 32768  (28672)
+    if (nvec <= 512 * 8 || LN) SQ_PIPE(512, 8);  // C <= 32768  (28672)
+    if constexpr (!LN) {                         // wider rows: plain quantiser only (the row stays packed in registers)
+        if (nvec <= 512 * 12) SQ_PIPE(512, 12);  // C <= 49152
+        if (nvec <= 512 * 16) SQ_PIPE(512, 16);  // C <= 65536
+        SQ_PIPE(512, 20);                        // C <= 81920
+    }
+    return SQ_ERR_UNSUPPORTED;
 #undef SQ_PIPE
 }
 
@@ -341,9 +369,11 @@ sq_status dispatch_pipe_mul(const void* X, int64_t M, int64_t C, const float* co
 
 }  // namespace
 
-bool row_pipeline_supports(int64_t M, int64_t C, bool has_col_mul) {
-    (void)has_col_mul;  // both plain and column-multiplied rows are served
-    return M > 0 && C % 8 == 0 && C / 8 <= 512 * 8;
+bool row_pipeline_supports(int64_t M, int64_t C, bool ln, bool has_col_mul) {
+    // LayerNorm and column-multiplied rows are held as fp32 (up to 32 768 elements); the plain
+    // quantiser holds the packed row (up to 81 920)
+    const int64_t max_vec = (ln || has_col_mul) ? 512 * 8 : 512 * 20;
+    return M > 0 && C % 8 == 0 && C / 8 <= max_vec;
 }
 
 sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul, const void* gamma,

@@ -463,8 +463,9 @@ sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const floa
                     const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
                     float* scale, float* absmax_word, float* stats, int stats_are_input,
                     cudaStream_t st) {
-    // rows up to 32768 elements take the bulk-copy pipeline (LayerNorm never comes with a column multiplier)
-    if (row_pipeline_supports(M, C, col_mul != nullptr) && !(ln && col_mul != nullptr))
+    // the bulk-copy pipeline takes rows up to 32 768 elements (81 920 for the plain quantiser);
+    // LayerNorm never comes with a column multiplier
+    if (row_pipeline_supports(M, C, ln, col_mul != nullptr) && !(ln && col_mul != nullptr))
         return row_pipeline(X, dt, M, C, col_mul, gamma, beta, eps, ln, mode, Xq, scale, absmax_word, stats,
                             stats_are_input, nullptr, st);
 #define SQ_DISPATCH(T)                                                                           \

@@ -79,7 +79,7 @@ def test_quant_weight_exact(dtype, gran, N, K, smooth):
 
 
 SHAPES_ACT = [(16, 512), (37, 5120), (5, 20480), (3, 28672), (2, 49152), (2, 81920), (3, 131072),
-              (1, 8), (130, 7168), (9, 4104), (1, 262144)]
+              (1, 8), (130, 7168), (9, 4104), (1, 262144), (3, 40968), (2, 57352), (2, 73736), (3, 32776)]
 
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
