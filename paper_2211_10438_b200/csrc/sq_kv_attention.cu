@@ -326,8 +326,9 @@ kv_cache_write_kernel(const int8_t* __restrict__ qkv, int64_t ld, int B, int T, 
     const int lane = threadIdx.x & 31;
     const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (wid >= (int64_t)B * H * groups) return;
-    const int gi = (int)(wid % groups);
-    const int h = (int)((wid / groups) % H);
+    // heads vary fastest: the warps of a CTA read neighbouring 128-byte pieces of the same QKV rows
+    const int h = (int)(wid % H);
+    const int gi = (int)((wid / H) % groups);
     const int b = (int)(wid / ((int64_t)groups * H));
     const int p0 = pos0 ? __ldg(pos0 + b) : 0;
     if (p0 < 0 || (int64_t)p0 + T > lmax) {  // would run off the cache: write nothing for this sequence
