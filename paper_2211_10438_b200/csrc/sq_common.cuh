@@ -118,6 +118,30 @@ __device__ __forceinline__ uint2 quant8(const float (&f)[8], float inv) {
     return r;
 }
 
+// The same codes from packed pairs: sm_100's two-wide fp32 multiply-add rounds each half exactly
+// like the scalar instruction and takes one issue slot for two values.
+template <typename T>
+__device__ __forceinline__ void unpack8_pairs(const uint4& v, float2 (&f)[4]) {
+    f[0] = Act<T>::to_float2(v.x); f[1] = Act<T>::to_float2(v.y);
+    f[2] = Act<T>::to_float2(v.z); f[3] = Act<T>::to_float2(v.w);
+}
+template <bool CLAMP = true>
+__device__ __forceinline__ uint2 quant8_pairs(const float2 (&f)[4], float inv) {
+    const float2 inv2 = make_float2(inv, inv), magic2 = make_float2(kRoundMagic, kRoundMagic);
+    uint32_t c[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        float2 r = __ffma2_rn(f[j], inv2, magic2);
+        if (CLAMP) {
+            r.x = fminf(fmaxf(r.x, kRoundMagic - 127.0f), kRoundMagic + 127.0f);
+            r.y = fminf(fmaxf(r.y, kRoundMagic - 127.0f), kRoundMagic + 127.0f);
+        }
+        c[2 * j] = __float_as_uint(r.x);
+        c[2 * j + 1] = __float_as_uint(r.y);
+    }
+    return make_uint2(pack4(c[0], c[1], c[2], c[3]), pack4(c[4], c[5], c[6], c[7]));
+}
+
 // ---------------------------------------------------------------------------------------
 // Reductions
 // ---------------------------------------------------------------------------------------
