@@ -40,9 +40,10 @@ template <bool IS_MAX, int GROUP, int CTA = CTA_THREADS>
 __device__ __forceinline__ float group_reduce(float v, float* red, int g, int gwarp, int lane) {
     // non-negative floats order like their bit patterns: one redux instruction per level
     v = IS_MAX ? __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(v))) : warp_sum(v);
+    constexpr int NW = GROUP / 32;
+    if constexpr (NW == 1) return v;  // one warp per row: every lane already holds the result
     if (lane == 0) red[gwarp] = v;
     group_sync<GROUP, CTA>(g);
-    constexpr int NW = GROUP / 32;
     // every thread folds the NW partials in the same order (identical result in all threads);
     // `red` is 16-byte aligned, so the partials come in with vector loads
     constexpr int NWP = (NW + 3) & ~3;
@@ -366,19 +367,35 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
         // LayerNorm is bound by instruction issue and by the three reductions a row costs: 384
         // threads leave room for 112 to 128 fp32 values per thread, so a row needs only two or
         // three warps (measured: 0.79 -> 0.89 of the copy bandwidth at 7168, 0.75 -> 0.91 at 12288)
-        if (nvec == 64 * 14)
-            return launch_pipe<T, 64, 14, LN, true, false, 384>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale,
-                                                              absmax_word, stats, stats_are_input, status, st);
-        if (nvec == 96 * 16)
-            return launch_pipe<T, 96, 16, LN, true, false, 384>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale,
-                                                              absmax_word, stats, stats_are_input, status, st);
+#define SQ_PIPE_LN384(GROUP, V)                                                                                  \
+        if (nvec == (GROUP) * (V))                                                                               \
+            return launch_pipe<T, GROUP, V, LN, true, false, 384>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale, \
+                                                                  absmax_word, stats, stats_are_input, status, st)
+        SQ_PIPE_LN384(32, 16);   // 4096: one warp per row, no barrier in the reductions
+        SQ_PIPE_LN384(64, 14);   // 7168
+        SQ_PIPE_LN384(64, 16);   // 8192
+        SQ_PIPE_LN384(96, 12);   // 9216
+        SQ_PIPE_LN384(96, 16);   // 12288
+        SQ_PIPE_LN384(128, 14);  // 14336
+#undef SQ_PIPE_LN384
     }
+    SQ_PIPE_EXACT(64, 8);    // 4096
     SQ_PIPE_EXACT(64, 10);   // 5120
     SQ_PIPE_EXACT(128, 7);   // 7168
     SQ_PIPE_EXACT(256, 6);   // 12288
     SQ_PIPE_EXACT(256, 10);  // 20480
     SQ_PIPE_EXACT(512, 7);   // 28672
 #undef SQ_PIPE_EXACT
+    if constexpr (LN) {
+#define SQ_PIPE_LN384_ANY(GROUP, V)                                                                              \
+        if (nvec <= (GROUP) * (V))                                                                               \
+            return launch_pipe<T, GROUP, V, LN, false, false, 384>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale, \
+                                                                   absmax_word, stats, stats_are_input, status, st)
+        SQ_PIPE_LN384_ANY(64, 16);   // C <= 8192
+        SQ_PIPE_LN384_ANY(96, 16);   // C <= 12288
+        SQ_PIPE_LN384_ANY(128, 14);  // C <= 14336
+#undef SQ_PIPE_LN384_ANY
+    }
     if (nvec <= 64 * 8) SQ_PIPE(64, 8);      // C <= 4096
     if (nvec <= 64 * 10) SQ_PIPE(64, 10);    // C <= 5120
     if (nvec <= 128 * 8) SQ_PIPE(128, 8);    // C <= 8192   (7168)
