@@ -33,7 +33,7 @@ struct DecCfg {
     static constexpr int STAGE = W_BYTES + X_BYTES;
     static constexpr int STAGES = DN <= 32 ? 10 : 9;
     static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
-    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 4) * 8 + 64;
+    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 4) * 8 + 64 + DN * 4;
 };
 
 struct DecParams {
@@ -65,9 +65,24 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
 }
 __device__ __forceinline__ void dec_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
-// Eq. 2 for one output channel (this thread) and all tokens, then the stores.
+// Per-channel constants of Eq. 2, fetched while the tile's weights are still streaming.
+struct DecChan { float ws, bs, rq; };
+__device__ __forceinline__ DecChan dec_chan(const DecParams& p, int64_t col) {
+    DecChan c = {1.0f, 0.0f, 1.0f};
+    if (col >= p.N || p.out_dt == SQ_I32) return c;
+    if (p.w_scale) c.ws = __ldg(p.w_scale + (p.w_per_col ? col : 0));
+    if (p.bias)
+        c.bs = p.bias_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
+                              : __half2float(static_cast<const __half*>(p.bias)[col]);
+    if (p.requant_mul) c.rq = __ldg(p.requant_mul + (p.requant_per_col ? col : 0));
+    return c;
+}
+
+// Eq. 2 for one output channel (this thread) and all tokens, then the stores.  xs: the tokens'
+// step sizes, staged in shared memory.
 template <int DN>
-__device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&acc)[DN], int64_t col) {
+__device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&acc)[DN], int64_t col, const DecChan& c,
+                                           const float* xs_smem) {
     if (col >= p.N) return;
     if (p.out_dt == SQ_I32) {
         int32_t* y = static_cast<int32_t*>(p.Y);
@@ -76,20 +91,13 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
             if (t < p.M) y[(int64_t)t * p.ldy + col] = acc[t];
         return;
     }
-    const float ws = p.w_scale ? __ldg(p.w_scale + (p.w_per_col ? col : 0)) : 1.0f;
-    float bs = 0.0f;
-    if (p.bias)
-        bs = p.bias_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(p.bias)[col])
-                            : __half2float(static_cast<const __half*>(p.bias)[col]);
-    const float rq = p.requant_mul ? __ldg(p.requant_mul + (p.requant_per_col ? col : 0)) : 1.0f;
 #pragma unroll
     for (int t = 0; t < DN; ++t) {
         if (t < p.M) {
-            const float xs = __ldg(p.x_scale + (p.x_per_row ? t : 0));
-            float v = __fmaf_rn(__int2float_rn(acc[t]), __fmul_rn(xs, ws), bs);
+            float v = __fmaf_rn(__int2float_rn(acc[t]), __fmul_rn(xs_smem[t], c.ws), c.bs);
             if (p.relu) v = fmaxf(v, 0.0f);
             if (p.out_dt == SQ_I8)
-                static_cast<int8_t*>(p.Y)[(int64_t)t * p.ldy + col] = (int8_t)(quant_code(v, rq) & 0xffu);
+                static_cast<int8_t*>(p.Y)[(int64_t)t * p.ldy + col] = (int8_t)(quant_code(v, c.rq) & 0xffu);
             else if (p.out_dt == SQ_BF16)
                 static_cast<__nv_bfloat16*>(p.Y)[(int64_t)t * p.ldy + col] = __float2bfloat16_rn(v);
             else
@@ -114,6 +122,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     volatile uint32_t* abort_flag = tmem_holder + 1;
     volatile uint32_t* epi_go = tmem_holder + 2;
     volatile uint32_t* epi_last = tmem_holder + 3;
+    float* s_xs = reinterpret_cast<float*>(tmem_holder + 4);  // [DN] the tokens' step sizes
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -226,6 +235,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const int quarter = warp & 3;           // TMEM lanes this warp may read
         const int ch = quarter * 32 + lane;     // output channel within the tile
         const int et = threadIdx.x - 64;        // 0..127
+        if (et < DEC_N) s_xs[et] = (et < p.M && p.x_scale) ? __ldg(p.x_scale + (p.x_per_row ? et : 0)) : 1.0f;
+        dec_epi_sync();
         int slot = 0;
         uint32_t slot_phase = 0;
         int64_t pos = (int64_t)blockIdx.x * p.range;
@@ -234,6 +245,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             const int ni = (int)(pos / p.num_kb);
             const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
             pos += kb1 - kb0;
+            const int64_t col = (int64_t)ni * BLOCK_M + ch;
+            const DecChan chan = dec_chan(p, col);  // in flight while the K blocks stream
             if (et == 0) *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 9) ? 1u : 0u;
             dec_epi_sync();
             if (*epi_go == 0u) break;
@@ -252,9 +265,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             slot ^= 1;
             if (slot == 0) slot_phase ^= 1u;
 
-            const int64_t col = (int64_t)ni * BLOCK_M + ch;
             if (kb0 == 0 && kb1 == p.num_kb) {
-                dec_finish<DEC_N>(p, acc, col);  // the whole K range of this tile was ours
+                dec_finish<DEC_N>(p, acc, col, chan, s_xs);  // the whole K range of this tile was ours
             } else {
                 // The tile is shared: CTAs g0 .. g0 + count - 1 each hold one K piece.  Park this
                 // piece in its own slot (plain stores: integer partial sums add exactly in any
@@ -272,13 +284,24 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 dec_epi_sync();
                 if (*epi_last != 0u) {
                     __threadfence();
-                    for (int o = 0; o < count; ++o) {
-                        if (o == mine) continue;
+                    // the other pieces, several at a time so that their loads are in flight together
+                    constexpr int J = DEC_N <= 16 ? 4 : (DEC_N <= 32 ? 2 : 1);
+                    for (int o0 = 0; o0 < count; o0 += J) {
+                        int32_t other[J][DEC_N];
 #pragma unroll
-                        for (int t = 0; t < DEC_N; ++t)
-                            if (t < p.M) acc[t] += __ldcg(slot0 + ((int64_t)o * p.M + t) * BLOCK_M + ch);
+                        for (int j = 0; j < J; ++j) {
+                            const int o = o0 + j;
+                            const bool use = o < count && o != mine;
+#pragma unroll
+                            for (int t = 0; t < DEC_N; ++t)
+                                other[j][t] = (use && t < p.M) ? __ldcg(slot0 + ((int64_t)o * p.M + t) * BLOCK_M + ch) : 0;
+                        }
+#pragma unroll
+                        for (int j = 0; j < J; ++j)
+#pragma unroll
+                            for (int t = 0; t < DEC_N; ++t) acc[t] += other[j][t];
                     }
-                    dec_finish<DEC_N>(p, acc, col);
+                    dec_finish<DEC_N>(p, acc, col, chan, s_xs);
                     if (et == 0) p.counters[ni] = 0u;  // hand the counters back zeroed
                 }
             }
