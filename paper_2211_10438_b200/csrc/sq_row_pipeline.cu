@@ -19,6 +19,12 @@
 // HBM traffic per element), hence the two-wide fp32 instructions (same rounding per half as the
 // scalar ones), the single-FMA rounding, byte-permute packing, vector loads of the reduction
 // partials and multiplications by 1/C in the statistics.
+// Tried and measured no faster: gamma_hat / beta_hat in each thread's own tensor-memory lane
+// (tcgen05.st once, tcgen05.ld one vector ahead), which frees their shared memory for a second
+// ring stage at hidden sizes 8192 to 20480 -- bit-identical output, 0.79 instead of 0.81 of the copy
+// bandwidth at 20480 and 0.82 instead of 0.87 at 12288, so the bytes in flight are not what
+// limits those shapes; 256- and 320-thread CTAs with 128 to 160 values per thread at 20480 (too
+// few warps to cover the reductions); 640 threads with 64 values per thread.
 #include "sq_common.cuh"
 #include "sq_bulk.cuh"
 #include "sq_kernels.h"
