@@ -371,16 +371,18 @@ size_t decode_workspace_bytes(int64_t M, int64_t N) {
 }
 
 // Up to 32 tokens the activation slices are a small addition to the weight stream and this kernel
-// always wins.  At 33..64 tokens they are half as many bytes again, which a single SM's copy
-// rate does not absorb (measured 0.67-0.75 of HBM); the 128 x 256-tile prefill kernel is then
-// faster whenever its N / 256 tiles fill most of the machine, and slower when they do not
-// (N = 12288: 48 tiles, 0.58 against 0.71 here).
+// always wins.  At 33..64 tokens every K block of every tile re-reads 64 x 128 bytes of activations
+// next to its 128 x 128 bytes of weights -- half as many requests again for one SM's copy engine --
+// and the 128 x 256-tile prefill kernel, which reads an activation slice once per 256 output
+// channels, is faster (21504 x 7168: 38 against 50 us; 15360 x 5120: 22 against 33) unless K is
+// so long against N that its few tiles leave most SMs idle (7168 x 28672: 93 against 62 us;
+// 9216 x 36864: 119 against 78), which is where this kernel's even split of the K blocks pays.
 bool decode_supports(const GemmArgs& a) {
     if (!(a.M <= DEC_MAX_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn && a.row_absmax_out == nullptr &&
           a.strideA[2] == a.K && a.strideB[2] == a.K))
         return false;
     if (a.M <= 32) return true;
-    return (a.N + 255) / 256 <= (int64_t)(sm_count() * 2) / 3;
+    return a.K >= 4 * a.N;
 }
 
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st) {

@@ -148,7 +148,8 @@ def test_gemm_last_wave_k_split_is_exact(M, N, K):
 # decode-shaped calls (M <= 16): swapped operands, K splits with INT32 scratch in the workspace
 DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
                  (16, 36864, 1024), (2, 4096, 49152),
-                 (17, 512, 512), (32, 1280, 4096), (33, 200, 272), (64, 12288, 6144), (48, 136, 12288), (64, 36864, 1024)]
+                 (17, 512, 512), (32, 1280, 4096), (33, 200, 272), (64, 12288, 6144), (48, 136, 12288), (64, 36864, 1024),
+                 (64, 1024, 8192), (40, 520, 4096), (64, 1536, 6144)]  # 33..64 tokens stay on this kernel when K >= 4 N
 
 
 @pytest.mark.parametrize("M,N,K", DECODE_SHAPES)
