@@ -223,11 +223,12 @@ sq_status sq_ln_quant_tensor_noalloc(const void* X, sq_dtype dt, int64_t M, int6
  * before output rounding) via atomic max, so that the next layer's per-token step size
  * needs no extra pass.  Y: [M, N] with row stride ldy elements.
  * workspace: word 0 is the device status.  sq_workspace_bytes(SQ_OP_GEMM, M, N, K) bytes are
- * REQUIRED for M <= 64 (the weight-streaming kernel parks partial sums there) and RECOMMENDED
- * above: when the tile count does not fill the last wave of thread-block groups, the tiles of
- * that wave are cut along K and their INT32 partial sums meet in the workspace (integer sums:
- * the result does not depend on it).  With a smaller workspace (>= 256 bytes) the cut is not
- * made and the call is merely slower.
+ * REQUIRED for M <= 32 (the weight-streaming kernel parks partial sums there) and RECOMMENDED
+ * above: when the tiles do not fill the last wave of thread-block groups (or, with few tokens
+ * against a narrow weight, fill at most half of the only wave), the tiles of that wave are cut
+ * along K and their INT32 partial sums meet in the workspace (integer sums: the result does not
+ * depend on it).  With a smaller workspace (>= 256 bytes) the cut is not made and the call is
+ * merely slower.
  */
 sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
                        const float* x_scale, int x_scale_is_per_token, const float* w_scale,

@@ -1,5 +1,7 @@
 // extern "C" entry points of libsq: argument validation and kernel dispatch only.
 #include "sq_common.cuh"
+#include <algorithm>
+
 #include "sq_kernels.h"
 
 using namespace sq;
@@ -64,8 +66,9 @@ size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K) {
     switch (op) {
         case SQ_OP_LN_QUANT: return kWsHeader + (size_t)(M > 0 ? M : 0) * 2 * sizeof(float);
         case SQ_OP_GEMM:  // decode-shaped calls keep split-K partial sums in the workspace
-            if (M > 0 && M <= 64 && N > 0) return decode_workspace_bytes(M, N);
-            return (M > 0 && N > 0 && K > 0) ? gemm_workspace_bytes(M, N, K) : kWsHeader;
+            if (!(M > 0 && N > 0 && K > 0)) return kWsHeader;
+            if (M <= 32) return decode_workspace_bytes(M, N);
+            return gemm_workspace_bytes(M, N, K);
         case SQ_OP_QUANT_ACT:
         case SQ_OP_QUANT_WEIGHT:
         case SQ_OP_BMM: return kWsHeader;
@@ -183,7 +186,7 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
     if (bias && !is_act_dtype(bias_dt)) return SQ_ERR_INVALID_ARG;
     if (K % 16 != 0 || !aligned16(Xq) || !aligned16(Wq)) return SQ_ERR_ALIGN;
     // decode-shaped calls need their scratch; a prefill GEMM only uses what it is given (see sq.h)
-    if (!ws_ok(workspace, ws_bytes, M <= 64 ? sq_workspace_bytes(SQ_OP_GEMM, M, N, K) : kWsHeader)) return SQ_ERR_WORKSPACE;
+    if (!ws_ok(workspace, ws_bytes, M <= 32 ? sq_workspace_bytes(SQ_OP_GEMM, M, N, K) : kWsHeader)) return SQ_ERR_WORKSPACE;
     GemmArgs a{};
     a.ws_bytes = ws_bytes;
     a.A = Xq; a.B = Wq;

@@ -1,9 +1,9 @@
-// Decode-shaped W8A8 linear (M <= 16 tokens): the weight matrix is streamed once from HBM and
+// Decode-shaped W8A8 linear (M <= 32 tokens): the weight matrix is streamed once from HBM and
 // everything else is noise, so the kernel is laid out around that stream.
 //
 //   * operands are swapped: 128 OUTPUT CHANNELS of W (128 x 128 bytes per K slice) ride on the
-//     MMA's M dimension and the <= 16 tokens on its N dimension (tcgen05.mma.kind::i8,
-//     128 x 16 x 32), so no tile is padded from 16 to 128 rows and a stage is 18 KB;
+//     MMA's M dimension and the tokens on its N dimension (tcgen05.mma.kind::i8, 128 x 16 x 32
+//     or 128 x 32 x 32), so no tile is padded from 16 to 128 rows and a stage is 18 or 20 KB;
 //   * the (128-channel tile, K block) pairs, tile-major, are cut into equal contiguous ranges,
 //     one per CTA ("stream-K"): every SM streams the same number of weight bytes whatever N
 //     and K are, at the price of tiles whose K range is shared by two or more CTAs;
@@ -23,15 +23,15 @@ namespace {
 using namespace tc;
 
 constexpr int DEC_THREADS = 192;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
-constexpr int DEC_MAX_N = 64;         // most tokens this kernel takes
+constexpr int DEC_MAX_N = 32;         // most tokens this kernel takes
 constexpr int W_BYTES = BLOCK_M * BLOCK_K;  // 16 KB of weights per stage
-// DN = tokens per MMA (its N dimension): 16, 32 or 64.  A stage holds 16 KB of weights and
-// DN * 128 bytes of activations; the ring is as deep as shared memory allows (10 / 10 / 9 stages).
+// DN = tokens per MMA (its N dimension): 16 or 32.  A stage holds 16 KB of weights and
+// DN * 128 bytes of activations; the ring is as deep as shared memory allows (10 stages).
 template <int DN>
 struct DecCfg {
     static constexpr int X_BYTES = DN * BLOCK_K;
     static constexpr int STAGE = W_BYTES + X_BYTES;
-    static constexpr int STAGES = DN <= 32 ? 10 : 9;
+    static constexpr int STAGES = 10;
     static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
     static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 4) * 8 + 64 + DN * 4;
 };
@@ -285,7 +285,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 if (*epi_last != 0u) {
                     __threadfence();
                     // the other pieces, several at a time so that their loads are in flight together
-                    constexpr int J = DEC_N <= 16 ? 4 : (DEC_N <= 32 ? 2 : 1);
+                    constexpr int J = DEC_N <= 16 ? 4 : 2;
                     for (int o0 = 0; o0 < count; o0 += J) {
                         int32_t other[J][DEC_N];
 #pragma unroll
@@ -371,18 +371,14 @@ size_t decode_workspace_bytes(int64_t M, int64_t N) {
 }
 
 // Up to 32 tokens the activation slices are a small addition to the weight stream and this kernel
-// always wins.  At 33..64 tokens every K block of every tile re-reads 64 x 128 bytes of activations
-// next to its 128 x 128 bytes of weights -- half as many requests again for one SM's copy engine --
-// and the 128 x 256-tile prefill kernel, which reads an activation slice once per 256 output
-// channels, is faster (21504 x 7168: 38 against 50 us; 15360 x 5120: 22 against 33) unless K is
-// so long against N that its few tiles leave most SMs idle (7168 x 28672: 93 against 62 us;
-// 9216 x 36864: 119 against 78), which is where this kernel's even split of the K blocks pays.
+// wins.  Beyond, every K block of every tile would re-read 64 x 128 bytes of activations next to
+// its 128 x 128 bytes of weights -- half as many requests again for one SM's copy engine -- and a
+// 64-token instantiation measured slower than the prefill kernel on every shape once that kernel
+// cut a sparsely filled wave along K and took 128-channel tiles (7168 x 28672, 64 tokens: 62 us
+// here, 47 us there; 21504 x 7168: 50 against 38), so it is not built.
 bool decode_supports(const GemmArgs& a) {
-    if (!(a.M <= DEC_MAX_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn && a.row_absmax_out == nullptr &&
-          a.strideA[2] == a.K && a.strideB[2] == a.K))
-        return false;
-    if (a.M <= 32) return true;
-    return a.K >= 4 * a.N;
+    return a.M <= DEC_MAX_N && a.batch == 1 && a.heads == 1 && !a.b_is_kn && a.row_absmax_out == nullptr &&
+           a.strideA[2] == a.K && a.strideB[2] == a.K;
 }
 
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st) {
@@ -405,8 +401,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.part = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader + kDecCounterBytes);
     p.status = a.status;
     if (a.M <= 16) return launch_decode<16>(a, p, plan.ctas, st);
-    if (a.M <= 32) return launch_decode<32>(a, p, plan.ctas, st);
-    return launch_decode<64>(a, p, plan.ctas, st);
+    return launch_decode<32>(a, p, plan.ctas, st);
 }
 
 }  // namespace sq

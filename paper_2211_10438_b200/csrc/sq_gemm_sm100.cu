@@ -535,12 +535,27 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // reductions only (a 256 x 256 tile of K = 20480 takes 66 us: 156 -> 144 us on 2048 x 5120 x 20480,
 // 291 -> 271 us on 2048 x 7168 x 28672), loses for K = 5120 (tile 16 us) at every s, and loses badly
 // when the pieces need more than one round.  Hence: K >= 12288, s in {4, 3, 2} with R * s <= G
-// and at least 16 K blocks per piece.
+// and at least 16 K blocks per piece; and, when all tiles together fill at most half of the
+// groups, every tile is cut into up to 8 pieces of at least 8 K blocks.
 struct SplitPlan { uint32_t full; int split; int kb_per_piece; };
 inline SplitPlan plan_split(int64_t total_tiles, int num_kb, int groups, int64_t K, int tile_m, int tile_n) {
     SplitPlan pl{(uint32_t)total_tiles, 1, num_kb};
     (void)tile_m; (void)tile_n;
-    if (groups <= 0 || total_tiles <= 0 || K < 12288) return pl;
+    if (groups <= 0 || total_tiles <= 0) return pl;
+    if (K < 12288) return pl;
+    if (2 * total_tiles <= groups) {
+        // a single wave that fills at most half of the machine (few tokens against a narrow weight):
+        // every tile is cut (7168 x 28672, 128 tokens: 92 -> 60 us with 128 x 256 tiles)
+        for (int s = (int)std::min<int64_t>(8, groups / total_tiles); s >= 2; --s) {
+            const int per = (num_kb + s - 1) / s;
+            if (per < 8 || (num_kb + per - 1) / per != s) continue;
+            pl.split = s;
+            pl.kb_per_piece = per;
+            pl.full = 0;
+            return pl;
+        }
+        return pl;
+    }
     const int64_t R = total_tiles % groups;
     if (R == 0) return pl;
     for (int s = 4; s >= 2; --s) {
@@ -675,13 +690,23 @@ sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t 
     return launch_status();
 }
 
+static bool narrow_single_row_tiles(int64_t N) { return (N + 127) / 128 <= (int64_t)sm_count(); }
+
 // Scratch a plain GEMM of this shape can use for the K split of its last wave (the tile
 // configuration follows gemm_i8's dispatch); with less the split is simply not taken.
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-    if (M <= 128 || N <= 128 || K <= 1024) return kWsHeader;  // only the CTA-pair configuration splits
+    if (N <= 128 || K <= 1024) return kWsHeader;  // those configurations never split
+    const int num_kb = (int)((K + BLOCK_K - 1) / BLOCK_K);
+    if (M <= 128) {  // single CTAs, one row of 128 x 128 or 128 x 256 tiles
+        if (narrow_single_row_tiles(N)) {
+            const int64_t tiles = (N + 127) / 128;
+            return split_workspace_bytes<128, 1>(plan_split(tiles, num_kb, sm_count(), K, BLOCK_M, 128), tiles);
+        }
+        const int64_t tiles = (N + 255) / 256;
+        return split_workspace_bytes<256, 1>(plan_split(tiles, num_kb, sm_count(), K, BLOCK_M, 256), tiles);
+    }
     const int64_t tiles = ((M + 2 * BLOCK_M - 1) / (2 * BLOCK_M)) * ((N + 255) / 256);
     if (tiles >= (int64_t)1 << 31) return kWsHeader;
-    const int num_kb = (int)((K + BLOCK_K - 1) / BLOCK_K);
     const SplitPlan pl = plan_split(tiles, num_kb, sm_count() / 2, K, 2 * BLOCK_M, 256);
     return split_workspace_bytes<256, 2>(pl, tiles);
 }
@@ -690,7 +715,10 @@ sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
     if (decode_supports(a)) return decode_gemm(a, a.status, a.ws_bytes, st);
     // [K, N]-stored B is limited to one 128-byte swizzle row of N per tile
     if (a.b_is_kn || a.N <= 128) return launch<128, 1>(a, st);
-    if (a.M <= 128) return launch<256, 1>(a, st);
+    // Up to 128 tokens every tile is one row of tiles: 128 output channels per tile instead of 256
+    // whenever those still fit one wave (N <= 128 * SMs), so that twice as many SMs stream weights
+    // (12288 x 12288, 128 tokens: 46 -> 35 us; 15360 x 5120: 22 -> 18 us).
+    if (a.M <= 128) return narrow_single_row_tiles(a.N) ? launch<128, 1>(a, st) : launch<256, 1>(a, st);
     // CTA pairs with 256 x 256 tiles.  Narrower pair tiles (192, 128 columns) were measured: they
     // even out the last wave of some shapes but move more operand bytes per MAC and lose overall.
     return launch<256, 2>(a, st);

@@ -38,7 +38,7 @@ def decode_gemm(args):
     N, K = args.N, args.K
     Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device="cuda", generator=g)
     w_scale = torch.rand(N, device="cuda", generator=g) * 1e-3
-    ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 64, N, K))
+    ws = sq.new_workspace(max(sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K) for M in args.M))
     for M in args.M:
         X = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda", generator=g)
         xs = torch.rand(M, device="cuda", generator=g)

@@ -15,7 +15,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module")
 def ws():
-    w = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, 64, 65536, 32768))  # decode scratch is the largest
+    # the largest scratch any shape below asks for: the weight-streaming kernel's at 32 tokens, the K split's above
+    w = sq.new_workspace(max(sq.workspace_bytes(sq.SQ_OP_GEMM, 32, 65536, 32768), 64 << 20))
     yield w
     assert sq.device_status(w) == 0, "a device-side wait timed out"
 
@@ -121,7 +122,11 @@ def test_gemm_strided_output(ws):
 # long reductions whose tile count leaves a partly filled last wave: with the recommended workspace
 # the tiles of that wave are cut along K (2 .. 4 pieces) and meet in the workspace; without it they are not
 SPLIT_SHAPES = [(512, 4096, 12288), (2048, 5120, 20480), (300, 2304, 16400), (2048, 7168, 28672), (520, 1000, 12304),
-                (256, 20480, 12288)]
+                (256, 20480, 12288),
+                # a single wave filling at most half of the machine: every tile cut into up to 8 pieces
+                # (one row of 128 x 128 tiles up to 128 tokens, CTA pairs above)
+                (96, 2048, 12288), (128, 3000, 13008), (70, 7168, 14336), (128, 20480, 12288), (256, 7168, 14336),
+                (65, 4096, 12288)]
 
 
 @pytest.mark.parametrize("M,N,K", SPLIT_SHAPES)
@@ -145,11 +150,11 @@ def test_gemm_last_wave_k_split_is_exact(M, N, K):
     assert not big[4:33024].any(), "header and counters not handed back zero-filled"
 
 
-# decode-shaped calls (M <= 16): swapped operands, K splits with INT32 scratch in the workspace
+# decode-shaped calls: swapped operands and K splits with INT32 scratch in the workspace up to 32 tokens
 DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
                  (16, 36864, 1024), (2, 4096, 49152),
                  (17, 512, 512), (32, 1280, 4096), (33, 200, 272), (64, 12288, 6144), (48, 136, 12288), (64, 36864, 1024),
-                 (64, 1024, 8192), (40, 520, 4096), (64, 1536, 6144)]  # 33..64 tokens stay on this kernel when K >= 4 N
+                 (64, 1024, 8192), (40, 520, 4096), (64, 1536, 6144)]  # above 32 tokens: the prefill kernel, narrow tiles
 
 
 @pytest.mark.parametrize("M,N,K", DECODE_SHAPES)
