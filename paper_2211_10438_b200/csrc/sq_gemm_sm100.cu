@@ -537,6 +537,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // when the pieces need more than one round.  Hence: K >= 12288, s in {4, 3, 2} with R * s <= G
 // and at least 16 K blocks per piece; and, when all tiles together fill at most half of the
 // groups, every tile is cut into up to 8 pieces of at least 8 K blocks.
+// Also tried for K < 12288: equal contiguous ranges of (tile, K block) pairs per group ("stream-K",
+// at most two owners per tile).  Bit-exact, but slower wherever it applied (2048 x 21504 x 7168:
+// 204 -> 275 us; 256 x 21504 x 7168: 49 -> 54 us): groups that run side by side then work on tiles
+// far apart in the visiting order, so the weight tiles they stream no longer coincide in L2 (74
+// pairs x 1.8 MB live at once), and with few tokens a partly filled wave already runs faster per
+// tile because one SM's copy rate, not HBM, is the limit there.
 struct SplitPlan { uint32_t full; int split; int kb_per_piece; };
 inline SplitPlan plan_split(int64_t total_tiles, int num_kb, int groups, int64_t K, int tile_m, int tile_n) {
     SplitPlan pl{(uint32_t)total_tiles, 1, num_kb};
