@@ -238,6 +238,23 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
                        void* workspace, size_t ws_bytes, void* stream);
 
 /*
+ * The same W8A8 linear with the block's residual connection folded into its epilogue (Fig. 6
+ * keeps the residual stream in FP16; the two linears that feed it are out-proj and FC2):
+ *     y[t, o]  = round_to(out_dt)(fma((float)acc[t, o], Delta_x * Delta_w, bias[o]))   as above
+ *     Y[t, o]  = round_to(out_dt)((float)y[t, o] + (float)residual[t, o])
+ * i.e. bit for bit what sq_w8a8_gemm followed by sq_residual_add gives, without writing y and
+ * reading it back.  out_dt: SQ_F16 or SQ_BF16; residual: [M, N] of that type, row stride ld_res
+ * elements (>= N, a multiple of 8), 16-byte aligned, N a multiple of 8; must not overlap Y.  No
+ * activation function, no re-quantisation, no row_absmax_out.  Other arguments, workspace and
+ * errors as for sq_w8a8_gemm.
+ */
+sq_status sq_w8a8_gemm_residual(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
+                                const float* x_scale, int x_scale_is_per_token, const float* w_scale,
+                                int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt,
+                                const void* residual, int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy,
+                                void* workspace, size_t ws_bytes, void* stream);
+
+/*
  * INT8 batched matmul for attention (Fig. 6: the BMMs run in INT8):
  * for every b < batch, h < heads
  *     acc = A[b,h] * B[b,h]^T   (B stored [N, K], K contiguous;  b_is_kn == 0)   e.g. Q.K^T

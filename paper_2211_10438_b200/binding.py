@@ -25,7 +25,7 @@ SQ_MAX_K = 133144
 SQ_NOALLOC_MAX_ROWS = 16384
 
 EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_scales",
-           "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm",
+           "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm", "sq_w8a8_gemm_residual",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
            "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention",
            "sq_token_absmax", "sq_clipped_absmax"]
@@ -66,6 +66,8 @@ def lib():
         L.sq_ln_quant.argtypes = [vp, i32, i64, i64, vp, vp, f32, i32, vp, vp, vp, vp, sz, vp]
         L.sq_w8a8_gemm.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, i32, vp, i32, i32, vp, i32, vp,
                                    vp, i32, i64, vp, sz, vp]
+        L.sq_w8a8_gemm_residual.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, i32, vp, i32, vp, i64, vp, i32, i64,
+                                            vp, sz, vp]
         L.sq_w8a8_bmm.argtypes = [vp, vp, i64, i64, i64, i64, i64, c.POINTER(i64), c.POINTER(i64), i32, i32,
                                   f32, vp, vp, i32, c.POINTER(i64), vp, sz, vp]
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
@@ -209,6 +211,21 @@ def sq_w8a8_gemm(Xq, Wq, x_scale, w_scale, workspace, bias=None, relu=False, req
         _DT[bias.dtype] if bias is not None else SQ_F16, SQ_EPI_RELU if relu else SQ_EPI_NONE,
         _ptr(requant_mul), 1 if (requant_mul is not None and requant_mul.numel() > 1) else 0,
         _ptr(row_absmax_out), _ptr(out), _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_gemm")
+    return out
+
+
+def sq_w8a8_gemm_residual(Xq, Wq, x_scale, w_scale, workspace, residual, bias=None, out=None):
+    """The W8A8 linear plus the residual stream: out = round(round(y) + residual), out dtype = residual's."""
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=residual.dtype, device=Xq.device)
+    wp, wn = _ws(workspace)
+    _check(lib().sq_w8a8_gemm_residual(
+        _ptr(Xq), _ptr(Wq), M, N, K, _ptr(x_scale), 1 if (x_scale is not None and x_scale.numel() > 1) else 0,
+        _ptr(w_scale), 1 if (w_scale is not None and w_scale.numel() > 1) else 0, _ptr(bias),
+        _DT[bias.dtype] if bias is not None else SQ_F16, _ptr(residual), residual.stride(0),
+        _ptr(out), _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_gemm_residual")
     return out
 
 

@@ -169,11 +169,13 @@ sq_status sq_ln_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const vo
                              as_stream(stream));
 }
 
-sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
-                       const float* x_scale, int x_scale_is_per_token, const float* w_scale,
-                       int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt, sq_epilogue_act act,
-                       const float* requant_mul, int requant_is_per_channel, float* row_absmax_out, void* Y,
-                       sq_dtype out_dt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+static sq_status w8a8_gemm_impl(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K, const float* x_scale,
+                                int x_scale_is_per_token, const float* w_scale, int w_scale_is_per_channel,
+                                const void* bias, sq_dtype bias_dt, sq_epilogue_act act, const float* requant_mul,
+                                int requant_is_per_channel, float* row_absmax_out, const void* residual,
+                                int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy, void* workspace,
+                                size_t ws_bytes, void* stream) {
+
     if (M < 0 || N < 0 || K < 0) return SQ_ERR_SHAPE;
     if (out_dt < SQ_F16 || out_dt > SQ_I32 || (act != SQ_EPI_NONE && act != SQ_EPI_RELU)) return SQ_ERR_INVALID_ARG;
     if (M == 0 || N == 0) return SQ_OK;
@@ -185,6 +187,11 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
     if ((out_dt == SQ_I8) != (requant_mul != nullptr)) return SQ_ERR_INVALID_ARG;
     if (bias && !is_act_dtype(bias_dt)) return SQ_ERR_INVALID_ARG;
     if (K % 16 != 0 || !aligned16(Xq) || !aligned16(Wq)) return SQ_ERR_ALIGN;
+    if (residual) {  // the residual stream has the output's 16-bit type and is read in 16-byte pieces
+        if (!is_act_dtype(out_dt) || row_absmax_out) return SQ_ERR_INVALID_ARG;
+        if (ld_res < N) return SQ_ERR_SHAPE;
+        if (!aligned16(residual) || ld_res % 8 != 0 || N % 8 != 0) return SQ_ERR_ALIGN;
+    }
     // decode-shaped calls need their scratch; a prefill GEMM only uses what it is given (see sq.h)
     if (!ws_ok(workspace, ws_bytes, M <= 32 ? sq_workspace_bytes(SQ_OP_GEMM, M, N, K) : kWsHeader)) return SQ_ERR_WORKSPACE;
     GemmArgs a{};
@@ -201,10 +208,32 @@ sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N,
     a.relu = act == SQ_EPI_RELU;
     a.requant_mul = requant_mul; a.requant_per_col = requant_is_per_channel;
     a.row_absmax_out = row_absmax_out;
+    a.residual = residual; a.ld_res = ld_res;
     a.C = Y; a.out_dt = out_dt;
     a.strideC[0] = 0; a.strideC[1] = 0; a.strideC[2] = ldy;
     a.status = reinterpret_cast<uint32_t*>(workspace);
     return gemm_i8(a, as_stream(stream));
+}
+
+sq_status sq_w8a8_gemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
+                       const float* x_scale, int x_scale_is_per_token, const float* w_scale,
+                       int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt,
+                       sq_epilogue_act act, const float* requant_mul, int requant_is_per_channel,
+                       float* row_absmax_out, void* Y, sq_dtype out_dt, int64_t ldy,
+                       void* workspace, size_t ws_bytes, void* stream) {
+    return w8a8_gemm_impl(Xq, Wq, M, N, K, x_scale, x_scale_is_per_token, w_scale, w_scale_is_per_channel, bias, bias_dt,
+                          act, requant_mul, requant_is_per_channel, row_absmax_out, nullptr, 0, Y, out_dt, ldy,
+                          workspace, ws_bytes, stream);
+}
+
+sq_status sq_w8a8_gemm_residual(const int8_t* Xq, const int8_t* Wq, int64_t M, int64_t N, int64_t K,
+                                const float* x_scale, int x_scale_is_per_token, const float* w_scale,
+                                int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt,
+                                const void* residual, int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy,
+                                void* workspace, size_t ws_bytes, void* stream) {
+    if (!residual) return SQ_ERR_INVALID_ARG;
+    return w8a8_gemm_impl(Xq, Wq, M, N, K, x_scale, x_scale_is_per_token, w_scale, w_scale_is_per_channel, bias, bias_dt,
+                          SQ_EPI_NONE, nullptr, 0, nullptr, residual, ld_res, Y, out_dt, ldy, workspace, ws_bytes, stream);
 }
 
 sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M, int64_t N,

@@ -51,6 +51,8 @@ struct DecParams {
     void* Y; int out_dt; int64_t ldy;
     int32_t* part;       // [num_n][maxcount][M][128] partial sums of tiles shared by several CTAs
     uint32_t* counters;  // [num_n] arrivals per shared tile, zero on entry and on exit
+    const void* residual;  // nullable: [M, N] of the output type, row stride ld_res
+    int64_t ld_res;
     uint32_t* status;
 };
 
@@ -80,9 +82,20 @@ __device__ __forceinline__ DecChan dec_chan(const DecParams& p, int64_t col) {
 
 // Eq. 2 for one output channel (this thread) and all tokens, then the stores.  xs: the tokens'
 // step sizes, staged in shared memory.
+// The residual elements of one output channel, all tokens (16-bit bit patterns).  Fetched with the
+// per-channel constants, before the accumulators are waited for: in the last arriver's tail a
+// demand load would wait microseconds behind the other CTAs' weight streams.
+template <int DN>
+__device__ __forceinline__ void dec_residual(const DecParams& p, int64_t col, uint16_t (&res)[DN]) {
+#pragma unroll
+    for (int t = 0; t < DN; ++t)
+        res[t] = (p.residual && t < p.M && col < p.N)
+                     ? __ldg(static_cast<const uint16_t*>(p.residual) + (int64_t)t * p.ld_res + col) : (uint16_t)0;
+}
+
 template <int DN>
 __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&acc)[DN], int64_t col, const DecChan& c,
-                                           const float* xs_smem) {
+                                           const float* xs_smem, const uint16_t (&res)[DN]) {
     if (col >= p.N) return;
     if (p.out_dt == SQ_I32) {
         int32_t* y = static_cast<int32_t*>(p.Y);
@@ -96,6 +109,11 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
         if (t < p.M) {
             float v = __fmaf_rn(__int2float_rn(acc[t]), __fmul_rn(xs_smem[t], c.ws), c.bs);
             if (p.relu) v = fmaxf(v, 0.0f);
+            if (p.residual) {  // round to the output type, then the residual add (rounded by the store below)
+                v = p.out_dt == SQ_BF16
+                        ? __bfloat162float(__float2bfloat16_rn(v)) + __uint_as_float((uint32_t)res[t] << 16)
+                        : __half2float(__float2half_rn(v)) + __half2float(__ushort_as_half(res[t]));
+            }
             if (p.out_dt == SQ_I8)
                 static_cast<int8_t*>(p.Y)[(int64_t)t * p.ldy + col] = (int8_t)(quant_code(v, c.rq) & 0xffu);
             else if (p.out_dt == SQ_BF16)
@@ -247,6 +265,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             pos += kb1 - kb0;
             const int64_t col = (int64_t)ni * BLOCK_M + ch;
             const DecChan chan = dec_chan(p, col);  // in flight while the K blocks stream
+            uint16_t res[DEC_N];
+            dec_residual<DEC_N>(p, col, res);
             if (et == 0) *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 9) ? 1u : 0u;
             dec_epi_sync();
             if (*epi_go == 0u) break;
@@ -266,7 +286,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             if (slot == 0) slot_phase ^= 1u;
 
             if (kb0 == 0 && kb1 == p.num_kb) {
-                dec_finish<DEC_N>(p, acc, col, chan, s_xs);  // the whole K range of this tile was ours
+                dec_finish<DEC_N>(p, acc, col, chan, s_xs, res);  // the whole K range of this tile was ours
             } else {
                 // The tile is shared: CTAs g0 .. g0 + count - 1 each hold one K piece.  Park this
                 // piece in its own slot (plain stores: integer partial sums add exactly in any
@@ -301,7 +321,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
 #pragma unroll
                             for (int t = 0; t < DEC_N; ++t) acc[t] += other[j][t];
                     }
-                    dec_finish<DEC_N>(p, acc, col, chan, s_xs);
+                    dec_finish<DEC_N>(p, acc, col, chan, s_xs, res);
                     if (et == 0) p.counters[ni] = 0u;  // hand the counters back zeroed
                 }
             }
@@ -397,6 +417,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.relu = a.relu;
     p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
     p.Y = a.C; p.out_dt = (int)a.out_dt; p.ldy = a.strideC[2];
+    p.residual = a.residual; p.ld_res = a.ld_res;
     p.counters = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsHeader);
     p.part = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader + kDecCounterBytes);
     p.status = a.status;

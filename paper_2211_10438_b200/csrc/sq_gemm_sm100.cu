@@ -69,6 +69,7 @@ struct Params {
     int relu;
     const float* requant_mul; int requant_per_col;
     float* row_absmax_out;
+    const void* residual; int64_t ld_res;  // [M, N] of the output type, added after the output rounding (plain GEMMs)
     void* C; int out_dt;
     int64_t c_stride_batch, c_stride_head, c_stride_row;
     int c_tma;  // C leaves through TMA stores (needs 16-byte aligned base and strides)
@@ -143,7 +144,7 @@ __device__ __forceinline__ int tile_num_kb(const Params& p, int mi, int tile_m) 
 // ------------------------------------------------------------------------------------
 // FIX: this CTA arrived last for a K-split tile: the other pieces' partial sums (fix_count slots,
 // fix_stride ints apart, fix_base already at this thread's row) are added to the accumulators first.
-template <int BLOCK_N, bool FIX = false>
+template <int BLOCK_N, bool FIX = false, bool EW8 = false>
 __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
                                               uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
                                               int h, int64_t c_off, const float* s_wscale,
@@ -211,6 +212,30 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                 for (int j = 0; j < 32; ++j)
                     if (j < ncols) row_max = fmaxf(row_max, fabsf(y[j]));
             }
+            if (p.residual && !p.c_tma) {
+                // the block's residual connection: round y to the output type first, then add the
+                // residual element in fp32 (the final rounding below is the 16-bit add's rounding)
+                const uint4* rrow = reinterpret_cast<const uint4*>(
+                    static_cast<const uint16_t*>(p.residual) + (row_ok ? row : 0) * p.ld_res + col0 + cc * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    if (row_ok && 8 * v < ncols) {  // N is a multiple of 8: whole vectors only
+                        const uint4 rv = __ldg(rrow + v);
+                        float rf[8];
+                        if (p.out_dt == SQ_BF16) {
+                            unpack8<__nv_bfloat16>(rv, rf);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                y[8 * v + k] = __bfloat162float(__float2bfloat16_rn(y[8 * v + k])) + rf[k];
+                        } else {
+                            unpack8<__half>(rv, rf);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                y[8 * v + k] = __half2float(__float2half_rn(y[8 * v + k])) + rf[k];
+                        }
+                    }
+                }
+            }
             if (p.out_dt == SQ_I8) {
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
@@ -253,9 +278,58 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                 }
             }
             if (sub == chunks_per_store - 1) {
+                const int64_t gcol = col0 + (int64_t)(cc - sub) * 32;  // first column of the staged group
+                if (p.residual) {
+                    // The residual connection, on the staged tile (32 rows x 64 rounded outputs): the
+                    // warp walks it in the layout of the global rows -- 8 lanes per row, 16 bytes per
+                    // lane -- so that the residual arrives in whole 128-byte lines, adds in fp32 and
+                    // rounds again (the 16-bit add's rounding).
+                    __syncwarp();
+                    const int piece_c = lane & 7;
+                    const int64_t rcol = gcol + piece_c * 8;
+                    constexpr int RB = EW8 ? 4 : 8;  // loads in flight per batch (register budget)
+#pragma unroll 1
+                    for (int i0 = 0; i0 < 8; i0 += RB) {
+                    uint4 rv[RB];
+#pragma unroll
+                    for (int i = 0; i < RB; ++i) {
+                        const int64_t rr = (int64_t)row0_warp + 4 * (i0 + i) + (lane >> 3);
+                        rv[i] = (rr < p.M && rcol < p.N)  // N is a multiple of 8: whole vectors only
+                                    ? __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.residual) +
+                                                                           rr * p.ld_res + rcol))
+                                    : make_uint4(0u, 0u, 0u, 0u);
+                    }
+#pragma unroll
+                    for (int i = 0; i < RB; ++i) {
+                        const int r = 4 * (i0 + i) + (lane >> 3);
+                        uint4* cell = reinterpret_cast<uint4*>(buf + r * 128 + ((piece_c ^ (r & 7)) << 4));
+                        float a[8], b[8];
+                        uint4 o;
+                        if (p.out_dt == SQ_BF16) {
+                            unpack8<__nv_bfloat16>(*cell, a);
+                            unpack8<__nv_bfloat16>(rv[i], b);
+                            __nv_bfloat162 t0 = __halves2bfloat162(__float2bfloat16_rn(a[0] + b[0]), __float2bfloat16_rn(a[1] + b[1]));
+                            __nv_bfloat162 t1 = __halves2bfloat162(__float2bfloat16_rn(a[2] + b[2]), __float2bfloat16_rn(a[3] + b[3]));
+                            __nv_bfloat162 t2 = __halves2bfloat162(__float2bfloat16_rn(a[4] + b[4]), __float2bfloat16_rn(a[5] + b[5]));
+                            __nv_bfloat162 t3 = __halves2bfloat162(__float2bfloat16_rn(a[6] + b[6]), __float2bfloat16_rn(a[7] + b[7]));
+                            o = make_uint4(*reinterpret_cast<uint32_t*>(&t0), *reinterpret_cast<uint32_t*>(&t1),
+                                           *reinterpret_cast<uint32_t*>(&t2), *reinterpret_cast<uint32_t*>(&t3));
+                        } else {
+                            unpack8<__half>(*cell, a);
+                            unpack8<__half>(rv[i], b);
+                            __half2 t0 = __halves2half2(__float2half_rn(a[0] + b[0]), __float2half_rn(a[1] + b[1]));
+                            __half2 t1 = __halves2half2(__float2half_rn(a[2] + b[2]), __float2half_rn(a[3] + b[3]));
+                            __half2 t2 = __halves2half2(__float2half_rn(a[4] + b[4]), __float2half_rn(a[5] + b[5]));
+                            __half2 t3 = __halves2half2(__float2half_rn(a[6] + b[6]), __float2half_rn(a[7] + b[7]));
+                            o = make_uint4(*reinterpret_cast<uint32_t*>(&t0), *reinterpret_cast<uint32_t*>(&t1),
+                                           *reinterpret_cast<uint32_t*>(&t2), *reinterpret_cast<uint32_t*>(&t3));
+                        }
+                        *cell = o;
+                    }
+                    }
+                }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> async proxy
                 __syncwarp();
-                const int64_t gcol = col0 + (int64_t)(cc - sub) * 32;  // first column of the staged group
                 if (lane == 0 && gcol < p.N && row0_warp < p.M) {
                     cc_coord[0] = (int)gcol;
                     tma_store_4d(tmap_c, buf, cc_coord[0], cc_coord[1], cc_coord[2], cc_coord[3]);
@@ -452,6 +526,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
                 s_wscale[c] = ws; s_bias[c] = bs; s_requant[c] = rq;
             }
+            if (p.residual) {
+                // pull this thread's row of the residual tile into L2 while the tile's MMAs still run:
+                // under a saturated memory system a demand load in the epilogue waits microseconds
+                const int64_t prow = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
+                if (prow < p.M) {
+                    const char* base = reinterpret_cast<const char*>(static_cast<const uint16_t*>(p.residual) + prow * p.ld_res + col0);
+                    const int64_t bytes = 2 * min((int64_t)BLOCK_N, p.N - col0);
+                    for (int64_t off = half * 128; off < bytes; off += (EW == 8 ? 256 : 128))
+                        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
+                }
+            }
             if (et == 0)
                 *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 4) ? 1u : 0u;
             epi_bar_sync<C::EPI_THREADS>();  // constants staged; outcome of the wait visible to all epilogue threads
@@ -471,7 +556,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int cc_begin = half == 0 ? 0 : g_split * cps;
             const int cc_end = half == 0 ? min(g_split * cps, BLOCK_N / 32) : BLOCK_N / 32;
             if (EW == 8 || piece < 0) {  // (the eight-warp configuration serves short reductions: never split)
-                epilogue_slot<BLOCK_N>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
+                epilogue_slot<BLOCK_N, false, EW == 8>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
                                        c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
             } else {
                 // K piece of a split tile: park the accumulators, then see who is last
@@ -626,6 +711,7 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     p.relu = a.relu;
     p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
     p.row_absmax_out = a.row_absmax_out;
+    p.residual = a.residual; p.ld_res = a.ld_res;
     p.C = a.C; p.out_dt = (int)a.out_dt;
     p.c_stride_batch = a.strideC[0]; p.c_stride_head = a.strideC[1]; p.c_stride_row = a.strideC[2];
     const int esz = a.out_dt == SQ_I32 ? 4 : (a.out_dt == SQ_I8 ? 1 : 2);

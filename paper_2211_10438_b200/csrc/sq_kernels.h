@@ -61,6 +61,7 @@ struct GemmArgs {
     int relu;
     const float* requant_mul; int requant_per_col;
     float* row_absmax_out;
+    const void* residual; int64_t ld_res;    // nullable: [M, N] of the output dtype, added after the output rounding
     void* C; sq_dtype out_dt;
     int64_t strideC[3];   // batch, head, row (elements)
     uint32_t* status;     // device status word (= workspace base)

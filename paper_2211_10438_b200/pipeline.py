@@ -169,10 +169,12 @@ def synth_device_weights(N, K, dtype, seed, std=0.02, device="cuda"):
 
 
 class DecoderBlockStatic:
-    """A full W8A8 decoder block with per-tensor STATIC activation steps (level O3), as eleven
-    libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> Q.K^T BMM -> softmax+quantise P ->
-    P.V BMM (INT8 out) -> out-proj GEMM -> residual -> LN2+quantise -> FC1 GEMM (+ReLU, INT8 out)
-    -> FC2 GEMM -> residual.  Q, K, V are read in place from the fused QKV buffer.
+    """A full W8A8 decoder block with per-tensor STATIC activation steps (level O3), as seven libsq
+    launches from 1024 tokens up (nine below; two more without the fused attention kernel):
+    LN1+quantise -> QKV GEMM (INT8 out) -> fused attention (or Q.K^T BMM -> softmax+quantise P ->
+    P.V BMM; INT8 out) -> out-proj GEMM with the residual add in its epilogue (or GEMM -> residual
+    add) -> LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM with the residual add in its
+    epilogue.  Q, K, V are read in place from the fused QKV buffer.
 
     `lin` maps "qkv" / "out_proj" / "fc1" / "fc2" to PreparedLinear; `steps` holds the calibrated
     static steps d_ln1, d_q, d_k, d_v, d_attn, d_ln2, d_fc1 (python floats)."""
@@ -199,13 +201,15 @@ class DecoderBlockStatic:
         e = lambda shape, dt: torch.empty(shape, dtype=dt, device=dev)
         self.x1q, self.qkv = e((M, hid), torch.int8), e((M, 3 * hid), torch.int8)
         self.scores, self.P = e((B * H, S, S), act_dtype), e((B * H, S, S), torch.int8)
-        self.attn, self.proj, self.h = e((M, hid), torch.int8), e((M, hid), act_dtype), e((M, hid), act_dtype)
+        self.attn, self.h = e((M, hid), torch.int8), e((M, hid), act_dtype)
         self.x2q, self.f1q = e((M, hid), torch.int8), e((M, ffn), torch.int8)
-        self.fc2, self.y = e((M, hid), act_dtype), e((M, hid), act_dtype)
+        self.y = e((M, hid), act_dtype)
         need = max([sq.workspace_bytes(sq.SQ_OP_GEMM, M, l.Wq.shape[0], l.Wq.shape[1]) for l in lin.values()] +
                    [sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, hid)])
         self.ws = sq.new_workspace(need, dev)
-        self.launches_per_step = 9 if self.fused_attention else 11
+        self.fuse_residual = M >= 1024
+        self.tmp = None if self.fuse_residual else e((M, hid), act_dtype)
+        self.launches_per_step = (7 if self.fused_attention else 9) + (0 if self.fuse_residual else 2)
 
     def forward(self, x):
         L, s, B, S, H, d, hid = self.lin, self.s, self.B, self.S, self.H, self.d, self.hid
@@ -223,17 +227,23 @@ class DecoderBlockStatic:
             sq.sq_softmax_quant_p(self.scores, self.P)
             sq.sq_w8a8_bmm(self.P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
                            self.alpha_pv, self.attn, (S * hid, d, hid), self.ws, requant_mul=self.r_attn, causal=True)
-        sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
-                        bias=L["out_proj"].bias, out=self.proj)
-        sq.sq_residual_add(x, self.proj, out=self.h)
+        self._linear_residual(self.attn, L["out_proj"], s["d_attn"], x, self.h)
         sq.sq_ln_quant(self.h, L["fc1"].gamma_hat, L["fc1"].beta_hat, self.eps, "per_tensor_static", Xq=self.x2q,
                        x_scale=s["d_ln2"], workspace=self.ws)
         sq.sq_w8a8_gemm(self.x2q, L["fc1"].Wq, s["d_ln2"], L["fc1"].w_scale, self.ws, bias=L["fc1"].bias, relu=True,
                         requant_mul=self.r_fc1, out=self.f1q)
-        sq.sq_w8a8_gemm(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, bias=L["fc2"].bias,
-                        out=self.fc2)
-        sq.sq_residual_add(self.h, self.fc2, out=self.y)
+        self._linear_residual(self.f1q, L["fc2"], s["d_fc1"], self.h, self.y)
         return self.y
+
+    def _linear_residual(self, xq, l, d_x, residual, out):
+        """out = residual + W8A8 linear(xq): one launch with the add in the GEMM epilogue from 1024 tokens
+        up (measured on B200: 3312 -> 3262 us per layer at 8192 tokens), two launches below, where the
+        single tile per CTA leaves the longer epilogue exposed (512 tokens: 291 against 296 us)."""
+        if self.fuse_residual:
+            sq.sq_w8a8_gemm_residual(xq, l.Wq, d_x, l.w_scale, self.ws, residual, bias=l.bias, out=out)
+        else:
+            sq.sq_w8a8_gemm(xq, l.Wq, d_x, l.w_scale, self.ws, bias=l.bias, out=self.tmp)
+            sq.sq_residual_add(residual, self.tmp, out=out)
 
     def ops(self):
         """Integer ops of the four GEMMs and two BMMs of one forward."""
@@ -246,7 +256,8 @@ class DecoderBlockDecode:
     """Generation stage of DecoderBlockStatic: one new token per sequence against an INT8 KV cache,
     as nine libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> attention of the new token over
     the cache, which also appends its k, v (INT8 out) -> out-proj GEMM -> residual ->
-    LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM -> residual.  Same `lin` / `steps` as the
+    LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM -> residual (the add folded into the GEMM
+    epilogue measured the same time here, so the two small launches stay).  Same `lin` / `steps` as the
     prompt block.  `ctx` (int32 device tensor [B]) counts the positions each sequence has cached."""
 
     def __init__(self, lin, steps, B, H, d, L_max, act_dtype, eps=1e-5):

@@ -150,6 +150,46 @@ def test_gemm_last_wave_k_split_is_exact(M, N, K):
     assert not big[4:33024].any(), "header and counters not handed back zero-filled"
 
 
+# the residual connection folded into the epilogue: bit for bit the unfused pair of calls.  Shapes: one
+# CTA pair tile with ragged M, single-CTA narrow and wide tiles, the weight-streaming kernel (shared
+# tiles), a K-split last wave (fix-up path), a strided residual and output
+RESIDUAL_SHAPES = [(300, 520, 272), (2048, 1024, 512), (128, 3000, 13008), (100, 40960, 256), (1, 128, 128),
+                   (16, 1280, 4096), (32, 12288, 6144), (512, 4096, 12288), (2, 4096, 49152)]
+
+
+@pytest.mark.parametrize("dtype", ["f16", "bf16"])
+@pytest.mark.parametrize("M,N,K", RESIDUAL_SHAPES)
+def test_gemm_residual_epilogue(ws, dtype, M, N, K):
+    Xq, Wq = synth.int8_tensor(29, 1, (M, K)), synth.int8_tensor(29, 2, (N, K))
+    rng = synth.rng_for(29, 3)
+    xs = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = synth.bias(29, 4, N, dtype, std=0.5)
+    ld = N + 24  # residual and output rows are strided views
+    res = synth.to_dtype_f32(rng.standard_normal((M, ld)).astype(np.float32) * 4, dtype)
+    y = oracle.round_to(oracle.dequant(oracle.gemm_i32(Xq, Wq), xs, wsc, bias), dtype)
+    want = oracle.round_to(y + res[:, :N], dtype)
+    tdt = torch.float16 if dtype == "f16" else torch.bfloat16
+    res_d = dev(res, dtype)
+    out = torch.zeros((M, ld), dtype=tdt, device="cuda")
+    sq.sq_w8a8_gemm_residual(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, res_d[:, :N], bias=dev(bias, dtype), out=out[:, :N])
+    assert np.array_equal(host(out)[:, :N], want)
+    assert not host(out)[:, N:].any(), "wrote outside the N columns"
+    # and it equals the two separate calls
+    y_d = sq.sq_w8a8_gemm(dev(Xq), dev(Wq), dev(xs), dev(wsc), ws, bias=dev(bias, dtype), out_dtype=tdt)
+    two = sq.sq_residual_add(y_d, res_d[:, :N].contiguous())
+    assert torch.equal(out[:, :N], two)
+
+
+def test_gemm_residual_argument_checks(ws):
+    X, W = torch.zeros((4, 64), dtype=torch.int8, device="cuda"), torch.zeros((12, 64), dtype=torch.int8, device="cuda")
+    one = torch.ones(1, device="cuda")
+    r = torch.zeros((4, 16), dtype=torch.float16, device="cuda")
+    with pytest.raises(sq.SqError) as e:  # N = 12 is not a multiple of 8
+        sq.sq_w8a8_gemm_residual(X, W, one, one, ws, r[:, :12], out=torch.empty((4, 12), dtype=torch.float16, device="cuda"))
+    assert e.value.code == sq.SQ_ERR_ALIGN
+
+
 # decode-shaped calls: swapped operands and K splits with INT32 scratch in the workspace up to 32 tokens
 DECODE_SHAPES = [(1, 128, 128), (16, 512, 512), (3, 200, 272), (16, 1280, 4096), (8, 12288, 6144), (5, 136, 12288),
                  (16, 36864, 1024), (2, 4096, 49152),
