@@ -12,7 +12,9 @@
 //   * the folded LayerNorm parameters gamma_hat / beta_hat live in shared memory for the whole
 //     kernel; a row is unpacked once into registers, so HBM sees 2 bytes in + 1 byte out per
 //     element and nothing else;
-//   * reductions (sum, sum of squares, absmax) are warp shuffles + one named barrier each.
+//   * reductions are warp shuffles + one named barrier each: one for the statistics (per-thread
+//     mean and squared deviations merged with the parallel-variance update; rows with a ragged
+//     tail take the sum first and the deviations second), one for the absolute maximum.
 // Arithmetic is the normative fp32 sequence: n = fma(x, rstd, -(mu*rstd)),
 // y = fma(n, gamma_hat, beta_hat), Delta = max(|y|, 1e-5)/127, q = round(y * (1/Delta)).
 // The kernel is instruction-issue sensitive (about 12 instructions per element at 3 bytes of
@@ -68,6 +70,44 @@ __device__ __forceinline__ float group_reduce(float v, float* red, int g, int gw
 #pragma unroll
     for (int i = 1; i < NW; ++i) r = IS_MAX ? fmaxf(r, p[i]) : r + p[i];
     return r;
+}
+
+// Mean and sum of squared deviations of a row whose threads all hold the same number of values
+// (n_lane each): every thread brings the statistics of its own values, pairs are merged with the
+// parallel-variance update (equal counts: mean = (a + b) / 2, M2 = M2a + M2b + (a - b)^2 * n / 2,
+// written symmetrically so that both lanes of a pair compute identical bits), warps are merged in
+// a fixed order by every thread.  One barrier instead of the two of "mean, then deviations".
+template <int GROUP, int CTA>
+__device__ __forceinline__ void group_merge_stats(float& mean, float& m2, float n_lane, float* red_mean, float* red_m2,
+                                                  int g, int gwarp, int lane) {
+    float n = n_lane;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, mean, o), o2 = __shfl_xor_sync(0xffffffffu, m2, o);
+        const float d = mean - om;
+        m2 = (m2 + o2) + (d * d) * (n * 0.5f);
+        mean = (mean + om) * 0.5f;
+        n += n;
+    }
+    constexpr int NW = GROUP / 32;
+    if constexpr (NW == 1) return;
+    if (lane == 0) { red_mean[gwarp] = mean; red_m2[gwarp] = m2; }
+    group_sync<GROUP, CTA>(g);
+    constexpr int NWP = (NW + 3) & ~3;
+    float pm[NWP], p2[NWP];
+#pragma unroll
+    for (int i = 0; i < NWP / 4; ++i) {
+        const float4 a = reinterpret_cast<const float4*>(red_mean)[i], b = reinterpret_cast<const float4*>(red_m2)[i];
+        pm[4 * i] = a.x; pm[4 * i + 1] = a.y; pm[4 * i + 2] = a.z; pm[4 * i + 3] = a.w;
+        p2[4 * i] = b.x; p2[4 * i + 1] = b.y; p2[4 * i + 2] = b.z; p2[4 * i + 3] = b.w;
+    }
+    mean = pm[0]; m2 = p2[0];
+#pragma unroll
+    for (int i = 1; i < NW; ++i) {  // i warps merged so far, one more of the same size
+        const float d = pm[i] - mean;
+        mean = fmaf(d, 1.0f / (float)(i + 1), mean);
+        m2 = (m2 + p2[i]) + (d * d) * (n * ((float)i / (float)(i + 1)));
+    }
 }
 
 // 1/sqrt(v) for the LayerNorm statistic: the hardware approximation plus one Newton step (about
@@ -214,8 +254,12 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                     sum2[1] = __fadd2_rn(sum2[1], __fadd2_rn(f[2], f[3]));
                 }
                 const float sum = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
-                mu = group_reduce<false, GROUP, CTA>(sum, red, g, gwarp, lane) * inv_C;
-                refill();
+                if constexpr (!EXACT) {
+                    mu = group_reduce<false, GROUP, CTA>(sum, red, g, gwarp, lane) * inv_C;
+                    refill();
+                } else {
+                    mu = sum * (1.0f / (float)(8 * V));  // this thread's own mean first
+                }
                 const float2 nmu2 = make_float2(-mu, -mu);
                 float2 ss2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
@@ -228,8 +272,14 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                         }
                     }
                 }
-                const float ss = (ss2[0].x + ss2[0].y) + (ss2[1].x + ss2[1].y);
-                const float var = group_reduce<false, GROUP, CTA>(ss, red + NWP, g, gwarp, lane) * inv_C;
+                float ss = (ss2[0].x + ss2[0].y) + (ss2[1].x + ss2[1].y);
+                if constexpr (!EXACT) {
+                    ss = group_reduce<false, GROUP, CTA>(ss, red + NWP, g, gwarp, lane);
+                } else {
+                    group_merge_stats<GROUP, CTA>(mu, ss, (float)(8 * V), red, red + NWP, g, gwarp, lane);
+                    refill();
+                }
+                const float var = ss * inv_C;
                 rstd = rsqrt_refined(var + eps);
                 if (stats != nullptr && gt == 0) {
                     stats[2 * row] = mu;
