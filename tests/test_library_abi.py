@@ -67,6 +67,17 @@ def test_validation_without_cuda(lib):
     assert args(64, wsp=None, wsn=0) == 7
     assert args(64, out_dt=sq.SQ_I8) == 1
     assert args(64, rq=p) == 1
+    # GEMM with the residual add: residual required, 16-bit output only, whole 8-element vectors
+    big = sq.workspace_bytes(sq.SQ_OP_GEMM, 16, 16, 64)
+    res = lambda r=p, out_dt=sq.SQ_F16, N=16, ldr=16, M=16: lib.sq_w8a8_gemm_residual(
+        i8, i8, M, N, 64, p, 1, p, 1, None, 0, r, ldr, p, out_dt, 16, ws, big, None)
+    assert res(r=None) == 1
+    assert res(out_dt=sq.SQ_I32) == 1
+    assert res(ldr=8) == 2
+    assert res(ldr=20) == 3
+    assert res(N=12, ldr=16) == 3
+    assert res(r=ctypes.c_void_p(0x1008)) == 3
+    assert res(M=0) == 0
     arr = ctypes.c_int64 * 3
     assert lib.sq_w8a8_bmm(i8, i8, 1, 1, 16, 256, 64, arr(0, 0, 64), arr(0, 0, 256), 1, 0, 1.0, None, p,
                            sq.SQ_F16, arr(0, 0, 256), ws, 256, None) == 4  # [K,N] B limited to N <= 128
