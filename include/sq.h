@@ -92,7 +92,8 @@ size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K);
  * first batch and may call once per calibration batch.  Applied to the stored weight
  * W[C_o, C_i] it yields max(|W_j|) of Eq. 4 (one value per INPUT channel).
  * The fast path needs X 16-byte aligned with cols and ld multiples of 8; other shapes run
- * a slower element-wise kernel.
+ * a slower element-wise kernel.  Batches of 2^27 elements or more stream through bulk copies
+ * whose waits are bounded: should one never land, the columns concerned receive NaN.
  */
 sq_status sq_calib_absmax(const void* X, sq_dtype dt, int64_t rows, int64_t cols, int64_t ld,
                           float* absmax_inout, void* stream);

@@ -5,6 +5,7 @@
 // its statistics pass and its quantise pass, so each element is read from HBM once.
 #include <cooperative_groups.h>
 
+#include "sq_bulk.cuh"
 #include "sq_common.cuh"
 #include "sq_kernels.h"
 
@@ -87,11 +88,137 @@ __global__ void col_absmax_scalar_kernel(const T* __restrict__ X, int64_t rows, 
     atomic_max_nonneg(absmax + j, m);
 }
 
+// The same reduction as a stream for large calibration batches: the columns are cut into slabs of
+// at most 640 vectors (5120 columns), the rows into gridDim.x / n_slabs parts; a CTA owns one slab
+// of one part.  Its 8 groups of 64 threads each walk their own rows: a row's slab segment (up to
+// 10 KB, contiguous) arrives by one bulk copy into the group's ring, every thread folds its 10
+// vectors into packed running maxima, and only at the end do the groups meet in shared memory and
+// issue one atomic max per column and CTA.  One named barrier per row and group: passing the
+// barrier of row k proves that everybody finished reading row k - 1, whose stage is then refilled.
+// A bulk copy that never lands (bounded wait) poisons the CTA's columns with NaN.
+constexpr int CAL_THREADS = 512, CAL_GROUP = 64, CAL_V = 10, CAL_G = CAL_THREADS / CAL_GROUP;
+template <typename T>
+__global__ void __launch_bounds__(CAL_THREADS, 1)
+col_absmax_stream_kernel(const T* __restrict__ X, int64_t rows, int64_t nvec, int64_t ld, int slab_vecs, int n_slabs,
+                         int stages, float* __restrict__ absmax) {
+    using namespace bulk;
+    extern __shared__ __align__(128) uint8_t cal_smem[];
+    const int tid = threadIdx.x, g = tid / CAL_GROUP, gt = tid % CAL_GROUP;
+    const int slab = blockIdx.x % n_slabs, part = blockIdx.x / n_slabs, parts = gridDim.x / n_slabs;
+    const int64_t v0 = (int64_t)slab * slab_vecs;
+    const int nv = (int)min((int64_t)slab_vecs, nvec - v0);  // vectors of this slab
+    const uint32_t seg_bytes = (uint32_t)nv * 16u;
+    const size_t stage_bytes = (size_t)slab_vecs * 16;
+    uint8_t* ring = cal_smem + (size_t)g * stages * stage_bytes;
+    uint64_t* full = reinterpret_cast<uint64_t*>(cal_smem + (size_t)CAL_G * stages * stage_bytes) + g * stages;
+    volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(
+        reinterpret_cast<uint64_t*>(cal_smem + (size_t)CAL_G * stages * stage_bytes) + CAL_G * stages);
+    volatile uint32_t* my_flag = flags + g;
+    volatile uint32_t* bad = flags + CAL_G;
+    if (tid == 0) *bad = 0u;
+    if (gt == 0) {
+        for (int s = 0; s < stages; ++s) mbar_init(full + s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const int64_t first = (int64_t)part * CAL_G + g, stride = (int64_t)parts * CAL_G;
+    const T* src = X + v0 * 8;
+    if (gt == 0) {
+        for (int s = 0; s < stages; ++s) {
+            const int64_t r = first + s * stride;
+            if (r < rows) {
+                mbar_expect_tx(full + s, seg_bytes);
+                bulk_load(ring + (size_t)s * stage_bytes, src + r * ld, seg_bytes, full + s);
+            }
+        }
+    }
+    uint4 cm[CAL_V];
+#pragma unroll
+    for (int i = 0; i < CAL_V; ++i) cm[i] = make_uint4(0u, 0u, 0u, 0u);
+    int s = 0, prev = -1;
+    uint32_t parity = 0;
+    int64_t prev_row = 0;
+    for (int64_t row = first; row < rows; row += stride) {
+        if (gt == 0) {
+            const bool ok = mbar_wait_bounded(full + s, parity);
+            *my_flag = ok ? 1u : 0u;
+        }
+        asm volatile("bar.sync %0, %1;" ::"r"(g + 1), "n"(CAL_GROUP) : "memory");
+        if (*my_flag == 0u) { *bad = 1u; break; }
+        if (gt == 0 && prev >= 0) {  // everybody is past the reads of the previous row: refill its stage
+            const int64_t nxt = prev_row + (int64_t)stages * stride;
+            if (nxt < rows) {
+                mbar_expect_tx(full + prev, seg_bytes);
+                bulk_load(ring + (size_t)prev * stage_bytes, src + nxt * ld, seg_bytes, full + prev);
+            }
+        }
+        const uint4* seg = reinterpret_cast<const uint4*>(ring + (size_t)s * stage_bytes);
+#pragma unroll
+        for (int i = 0; i < CAL_V; ++i) {
+            const int v = gt + i * CAL_GROUP;
+            if (v < nv) {
+                const uint4 x = seg[v];
+                cm[i].x = Act<T>::absmax2(cm[i].x, x.x); cm[i].y = Act<T>::absmax2(cm[i].y, x.y);
+                cm[i].z = Act<T>::absmax2(cm[i].z, x.z); cm[i].w = Act<T>::absmax2(cm[i].w, x.w);
+            }
+        }
+        prev = s; prev_row = row;
+        if (++s == stages) { s = 0; parity ^= 1u; }
+    }
+    __syncthreads();  // every group is done with its ring: the space becomes [group][vector] scratch
+    uint4* scratch = reinterpret_cast<uint4*>(cal_smem);
+#pragma unroll
+    for (int i = 0; i < CAL_V; ++i) {
+        const int v = gt + i * CAL_GROUP;
+        if (v < nv) scratch[(size_t)g * slab_vecs + v] = cm[i];
+    }
+    __syncthreads();
+    const bool poisoned = *bad != 0u;
+    for (int v = tid; v < nv; v += CAL_THREADS) {
+        uint4 m = scratch[v];
+#pragma unroll
+        for (int o = 1; o < CAL_G; ++o) {
+            const uint4 x = scratch[(size_t)o * slab_vecs + v];
+            m.x = Act<T>::absmax2(m.x, x.x); m.y = Act<T>::absmax2(m.y, x.y);
+            m.z = Act<T>::absmax2(m.z, x.z); m.w = Act<T>::absmax2(m.w, x.w);
+        }
+        float f[8];
+        unpack8<T>(m, f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            atomic_max_nonneg(absmax + (v0 + v) * 8 + i, poisoned ? __uint_as_float(0x7fc00000u) : f[i]);
+    }
+}
+
 template <typename T>
 static sq_status calib_absmax_t(const void* X, int64_t rows, int64_t cols, int64_t ld, float* a,
                                 cudaStream_t st) {
     const T* x = static_cast<const T*>(X);
     const int sms = sm_count();
+    // (from about 256 MB per call the stream wins -- 16384 x 20480: 120 -> 101 us; below, its ring fill and
+    // its final meeting of the groups cost more than they save, and a batch that fits L2 favours plain loads)
+    if (aligned16(X) && cols % 8 == 0 && ld % 8 == 0 && cols >= 2048 && rows * cols >= ((int64_t)1 << 27)) {
+        const int64_t nvec = cols / 8;
+        const int n_slabs = (int)((nvec + CAL_GROUP * CAL_V - 1) / (CAL_GROUP * CAL_V));
+        if (n_slabs <= sms) {
+            const int slab_vecs = (int)((nvec + n_slabs - 1) / n_slabs);
+            const int parts = (int)std::max<int64_t>(1, std::min<int64_t>(sms / n_slabs, (rows + CAL_G - 1) / CAL_G));
+            const size_t stage_all = (size_t)CAL_G * slab_vecs * 16;
+            const int stages = (int)std::min<size_t>(4, (size_t)(200 * 1024) / stage_all);  // >= 2: a slab is at most 10 KB
+            const size_t smem = stage_all * stages + (size_t)CAL_G * stages * 8 + (CAL_G + 1) * 4 + 64;
+            auto kern = col_absmax_stream_kernel<T>;
+            static bool attr_set[64] = {false};
+            int dev = 0;
+            SQ_CUDA_OK(cudaGetDevice(&dev));
+            if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+                SQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+                if (dev >= 0 && dev < 64) attr_set[dev] = true;
+            }
+            kern<<<dim3((unsigned)(parts * n_slabs)), CAL_THREADS, smem, st>>>(x, rows, nvec, ld, slab_vecs, n_slabs, stages, a);
+            return launch_status();
+        }
+    }
     if (aligned16(X) && cols % 8 == 0 && ld % 8 == 0) {
         const int64_t gx = (cols / 8 + 31) / 32;
         // enough row slices for ~8 resident CTAs per SM, but at least 32 rows per slice

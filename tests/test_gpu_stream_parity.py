@@ -22,7 +22,11 @@ def _acts(cfg, tid, M, C, dtype, n_out=4, fac=50.0):
 
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
 @pytest.mark.parametrize("rows,cols,ld", [(300, 1000, 1000), (2048, 5120, 5120), (77, 264, 512),
-                                          (129, 1003, 1003), (1, 8, 8), (64, 7168, 7168)])
+                                          (129, 1003, 1003), (1, 8, 8), (64, 7168, 7168),
+                                          # the streaming kernel: several column slabs, ragged last slab,
+                                          # strided rows, fewer rows than row groups, many rows per group
+                                          (6600, 20480, 20480), (11000, 12296, 12360), (66000, 2048, 2048),
+                                          (13200, 10240, 10304)])
 def test_calib_absmax_exact(dtype, rows, cols, ld):
     x = _acts(7, 1, rows, ld, dtype)
     xd = dev(x, dtype)
