@@ -146,7 +146,9 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
 
     const int tid = threadIdx.x;
     const int g = tid / GROUP, gt = tid % GROUP, gwarp = gt >> 5, lane = tid & 31;
-    const int64_t first = (int64_t)blockIdx.x * G + g;
+    // rows go round the CTAs first and round a CTA's groups second: a handful of rows (one token per
+    // sequence at the generation stage) then sit on as many SMs instead of sharing one
+    const int64_t first = (int64_t)g * gridDim.x + blockIdx.x;
     const int64_t stride = (int64_t)gridDim.x * G;
     uint64_t* my_full = full + g * stages;
     uint8_t* my_rows = s_rows + (size_t)g * stages * row_bytes;
@@ -400,7 +402,7 @@ sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, co
         SQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    const int grid = (int)std::min<int64_t>((M + G - 1) / G, sm_count());
+    const int grid = (int)std::min<int64_t>(M, sm_count());
     return launch_pdl(kern, dim3((unsigned)grid), dim3(CTA), smem, st, 1, static_cast<const T*>(X), M,
                       (int)C, static_cast<const T*>(gamma), static_cast<const T*>(beta), col_mul, eps, mode, stages, Xq, scale,
                       absmax_word, stats, stats_are_input, status);
