@@ -83,12 +83,13 @@ def kv_attention(args):
 def _rows(args, ln):
     g = _gen()
     M, C = args.rows, args.C
-    x = torch.randn((M, C), device="cuda", dtype=torch.bfloat16, generator=g)
+    dt = torch.float16 if args.dtype == "f16" else torch.bfloat16
+    x = torch.randn((M, C), device="cuda", dtype=dt, generator=g)
     x[:, ::200] *= 100
     Xq = torch.empty((M, C), dtype=torch.int8, device="cuda")
     xs = torch.empty(M, dtype=torch.float32, device="cuda")
-    gamma = torch.ones(C, dtype=torch.bfloat16, device="cuda")
-    beta = torch.zeros(C, dtype=torch.bfloat16, device="cuda")
+    gamma = torch.ones(C, dtype=dt, device="cuda")
+    beta = torch.zeros(C, dtype=dt, device="cuda")
     ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_LN_QUANT, M, 0, C))
     if ln:
         us = _time(lambda: sq.sq_ln_quant(x, gamma, beta, 1e-5, "per_token", Xq=Xq, x_scale=xs, workspace=ws), args.calls)
@@ -99,12 +100,12 @@ def _rows(args, ln):
 
 
 def ln_quant(args):
-    """Fused LayerNorm + per-token quantise of a bf16 [rows, C] tensor (default 8192 x 20480)."""
+    """Fused LayerNorm + per-token quantise of a bf16 / fp16 [rows, C] tensor (default 8192 x 20480)."""
     return _rows(args, True)
 
 
 def quant_act(args):
-    """Per-token quantise of a bf16 [rows, C] tensor (default 8192 x 20480)."""
+    """Per-token quantise of a bf16 / fp16 [rows, C] tensor (default 8192 x 20480)."""
     return _rows(args, False)
 
 
@@ -121,6 +122,7 @@ def main(argv=None):
     ap.add_argument("--L", type=int, default=2048)
     ap.add_argument("--rows", type=int, default=8192)
     ap.add_argument("--C", type=int, default=20480)
+    ap.add_argument("--dtype", choices=["bf16", "f16"], default="bf16", help="ln_quant / quant_act: activation type")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device: the library has no CPU fallback")
