@@ -26,7 +26,9 @@
 // ring stage at hidden sizes 8192 to 20480 -- bit-identical output, 0.79 instead of 0.81 of the copy
 // bandwidth at 20480 and 0.82 instead of 0.87 at 12288, so the bytes in flight are not what
 // limits those shapes; 256- and 320-thread CTAs with 128 to 160 values per thread at 20480 (too
-// few warps to cover the reductions); 640 threads with 64 values per thread.
+// few warps to cover the reductions); 640 threads with 64 values per thread; fp32 copies of
+// gamma_hat / beta_hat in shared memory, which take the two unpacks per element out of the inner
+// loop but double the bytes every row reads back from shared memory (65536 x 7168: 0.96 -> 0.71).
 #include "sq_common.cuh"
 #include "sq_bulk.cuh"
 #include "sq_kernels.h"
