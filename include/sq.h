@@ -18,8 +18,13 @@
  *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *    Calls only enqueue work: they never synchronise and never change the current device.
  *  - The return code reports argument validation and launch errors.  Device-side waits
- *    are bounded; if one expires the kernel records a non-zero word at workspace[0]
- *    (see sq_w8a8_gemm) and returns instead of hanging.
+ *    are bounded; if one expires the kernel records SQ_ERR_TIMEOUT | where << 8 at
+ *    workspace[0] (the sticky device status word: written only while it is zero) and returns
+ *    instead of hanging; the rows or tiles it had not finished stay unwritten.  This needs a
+ *    workspace: the quantisers (sq_quant_act, sq_ln_quant, sq_quant_weight) accept NULL in
+ *    their per-token / static / per-channel modes, and a call made without one cannot report
+ *    an expired wait (it still returns).  sq_calib_absmax, which takes no workspace, marks the
+ *    columns concerned with NaN instead.
  *  - Rounding is round-to-nearest-even everywhere; INT8 codes lie in [-127, 127].
  *  - Inputs must be finite; NaN/Inf give unspecified codes (never a fault).
  *  - A zero-sized problem (M == 0 or N == 0 ...) is a no-op that returns SQ_OK.
@@ -142,7 +147,11 @@ sq_status sq_fold_ln_weight(const void* gamma, const void* beta, sq_dtype dt, co
  * Wq = clamp(round(W_hat / Delta_w), -127, 127).
  * W: [N, K] dtype dt, contiguous.  Wq: [N, K] int8.  w_scale: [N] (per channel) or [1]
  * fp32, receives Delta_w.  workspace: sq_workspace_bytes(SQ_OP_QUANT_WEIGHT, ...) bytes
- * (only the per-tensor mode uses it).  K must be a multiple of 8 and W 16-byte aligned.
+ * (required by the per-tensor mode; in the per-channel mode it may be NULL and only serves as
+ * the device status word).  K must be a multiple of 8 and W 16-byte aligned.
+ * This is the one call of the library that WRITES weights, and sq_w8a8_gemm with M <= 32 starts
+ * fetching Wq before it waits for the launch in front of it; the call therefore ends with an
+ * empty, fully serialised launch, so that it may be followed directly by a GEMM on the stream.
  */
 sq_status sq_quant_weight(const void* W, sq_dtype dt, int64_t N, int64_t K, const float* s,
                           sq_w_gran g, int8_t* Wq, float* w_scale, void* workspace,
@@ -157,8 +166,8 @@ sq_status sq_quant_weight(const void* W, sq_dtype dt, int64_t N, int64_t K, cons
  * Xq = clamp(round(x * (1/Delta)), -127, 127); maxima are floored at 1e-5.
  * X: [M, C] dtype dt, contiguous, 16-byte aligned, C a multiple of 8.  col_mul: optional
  * [C] fp32 multiplier applied first in fp32 (an explicit 1/s when the producer is not a
- * LayerNorm); NULL for none.  Xq: [M, C] int8.  workspace: used by the per-tensor dynamic
- * mode only.
+ * LayerNorm); NULL for none.  Xq: [M, C] int8.  workspace: required by the per-tensor dynamic
+ * mode (sq_workspace_bytes(SQ_OP_QUANT_ACT, ...)); otherwise optional, word 0 = device status.
  */
 sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_gran g,
                        const float* col_mul, int8_t* Xq, float* x_scale, void* workspace,
@@ -167,9 +176,14 @@ sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_
 /*
  * Fused LayerNorm (with the smoothing factor already folded into gamma_hat, beta_hat by
  * sq_fold_ln_weight) + Eq. 1, one pass over X:
- *     mu_t, var_t = mean and biased variance of row t (fp32, two-pass),
- *     y = fma((x - mu_t) * rstd_t, gamma_hat_j, beta_hat_j),  rstd_t = 1/sqrt(var_t + eps),
- * then y is quantised exactly as in sq_quant_act WITHOUT being rounded to A first.
+ *     mu_t, var_t = mean and biased variance of row t: fp32, one pass -- per-thread (mean, sum of
+ *                   squared deviations) pairs merged with the parallel-variance update; rows whose
+ *                   length does not divide evenly take the sum first and the deviations second,
+ *     rstd_t = 1/sqrt(var_t + eps),
+ *     n = fma(x, rstd_t, -(mu_t * rstd_t)),  y = fma(n, gamma_hat_j, beta_hat_j)     (fp32),
+ * then y is quantised exactly as in sq_quant_act WITHOUT being rounded to A first.  The
+ * statistics are a tolerance quantity (within 1e-6 relative of the fp64 two-pass values); the
+ * element-wise part, given them, is bit-exact.
  * X: [M, C] dtype dt; gamma_hat, beta_hat: [C] dtype dt (beta_hat may be NULL).
  * dbg_mean_rstd: optional [2*M] fp32, receives mu_t at [2t] and rstd_t at [2t+1] so that a
  * checker can reproduce the element-wise part bit for bit.  Other arguments as sq_quant_act.
@@ -341,8 +355,9 @@ sq_status sq_kv_cache_write(const int8_t* qkv, int64_t ld, int64_t B, int64_t T,
  * for the steps to come -- one launch less per generated token; the result is the same.
  * max_len: a host-side upper bound of seq_lens[] (<= L_max) that sizes shared memory and the
  * split of one sequence over a thread-block cluster -- a longer sequence is truncated to max_len
- * and the device status word is set (SQ_ERR_SHAPE); seq_lens[b] <= 0 gives a zero output row
- * (and appends nothing).
+ * and the device status word is set (SQ_ERR_SHAPE): its output is the attention over the first
+ * max_len cached positions and k_new / v_new are NOT appended (the cache is left as it was);
+ * seq_lens[b] <= 0 gives a zero output row (and appends nothing).
  * out: [B, ldo] of out_dt (SQ_I8 needs requant_mul, a device pointer to one fp32; SQ_F16 / SQ_BF16
  * ignore it).  d must be 128 (else SQ_ERR_UNSUPPORTED), L_max a multiple of 4, ldq and ld_new
  * multiples of 16, q / k_new / v_new / caches 16-byte aligned; max_len beyond what eight CTAs can
@@ -385,6 +400,14 @@ sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, 
  * context stays usable.  status_word: device pointer to a zero-initialised uint32.
  */
 sq_status sq_selftest_bounded_wait(uint32_t* status_word, uint32_t budget_cycles, void* stream);
+
+/*
+ * The same self-test for the bounded wait of the row kernels (sq_quant_act, sq_ln_quant,
+ * sq_quant_weight wait for each row's bulk copy on an mbarrier; no counterpart in the paper): one
+ * thread waits `budget_cycles` on a barrier nothing completes, then stores
+ * SQ_ERR_TIMEOUT | (5 << 8) into *status_word exactly as those kernels do, and returns.
+ */
+sq_status sq_selftest_row_wait(uint32_t* status_word, uint32_t budget_cycles, void* stream);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,7 @@ EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm", "sq_w8a8_gemm_residual",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
            "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention",
-           "sq_token_absmax", "sq_clipped_absmax"]
+           "sq_token_absmax", "sq_clipped_absmax", "sq_selftest_row_wait"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -74,6 +74,7 @@ def lib():
         L.sq_residual_add.argtypes = [vp, vp, i32, i64, vp, vp]
         L.sq_ln_quant_tensor_noalloc.argtypes = [vp, i32, i64, i64, vp, vp, f32, vp, vp, vp]
         L.sq_selftest_bounded_wait.argtypes = [vp, c.c_uint32, vp]
+        L.sq_selftest_row_wait.argtypes = [vp, c.c_uint32, vp]
         L.sq_w8a8_attention.argtypes = [vp, i64, i64, i64, i64, f32, f32, vp, vp, vp, sz, vp]
         L.sq_token_absmax.argtypes = [vp, i32, i64, i64, i64, vp, vp]
         L.sq_clipped_absmax.argtypes = [vp, i64, i64, vp, vp, vp]
@@ -279,6 +280,13 @@ def sq_selftest_bounded_wait(budget_cycles=200000):
     (SQ_ERR_TIMEOUT | where << 8 when the wait gave up as designed)."""
     word = torch.zeros(1, dtype=torch.int32, device="cuda")
     _check(lib().sq_selftest_bounded_wait(_ptr(word), int(budget_cycles), _stream()), "sq_selftest_bounded_wait")
+    return int(word.item())
+
+
+def sq_selftest_row_wait(budget_cycles=200000):
+    """The same self-test for the row kernels' wait on a row's bulk copy (expected: SQ_ERR_TIMEOUT | 5 << 8)."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().sq_selftest_row_wait(_ptr(word), int(budget_cycles), _stream()), "sq_selftest_row_wait")
     return int(word.item())
 
 

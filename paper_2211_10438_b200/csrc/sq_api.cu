@@ -21,22 +21,24 @@ sq_status quant_rows_common(const void* X, sq_dtype dt, int64_t M, int64_t C, co
                             const void* gamma, const void* beta, float eps, bool ln, int gran /*sq_act_gran*/,
                             int8_t* Xq, float* scale, float* dbg_stats, void* workspace, size_t ws_bytes,
                             size_t ws_need, cudaStream_t st) {
+    // word 0 of a workspace, when the caller gave one, receives the device status of an expired wait
+    uint32_t* status = ws_ok(workspace, ws_bytes, sizeof(uint32_t)) ? static_cast<uint32_t*>(workspace) : nullptr;
     if (gran == SQ_PER_TOKEN_DYNAMIC)
         return row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_DYNAMIC, Xq, scale, nullptr,
-                         dbg_stats, 0, st);
+                         dbg_stats, 0, status, st);
     if (gran == SQ_PER_TENSOR_STATIC)
         return row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_GIVEN_SCALE, Xq, scale, nullptr,
-                         dbg_stats, 0, st);
+                         dbg_stats, 0, status, st);
     // per-tensor dynamic: pass 1 folds every row's maximum into one word (and keeps the
     // LayerNorm statistics), pass 2 quantises with the step derived from it
     if (!ws_ok(workspace, ws_bytes, ws_need)) return SQ_ERR_WORKSPACE;
     float* word = ws_absmax(workspace);
     float* stats = ln ? (dbg_stats ? dbg_stats : ws_stats(workspace)) : nullptr;
     sq_status s = row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_ABSMAX_ONLY, nullptr, nullptr,
-                            word, stats, 0, st);
+                            word, stats, 0, status, st);
     if (s != SQ_OK) return s;
     s = row_quant(X, dt, M, C, col_mul, gamma, beta, eps, ln, ROW_FROM_ABSMAX_WORD, Xq, scale, word, stats,
-                  ln ? 1 : 0, st);
+                  ln ? 1 : 0, status, st);
     if (s != SQ_OK) return s;
     SQ_CUDA_OK(cudaMemsetAsync(word, 0, sizeof(float), st));  // leave the workspace zero-filled
     if (ln && !dbg_stats) SQ_CUDA_OK(cudaMemsetAsync(stats, 0, (size_t)M * 2 * sizeof(float), st));
@@ -133,10 +135,15 @@ sq_status sq_quant_weight(const void* W, sq_dtype dt, int64_t N, int64_t K, cons
     if (K % 8 != 0 || !aligned16(W) || (reinterpret_cast<uintptr_t>(Wq) & 7) != 0 || (s && !aligned16(s)))
         return SQ_ERR_ALIGN;
     // a weight row is quantised exactly like a token row whose column multiplier is s
-    return quant_rows_common(W, dt, N, K, s, nullptr, nullptr, 0.0f, false,
-                             g == SQ_W_PER_CHANNEL ? SQ_PER_TOKEN_DYNAMIC : SQ_PER_TENSOR_DYNAMIC, Wq, w_scale,
-                             nullptr, workspace, ws_bytes, sq_workspace_bytes(SQ_OP_QUANT_WEIGHT, N, N, K),
-                             as_stream(stream));
+    sq_status st = quant_rows_common(W, dt, N, K, s, nullptr, nullptr, 0.0f, false,
+                                     g == SQ_W_PER_CHANNEL ? SQ_PER_TOKEN_DYNAMIC : SQ_PER_TENSOR_DYNAMIC, Wq, w_scale,
+                                     nullptr, workspace, ws_bytes, sq_workspace_bytes(SQ_OP_QUANT_WEIGHT, N, N, K),
+                                     as_stream(stream));
+    if (st != SQ_OK) return st;
+    // The decode-shaped GEMM fetches weights before it waits for the launch in front of it (weights
+    // are normally static).  This offline call is the one library kernel that WRITES weights, so it
+    // ends with a fully serialised empty launch: whatever follows on the stream finds Wq complete.
+    return stream_full_dependency(as_stream(stream));
 }
 
 sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_gran g, const float* col_mul,
@@ -340,6 +347,12 @@ sq_status sq_selftest_bounded_wait(uint32_t* status_word, uint32_t budget_cycles
     if (!status_word) return SQ_ERR_INVALID_ARG;
     if (budget_cycles > 100000000u) return SQ_ERR_INVALID_ARG;  // a self-test never waits longer than ~50 ms
     return bounded_wait_selftest(status_word, budget_cycles, as_stream(stream));
+}
+
+sq_status sq_selftest_row_wait(uint32_t* status_word, uint32_t budget_cycles, void* stream) {
+    if (!status_word) return SQ_ERR_INVALID_ARG;
+    if (budget_cycles > 100000000u) return SQ_ERR_INVALID_ARG;
+    return row_wait_selftest(status_word, budget_cycles, as_stream(stream));
 }
 
 sq_status sq_residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out, void* stream) {

@@ -24,13 +24,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// false when the phase did not complete within kWaitCycles: the caller records it and stops
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+// false when the phase did not complete within `budget` cycles: the caller records it and stops
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t budget = kWaitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity))
-        if ((++spins & 63u) == 0u && (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) return false;
+        if ((++spins & 63u) == 0u && (unsigned long long)(clock64() - t0) > (unsigned long long)budget) return false;
     return true;
 }
 // contiguous global -> shared copy, completion counted in bytes on `bar`; both addresses 16-byte

@@ -142,6 +142,14 @@ __device__ __forceinline__ uint2 quant8_pairs(const float2 (&f)[4], float inv) {
     return make_uint2(pack4(c[0], c[1], c[2], c[3]), pack4(c[4], c[5], c[6], c[7]));
 }
 
+// 1/sqrt(v) for the LayerNorm statistic: the hardware approximation plus one Newton step (about
+// one unit in the last place; the statistic is a tolerance quantity, the element-wise part that
+// consumes it is the bit-exact one).
+__device__ __forceinline__ float rsqrt_refined(float v) {
+    const float r = rsqrtf(v), h = 0.5f * v;
+    return fmaf(r, fmaf(-h * r, r, 0.5f), r);
+}
+
 // ---------------------------------------------------------------------------------------
 // Reductions
 // ---------------------------------------------------------------------------------------

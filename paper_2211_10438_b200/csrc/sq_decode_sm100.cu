@@ -12,6 +12,12 @@
 //     with plain stores (INT32 partial sums add exactly in any order); the CTA that arrives
 //     last for a tile (one atomic counter per tile) adds the other slots, applies Eq. 2
 //     (dequant, bias, ReLU, requant), writes Y and leaves the counter zeroed for the next call.
+//   * optionally the activation quantiser runs INSIDE this kernel (Eq. 1 per token, or with a given
+//     static step; optionally behind the folded LayerNorm): while every CTA's first weight slices
+//     are already in flight, CTA r quantises token row r (16-bit values -> INT8 codes + step size,
+//     written to scratch in the workspace), the CTAs meet on one counter, and only then are the
+//     activation slices fetched.  The quantiser's cost hides behind the first fill of the ring
+//     instead of being a launch of its own in front of the GEMM.
 // Every wait is bounded (status word, as in the prefill kernel).
 #include "sq_kernels.h"
 #include "sq_tcgen05.cuh"
@@ -33,7 +39,7 @@ struct DecCfg {
     static constexpr int STAGE = W_BYTES + X_BYTES;
     static constexpr int STAGES = 10;
     static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
-    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 4) * 8 + 64 + DN * 4;
+    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 5) * 8 + 64 + DN * 4 + 32;
 };
 
 struct DecParams {
@@ -45,6 +51,7 @@ struct DecParams {
     int maxcount;        // most CTAs that share one tile
     const float* x_scale; int x_per_row;
     const float* w_scale; int w_per_col;
+    float alpha;         // the tokens' common factor when x_scale == nullptr (batched-matmul calls)
     const void* bias; int bias_is_bf16;
     int relu;
     const float* requant_mul; int requant_per_col;  // INT8 output: code = round(y * r)
@@ -54,6 +61,18 @@ struct DecParams {
     const void* residual;  // nullable: [M, N] of the output type, row stride ld_res
     int64_t ld_res;
     uint32_t* status;
+    // Activation quantiser in the prologue (x_raw != nullptr).  x_scale then points at the step sizes
+    // the prologue itself writes (per-token dynamic) or at the caller's static step.
+    const void* x_raw;      // [M, K] fp16 / bf16, contiguous
+    int x_is_bf16;
+    const void* ln_gamma;   // nullable: folded LayerNorm parameters [K] of x_raw's type -> LayerNorm first
+    const void* ln_beta;    // nullable
+    float ln_eps;
+    int x_static;           // 1: Delta = x_scale[0] is given; 0: Delta_t = absmax(row t) / 127 -> xs_out[t]
+    int8_t* xq;             // [M, K] codes: written here, read back through the tensor map of X
+    float* xs_out;          // [M] step sizes (dynamic mode)
+    float* stats_out;       // nullable [2 M]: mean and 1/sqrt(var + eps) of every row
+    uint32_t* sync;         // [2]: rows quantised so far, CTAs past the meeting point; zero between calls
 };
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -66,6 +85,154 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 __device__ __forceinline__ void dec_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------
+// The activation quantiser of the prologue: one token row per call, by the 128 epilogue threads.
+// Arithmetic is the library's normative fp32 sequence (Eq. 1: Delta = max(m, 1e-5) / 127,
+// code = round(v * (1 / Delta)); LayerNorm: n = fma(x, rstd, -(mu * rstd)), y = fma(n, g, b),
+// statistics two-pass in fp32), so codes and step sizes equal those of sq_quant_act /
+// sq_ln_quant given the same statistics.
+// ------------------------------------------------------------------------------------
+constexpr int QV = 12;  // 16-byte vectors of the row a thread keeps in registers (rows up to 12 288 elements)
+
+template <bool IS_MAX>
+__device__ __forceinline__ float dec_epi_reduce(float v, float* red, int wq, int lane) {
+    v = IS_MAX ? warp_max(v) : warp_sum(v);
+    if (lane == 0) red[wq] = v;
+    dec_epi_sync();
+    const float a = red[0], b = red[1], c = red[2], d = red[3];
+    dec_epi_sync();  // `red` is rewritten by the next reduction
+    return IS_MAX ? fmaxf(fmaxf(a, b), fmaxf(c, d)) : (a + b) + (c + d);
+}
+
+template <typename T>
+__device__ __forceinline__ void dec_ln_vec(const uint4& xv, const uint4* g4, const uint4* b4, int v, float rstd,
+                                           float shift, float (&y)[8]) {
+    float x[8], g[8], b[8];
+    unpack8<T>(xv, x);
+    unpack8<T>(__ldg(g4 + v), g);
+    if (b4 != nullptr) unpack8<T>(__ldg(b4 + v), b);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+        y[k] = __fmaf_rn(__fmaf_rn(x[k], rstd, shift), g[k], b4 != nullptr ? b[k] : 0.0f);
+}
+
+template <typename T>
+__device__ void dec_quant_row(const DecParams& p, int row, int et, float* red) {
+    const int wq = et >> 5, lane = et & 31;
+    const int nvec = (int)(p.K >> 3);
+    const uint4* src = reinterpret_cast<const uint4*>(static_cast<const T*>(p.x_raw) + (int64_t)row * p.K);
+    const uint4* g4 = reinterpret_cast<const uint4*>(p.ln_gamma);
+    const uint4* b4 = reinterpret_cast<const uint4*>(p.ln_beta);
+    const bool ln = p.ln_gamma != nullptr;
+    // the row comes from the kernel in front: read it through L2 (never a stale L1 line)
+    uint4 c[QV];
+#pragma unroll
+    for (int i = 0; i < QV; ++i) {
+        const int v = et + i * 128;
+        c[i] = v < nvec ? __ldcg(src + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
+    float rstd = 1.0f, shift = 0.0f;
+    if (ln) {
+        const float inv_C = __fdiv_rn(1.0f, (float)p.K);
+        float sum = 0.0f;
+#pragma unroll
+        for (int i = 0; i < QV; ++i) {  // zero-filled vectors add nothing
+            float f[8];
+            unpack8<T>(c[i], f);
+            sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
+        }
+        for (int v = et + QV * 128; v < nvec; v += 128) {
+            float f[8];
+            unpack8<T>(__ldcg(src + v), f);
+            sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
+        }
+        const float mu = dec_epi_reduce<false>(sum, red, wq, lane) * inv_C;
+        float ss = 0.0f;
+#pragma unroll
+        for (int i = 0; i < QV; ++i) {
+            if (et + i * 128 < nvec) {
+                float f[8];
+                unpack8<T>(c[i], f);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) { const float d = f[k] - mu; ss = fmaf(d, d, ss); }
+            }
+        }
+        for (int v = et + QV * 128; v < nvec; v += 128) {
+            float f[8];
+            unpack8<T>(__ldcg(src + v), f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { const float d = f[k] - mu; ss = fmaf(d, d, ss); }
+        }
+        ss = dec_epi_reduce<false>(ss, red, wq, lane);
+        rstd = rsqrt_refined(ss * inv_C + p.ln_eps);
+        shift = -__fmul_rn(mu, rstd);
+        if (p.stats_out != nullptr && et == 0) {
+            p.stats_out[2 * row] = mu;
+            p.stats_out[2 * row + 1] = rstd;
+        }
+    }
+    float delta;
+    if (p.x_static) {
+        delta = __ldg(p.x_scale);
+    } else {
+        float m = 0.0f;
+        if (ln) {
+#pragma unroll
+            for (int i = 0; i < QV; ++i) {
+                const int v = et + i * 128;
+                if (v < nvec) {
+                    float y[8];
+                    dec_ln_vec<T>(c[i], g4, b4, v, rstd, shift, y);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(y[k]));
+                }
+            }
+            for (int v = et + QV * 128; v < nvec; v += 128) {
+                float y[8];
+                dec_ln_vec<T>(__ldcg(src + v), g4, b4, v, rstd, shift, y);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(y[k]));
+            }
+        } else {
+            uint32_t pm = 0u;  // |x| and max are exact on the packed 16-bit values
+#pragma unroll
+            for (int i = 0; i < QV; ++i) {
+                pm = Act<T>::absmax2(pm, c[i].x); pm = Act<T>::absmax2(pm, c[i].y);
+                pm = Act<T>::absmax2(pm, c[i].z); pm = Act<T>::absmax2(pm, c[i].w);
+            }
+            for (int v = et + QV * 128; v < nvec; v += 128) {
+                const uint4 x = __ldcg(src + v);
+                pm = Act<T>::absmax2(pm, x.x); pm = Act<T>::absmax2(pm, x.y);
+                pm = Act<T>::absmax2(pm, x.z); pm = Act<T>::absmax2(pm, x.w);
+            }
+            m = Act<T>::hmax_of2(pm);
+        }
+        m = dec_epi_reduce<true>(m, red, wq, lane);
+        delta = step_size(m);
+        if (et == 0) p.xs_out[row] = delta;
+    }
+    const float inv = recip_step(delta);
+    uint2* dst = reinterpret_cast<uint2*>(p.xq + (int64_t)row * p.K);
+    auto emit = [&](const uint4& xv, int v) {
+        float y[8];
+        if (ln) dec_ln_vec<T>(xv, g4, b4, v, rstd, shift, y);
+        else unpack8<T>(xv, y);
+        dst[v] = p.x_static ? quant8<true>(y, inv) : quant8<false>(y, inv);  // a given step may be exceeded: saturate
+    };
+#pragma unroll
+    for (int i = 0; i < QV; ++i) {
+        const int v = et + i * 128;
+        if (v < nvec) emit(c[i], v);
+    }
+    for (int v = et + QV * 128; v < nvec; v += 128) emit(__ldcg(src + v), v);
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* ptr) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ptr) : "memory");
+    return v;
+}
 
 // Per-channel constants of Eq. 2, fetched while the tile's weights are still streaming.
 struct DecChan { float ws, bs, rq; };
@@ -136,11 +303,13 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     uint64_t* empty_bar = full_bar + DEC_STAGES;
     uint64_t* tmem_full = empty_bar + DEC_STAGES;
     uint64_t* tmem_empty = tmem_full + 2;
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* x_ready = tmem_empty + 2;  // prologue quantiser: every token row has been written
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(x_ready + 1);
     volatile uint32_t* abort_flag = tmem_holder + 1;
     volatile uint32_t* epi_go = tmem_holder + 2;
     volatile uint32_t* epi_last = tmem_holder + 3;
     float* s_xs = reinterpret_cast<float*>(tmem_holder + 4);  // [DN] the tokens' step sizes
+    float* s_red = s_xs + DEC_N;                              // [4] reduction scratch of the prologue quantiser
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -155,6 +324,7 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             mbar_init(tmem_full + s, 1);
             mbar_init(tmem_empty + s, 128);
         }
+        mbar_init(x_ready, 1);
         *abort_flag = 0u;
         *epi_go = 0u;
         *epi_last = 0u;
@@ -193,6 +363,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                         tma_load_4d<1>(smem + i * DEC_STAGE, &tmap_w, full_bar + i, (kb0 + i) * BLOCK_K, ni * BLOCK_M, 0, 0);
                     }
                     pdl_wait();
+                    // with the quantiser in the prologue the codes of X exist once every CTA's rows are done
+                    if (p.x_raw != nullptr && !(ok = mbar_wait(x_ready, 0u, abort_flag, p.status, 11))) break;
                     for (int i = 0; i < n_pre; ++i)
                         tma_load_4d<1>(smem + i * DEC_STAGE + W_BYTES, &tmap_x, full_bar + i, (kb0 + i) * BLOCK_K, 0, 0, 0);
                     prefetched = n_pre;
@@ -253,13 +425,57 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         const int quarter = warp & 3;           // TMEM lanes this warp may read
         const int ch = quarter * 32 + lane;     // output channel within the tile
         const int et = threadIdx.x - 64;        // 0..127
-        if (et < DEC_N) s_xs[et] = (et < p.M && p.x_scale) ? __ldg(p.x_scale + (p.x_per_row ? et : 0)) : 1.0f;
+        bool x_ok = true;
+        if (p.x_raw != nullptr) {
+            // ---- activation quantiser: CTA r takes token rows r, r + grid, ... ----
+            uint32_t done = 0;
+            for (int row = (int)blockIdx.x; row < p.M; row += (int)gridDim.x, ++done) {
+                if (p.x_is_bf16) dec_quant_row<__nv_bfloat16>(p, row, et, s_red);
+                else dec_quant_row<__half>(p, row, et, s_red);
+            }
+            if (done) __threadfence();  // this thread's codes are visible device-wide before the count moves
+            dec_epi_sync();
+            if (et == 0) {
+                if (done) {
+                    asm volatile("fence.proxy.async.global;" ::: "memory");  // they will be read by bulk-tensor copies
+                    atomicAdd(p.sync, done);
+                }
+                // meet: all M rows written (bounded, like every other wait of the kernel)
+                const long long t0 = clock64();
+                bool ok = true;
+                while (ld_acquire_gpu(p.sync) < (uint32_t)p.M) {
+                    if (*abort_flag || (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) {
+                        ok = false;
+                        break;
+                    }
+                }
+                if (ok) {
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                    mbar_arrive(x_ready);  // the producer lane may fetch activation slices now
+                } else {
+                    *abort_flag = 1u;
+                    atomicCAS(p.status, 0u, ((uint32_t)SQ_ERR_TIMEOUT) | (10u << 8));
+                }
+                *epi_go = ok ? 1u : 0u;
+                // whoever passes last hands the two counters back zeroed (every CTA has added its rows
+                // before it came here, and nobody looks at them again)
+                if (atomicAdd(p.sync + 1, 1u) == gridDim.x - 1) {
+                    p.sync[0] = 0u;
+                    p.sync[1] = 0u;
+                }
+            }
+            dec_epi_sync();
+            x_ok = *epi_go != 0u;
+            dec_epi_sync();  // epi_go is rewritten in the loop below
+        }
+        // step sizes: the caller's, or the ones the prologue just wrote (read through L2)
+        if (et < DEC_N) s_xs[et] = (et < p.M && p.x_scale) ? __ldcg(p.x_scale + (p.x_per_row ? et : 0)) : p.alpha;
         dec_epi_sync();
         int slot = 0;
         uint32_t slot_phase = 0;
         int64_t pos = (int64_t)blockIdx.x * p.range;
         const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
-        while (pos < end) {
+        while (x_ok && pos < end) {
             const int ni = (int)(pos / p.num_kb);
             const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
             pos += kb1 - kb0;
@@ -370,7 +586,8 @@ sq_status launch_decode(const GemmArgs& a, const DecParams& p, int ctas, cudaStr
     CUtensorMap mw, mx;
     int s0, s1, s2;
     if (!make_map(&mw, a.B, 1, a.K, a.N, 1, 1, a.K, 0, 0, BLOCK_K, BLOCK_M, &s0, &s1, &s2)) return SQ_ERR_CUDA;
-    if (!make_map(&mx, a.A, 1, a.K, a.M, 1, 1, a.K, 0, 0, BLOCK_K, DN, &s0, &s1, &s2)) return SQ_ERR_CUDA;
+    const void* x_codes = p.x_raw != nullptr ? static_cast<const void*>(p.xq) : static_cast<const void*>(a.A);
+    if (!make_map(&mx, x_codes, 1, a.K, a.M, 1, 1, a.K, 0, 0, BLOCK_K, DN, &s0, &s1, &s2)) return SQ_ERR_CUDA;
     static bool attr_set[64] = {false};  // per instantiation and device
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
@@ -388,6 +605,12 @@ sq_status launch_decode(const GemmArgs& a, const DecParams& p, int ctas, cudaStr
 size_t decode_workspace_bytes(int64_t M, int64_t N) {
     const int64_t num_n = (N + tc::BLOCK_M - 1) / tc::BLOCK_M;
     return kWsHeader + kDecCounterBytes + (size_t)(kMaxCtas + 2 * num_n) * (size_t)M * tc::BLOCK_M * sizeof(int32_t);
+}
+
+// The same plus what the prologue quantiser writes: 256 bytes of step sizes, then the [M, K] codes.
+static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
+size_t decode_fused_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    return round256(decode_workspace_bytes(M, N)) + 256 + round256((size_t)M * (size_t)K);
 }
 
 // Up to 32 tokens the activation slices are a small addition to the weight stream and this kernel
@@ -413,6 +636,7 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.maxcount = plan.maxcount;
     p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
     p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
+    p.alpha = a.alpha;
     p.bias = a.bias; p.bias_is_bf16 = a.bias_dt == SQ_BF16;
     p.relu = a.relu;
     p.requant_mul = a.requant_mul; p.requant_per_col = a.requant_per_col;
@@ -421,6 +645,17 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.counters = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsHeader);
     p.part = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + kWsHeader + kDecCounterBytes);
     p.status = a.status;
+    p.x_raw = a.x_raw; p.x_is_bf16 = a.x_raw_dt == SQ_BF16;
+    p.ln_gamma = a.ln_gamma; p.ln_beta = a.ln_beta; p.ln_eps = a.ln_eps;
+    p.x_static = a.x_static;
+    p.xq = nullptr; p.xs_out = nullptr; p.stats_out = a.ln_stats_out; p.sync = nullptr;
+    if (a.x_raw != nullptr) {  // the caller (sq_api.cu) has checked that the workspace holds the scratch
+        char* scratch = static_cast<char*>(workspace) + round256(decode_workspace_bytes(a.M, a.N));
+        p.xs_out = a.xs_out != nullptr ? a.xs_out : reinterpret_cast<float*>(scratch);
+        p.xq = a.xq_out != nullptr ? a.xq_out : reinterpret_cast<int8_t*>(scratch + 256);
+        p.sync = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsSyncOff);
+        if (!a.x_static) { p.x_scale = p.xs_out; p.x_per_row = 1; }
+    }
     if (a.M <= 16) return launch_decode<16>(a, p, plan.ctas, st);
     return launch_decode<32>(a, p, plan.ctas, st);
 }

@@ -35,7 +35,10 @@ sq_status fold_ln_weight(const void* g, const void* b, sq_dtype dt, const float*
 sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul,
                     const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
                     float* scale, float* absmax_word, float* stats, int stats_are_input,
+                    uint32_t* status /*nullable: device status word for an expired bulk-copy wait*/,
                     cudaStream_t st);
+sq_status stream_full_dependency(cudaStream_t st);  // empty, fully serialised launch (see its definition)
+sq_status row_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st);
 bool row_pipeline_supports(int64_t M, int64_t C, bool ln, bool has_col_mul);
 sq_status row_pipeline(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul, const void* gamma,
                        const void* beta, float eps, bool ln, int mode, int8_t* Xq, float* scale, float* absmax_word,
@@ -66,6 +69,13 @@ struct GemmArgs {
     int64_t strideC[3];   // batch, head, row (elements)
     uint32_t* status;     // device status word (= workspace base)
     size_t ws_bytes;      // size of the caller's workspace
+    // Decode-shaped calls only (M <= 32): the activation quantiser runs in the GEMM's prologue.
+    // A is then ignored; the codes go to xq_out (nullable: scratch in the workspace).
+    const void* x_raw; sq_dtype x_raw_dt;     // [M, K] fp16 / bf16, contiguous
+    const void* ln_gamma; const void* ln_beta; float ln_eps;  // nullable: folded LayerNorm in front of Eq. 1
+    int x_static;                             // x_scale[0] is a given static step (else per-token dynamic)
+    int8_t* xq_out; float* xs_out;            // nullable outputs: codes [M, K], step sizes [M] (dynamic mode)
+    float* ln_stats_out;                      // nullable [2 M]
 };
 sq_status gemm_i8(const GemmArgs& a, cudaStream_t st);
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);  // scratch for the K split of the last wave
@@ -82,6 +92,8 @@ sq_status bounded_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t 
 
 // Decode-shaped path (M <= 16): swapped operands, split-K with INT32 scratch in the workspace.
 size_t decode_workspace_bytes(int64_t M, int64_t N);
+size_t decode_fused_workspace_bytes(int64_t M, int64_t N, int64_t K);  // + codes and step sizes of the prologue quantiser
+constexpr size_t kWsSyncOff = 32;     // decode-shaped GEMM with the quantiser in its prologue: two meeting counters
 bool decode_supports(const GemmArgs& a);
 sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaStream_t st);
 

@@ -125,7 +125,8 @@ kv_decode_attention_kernel(const KvParams p) {
     pdl_wait();  // q, the cache and the lengths may come from the preceding launch
     pdl_launch_dependents();
     int len = __ldg(p.lens + b);
-    if (len > p.max_len) {  // the caller's bound was wrong: say so, and stay inside what was sized
+    const bool truncated = len > p.max_len;
+    if (truncated) {  // the caller's bound was wrong: say so, and stay inside what was sized
         if (tid == 0 && crank == 0) atomicCAS(p.status, 0u, (uint32_t)SQ_ERR_SHAPE | (40u << 8));
         len = p.max_len;
     }
@@ -146,8 +147,10 @@ kv_decode_attention_kernel(const KvParams p) {
     const int n = max(0, min(len - key0, chunk));
     // With k_new / v_new the newest position (len - 1) is not in the cache yet: the CTA that owns
     // it takes its key and value from the new rows, stores them for later steps, and streams only
-    // the positions before it.
-    const bool owns_new = p.k_new != nullptr && n > 0 && key0 + n == len;
+    // the positions before it.  A truncated sequence appends nothing: position max_len - 1 holds a
+    // valid earlier key and value, which the newest token's must not overwrite; the output is then
+    // the attention over the first max_len cached positions.
+    const bool owns_new = !truncated && p.k_new != nullptr && n > 0 && key0 + n == len;
     const int nc = owns_new ? n - 1 : n;  // positions of this CTA that come from the cache
     const int nt = (nc + KV_TILE - 1) / KV_TILE;
     const int ntw = nt > w ? (nt - w + KV_WARPS - 1) / KV_WARPS : 0;  // tiles of this warp, per operand

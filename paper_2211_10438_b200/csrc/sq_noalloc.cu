@@ -64,8 +64,8 @@ extern "C" sq_status sq_ln_quant_tensor_noalloc(const void* X, sq_dtype dt, int6
     // (The statistics are fully overwritten by pass 1 before pass 2 reads them.)
     SQ_CUDA_OK(cudaMemsetAsync(word, 0, sizeof(float), st));
     s = row_quant(X, dt, M, C, nullptr, gamma_hat, beta_hat, eps, true, ROW_ABSMAX_ONLY, nullptr, nullptr, word,
-                  stats, 0, st);
+                  stats, 0, nullptr, st);
     if (s != SQ_OK) return s;
     return row_quant(X, dt, M, C, nullptr, gamma_hat, beta_hat, eps, true, ROW_FROM_ABSMAX_WORD, Xq, x_scale,
-                     word, stats, 1, st);
+                     word, stats, 1, nullptr, st);
 }

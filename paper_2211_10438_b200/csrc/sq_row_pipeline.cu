@@ -112,12 +112,23 @@ __device__ __forceinline__ void group_merge_stats(float& mean, float& m2, float 
     }
 }
 
-// 1/sqrt(v) for the LayerNorm statistic: the hardware approximation plus one Newton step (about
-// one unit in the last place; the statistic is a tolerance quantity, the element-wise part that
-// consumes it is the bit-exact one).
-__device__ __forceinline__ float rsqrt_refined(float v) {
-    const float r = rsqrtf(v), h = 0.5f * v;
-    return fmaf(r, fmaf(-h * r, r, 0.5f), r);
+// One thread's bounded wait for a row's bulk copy.  An expiry is recorded in the device status word
+// (when the caller gave a workspace to hold one) as SQ_ERR_TIMEOUT | 5 << 8; the group then stops.
+__device__ __forceinline__ bool wait_row(uint64_t* bar, uint32_t parity, uint32_t* status,
+                                         uint32_t budget = bulk::kWaitCycles) {
+    const bool ok = mbar_wait_bounded(bar, parity, budget);
+    if (!ok && status != nullptr) atomicCAS(status, 0u, (uint32_t)SQ_ERR_TIMEOUT | (5u << 8));
+    return ok;
+}
+
+// Self-test of that wait: a barrier nothing will ever complete, a small cycle budget.
+__global__ void row_wait_selftest_kernel(uint32_t* status, uint32_t budget) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        wait_row(&bar, 0u, status, budget);
+    }
 }
 
 // EXACT: the row has exactly GROUP * V vectors, so no per-vector bounds checks are needed.
@@ -203,9 +214,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
         // One thread waits (bounded) for the row's bulk copy; its outcome reaches the group through
         // shared memory so that every thread takes the same branch.
         if (gt == 0) {
-            const bool ok = mbar_wait_bounded(my_full + s, parity);
-            if (!ok && status != nullptr) atomicCAS(status, 0u, (uint32_t)SQ_ERR_TIMEOUT | (5u << 8));
-            *my_flag = ok ? 1u : 0u;
+            *my_flag = wait_row(my_full + s, parity, status) ? 1u : 0u;
         }
         group_sync<GROUP, CTA>(g);
         if (*my_flag == 0u) break;  // the copy never landed: stop this group
@@ -489,6 +498,11 @@ sq_status dispatch_pipe_mul(const void* X, int64_t M, int64_t C, const float* co
 }
 
 }  // namespace
+
+sq_status row_wait_selftest(uint32_t* status, uint32_t budget, cudaStream_t st) {
+    row_wait_selftest_kernel<<<1, 32, 0, st>>>(status, budget);
+    return launch_status();
+}
 
 bool row_pipeline_supports(int64_t M, int64_t C, bool ln, bool has_col_mul) {
     // LayerNorm and column-multiplied rows are held as fp32 (up to 32 768 elements); the plain

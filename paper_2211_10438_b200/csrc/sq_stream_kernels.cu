@@ -586,15 +586,26 @@ static sq_status launch_rows(const void* X, int64_t M, int64_t C, const float* c
     return launch_status();
 }
 
+// An empty kernel launched WITHOUT the programmatic-serialisation attribute: it starts only when
+// everything queued before it on the stream has completed and is visible.  Placed after a kernel
+// whose output a later dependent launch reads BEFORE its programmatic-dependency wait (the
+// decode-shaped GEMM prefetches weights that early), it closes that window.
+__global__ void full_dependency_kernel() {}
+
+sq_status stream_full_dependency(cudaStream_t st) {
+    full_dependency_kernel<<<1, 32, 0, st>>>();
+    return launch_status();
+}
+
 sq_status row_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* col_mul,
                     const void* gamma, const void* beta, float eps, bool ln, int mode, int8_t* Xq,
                     float* scale, float* absmax_word, float* stats, int stats_are_input,
-                    cudaStream_t st) {
+                    uint32_t* status, cudaStream_t st) {
     // the bulk-copy pipeline takes rows up to 32 768 elements (81 920 for the plain quantiser);
     // LayerNorm never comes with a column multiplier
     if (row_pipeline_supports(M, C, ln, col_mul != nullptr) && !(ln && col_mul != nullptr))
         return row_pipeline(X, dt, M, C, col_mul, gamma, beta, eps, ln, mode, Xq, scale, absmax_word, stats,
-                            stats_are_input, nullptr, st);
+                            stats_are_input, status, st);
 #define SQ_DISPATCH(T)                                                                           \
     (ln ? launch_rows<T, true, false>(X, M, C, nullptr, gamma, beta, eps, mode, Xq, scale,       \
                                       absmax_word, stats, stats_are_input, st)                   \

@@ -247,6 +247,51 @@ def test_decode_gemm_without_scratch_falls_back_to_single_split():
         sq.sq_w8a8_gemm(dev(Xq), dev(Wq), None, None, small, out_dtype=torch.int32)
 
 
+@pytest.mark.parametrize("M", [1, 16, 32])
+def test_single_matrix_bmm_with_few_rows_applies_alpha(M):
+    """A one-matrix BMM with contiguous operands and M <= 32 takes the weight-streaming kernel:
+    its scalar factor alpha (there are no step-size arrays in a BMM call) must reach the epilogue."""
+    N, K = 384, 512
+    A, B = synth.int8_tensor(27, 1, (M, K)), synth.int8_tensor(27, 2, (N, K))
+    alpha = np.float32(0.00731)
+    r = np.array([3.7], np.float32)
+    ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K))
+    want_acc, want16 = oracle.w8a8_bmm(A[None], B[None], float(alpha), out_dtype="f16")
+    _, want8 = oracle.w8a8_bmm(A[None], B[None], float(alpha), requant_mul=r)
+    Ad, Bd = dev(A), dev(B)
+    for tdt, want in ((torch.int32, want_acc[0]), (torch.float16, want16[0]), (torch.int8, want8[0])):
+        C = torch.empty((M, N), dtype=tdt, device="cuda")
+        sq.sq_w8a8_bmm(Ad, Bd, 1, 1, M, N, K, (M * K, M * K, K), (N * K, N * K, K), False, alpha, C, (M * N, M * N, N), ws,
+                       requant_mul=dev(r) if tdt == torch.int8 else None)
+        assert np.array_equal(host(C), want), str(tdt)
+    assert np.abs(want8).max() > 20 and sq.device_status(ws) == 0
+
+
+@pytest.mark.parametrize("gran", ["per_channel", "per_tensor"])
+def test_quant_weight_then_decode_gemm_back_to_back(gran):
+    """sq_quant_weight followed directly, on the same stream, by a decode-shaped sq_w8a8_gemm that
+    consumes its output: the GEMM starts fetching weights before it waits for its predecessor, so
+    the weight writer must be complete by then -- repeated to give an overlap the chance to show."""
+    M, N, K = 16, 4096, 4096
+    W = synth.weights(28, 1, N, K, "bf16")
+    s = synth.rng_for(28, 2).uniform(0.5, 2.0, K).astype(np.float32)
+    Xq = synth.int8_tensor(28, 3, (M, K))
+    want_Wq, want_ws = oracle.quant_weight(W, s, gran)
+    want = oracle.gemm_i32(Xq, want_Wq)
+    ws = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K))
+    Wd, sd, Xd = dev(W, "bf16"), dev(s), dev(Xq)
+    Wq = torch.empty((N, K), dtype=torch.int8, device="cuda")
+    wsc = torch.empty(N if gran == "per_channel" else 1, dtype=torch.float32, device="cuda")
+    acc = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    for it in range(5):
+        Wq.fill_(it + 1)  # stale codes a too-early fetch would pick up
+        sq.sq_quant_weight(Wd, sd, gran, Wq=Wq, w_scale=wsc, workspace=ws)
+        sq.sq_w8a8_gemm(Xd, Wq, None, None, ws, out=acc)
+        assert np.array_equal(host(acc), want), "iteration %d" % it
+    assert np.array_equal(host(Wq), want_Wq) and np.array_equal(host(wsc), want_ws)
+    assert sq.device_status(ws) == 0
+
+
 @pytest.mark.parametrize("out", ["f16", "i8", "i32"])
 def test_gemm_unaligned_output_rows(ws, out):
     # row stride that is not a multiple of 16 bytes: the epilogue writes rows directly instead of by TMA

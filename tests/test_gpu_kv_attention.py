@@ -182,6 +182,18 @@ def test_decode_attention_flags_a_length_beyond_the_stated_bound():
     # what it computed is the attention over the first max_len positions
     want, _ = oracle.kv_decode_attention(q, K, V, [128], np.float32(0.001), np.float32(0.001), out_dtype="f16")
     assert np.abs(host(out).reshape(B, H, D) - want).max() <= 3 * 127 * 0.001 + 1e-2 * np.abs(want).max()
+    # with the newest token's rows given, a truncated sequence appends nothing: the cache keeps its bytes
+    kc, vc = _cache_layout(K, V, L_max)
+    kd, vd = dev(kc), dev(vc)
+    k_new = synth.int8_tensor(66, 4, (B, H * D))
+    v_new = synth.int8_tensor(66, 5, (B, H * D))
+    ws = sq.new_workspace(256)
+    out2 = sq.sq_w8a8_decode_attention(dev(q.reshape(B, H * D)), kd, vd, dev(np.array([200], np.int32)), B, H, D, L_max, 128,
+                                       0.001, 0.001, ws, out_dtype=torch.float16, k_new=dev(k_new), v_new=dev(v_new))
+    torch.cuda.synchronize()
+    assert sq.device_status(ws) & 0xff == sq.SQ_ERR_SHAPE
+    assert np.array_equal(host(kd), kc) and np.array_equal(host(vd), vc)
+    assert torch.equal(out2, out)  # the attention over the first max_len cached positions, as without the new rows
     ws = sq.new_workspace(256)
     with pytest.raises(sq.SqError):  # host-side validation
         sq.sq_w8a8_decode_attention(dev(q.reshape(1, D)), dev(K), dev(V), dev(np.array([5], np.int32)), 1, 1, D, L_max, 512,

@@ -22,6 +22,26 @@ def test_bounded_wait_gives_up_and_reports():
     assert float(x.sum()) == 8.0
 
 
+def test_row_kernel_wait_gives_up_and_reports():
+    """The wait of the row kernels (quantisers, fused LayerNorm) for a row's bulk copy: on a barrier
+    nothing completes it expires, leaves SQ_ERR_TIMEOUT | 5 << 8 in the status word and returns."""
+    word = sq.sq_selftest_row_wait(budget_cycles=200000)
+    assert word == (sq.SQ_ERR_TIMEOUT | (5 << 8)), "status word %d" % word
+    assert float(torch.ones(8, device="cuda").sum()) == 8.0  # the context is still usable
+
+
+def test_row_kernels_leave_a_given_status_word_alone_when_nothing_expires():
+    """Per-token and static calls now take the workspace as their status word: a clean run leaves it zero."""
+    x = dev(synth.activations(1, 2, 40, 5120, "bf16", [3], [50.0]), "bf16")
+    g = torch.ones(5120, dtype=torch.bfloat16, device="cuda")
+    ws = sq.new_workspace(256)
+    sq.sq_quant_act(x, "per_token", workspace=ws)
+    sq.sq_ln_quant(x, g, None, 1e-5, "per_token", workspace=ws)
+    sq.sq_quant_act(x, "per_tensor_static", x_scale=torch.full((1,), 0.1, device="cuda"), workspace=ws)
+    torch.cuda.synchronize()
+    assert not ws.any()
+
+
 def _guarded(nbytes, dtype):
     """A uint8 arena with canaries; returns (arena, view of the payload as `dtype`)."""
     arena = torch.full((GUARD + nbytes + GUARD,), 0xA5, dtype=torch.uint8, device="cuda")

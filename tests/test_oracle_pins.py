@@ -236,6 +236,47 @@ def test_layernorm_against_torch_fp64():
     assert np.array_equal(q, q2) and np.array_equal(d, d2) and np.array_equal(yy, y32)
 
 
+@pytest.mark.parametrize("mean_over_sigma", [0.0, 10.0, 100.0])
+def test_ln_apply_error_bound_on_rows_with_a_large_mean(mean_over_sigma):
+    """The normative fp32 element-wise LayerNorm is n = fma(x, rstd, -(mu * rstd)), y = fma(n, g, b).
+    Its rounding error against the same expression in exact arithmetic is bounded, per element, by
+        2^-24 * [ (|mu * rstd| + |n|) * |g| + |y| ]            (one rounding each: the product mu * rstd,
+                                                                n, and y)
+    which grows with |mu| / sigma.  Pinned here on rows whose mean is 0, 10 and 100 standard deviations
+    away from zero, (a) against fp64 evaluation with the SAME fp32 statistics (isolates the element-wise
+    path), (b) against the fp64 LayerNorm with its own fp64 statistics, where the fp32 rounding of mu and
+    rstd alone may contribute (|mu * rstd| + |n|) * |g| * 2^-24 more.  A wrong sign, a dropped shift or
+    a swapped operand is off by ~|mu| / sigma and fails at once."""
+    rng = np.random.default_rng(1905 + int(mean_over_sigma))
+    C = 512
+    sigma = 0.75
+    x = (mean_over_sigma * sigma + sigma * rng.standard_normal((24, C))).astype(np.float16).astype(np.float32)
+    g = (1 + 0.1 * rng.standard_normal(C)).astype(np.float16).astype(np.float32)
+    b = (0.1 * rng.standard_normal(C)).astype(np.float16).astype(np.float32)
+    mu, rstd = oracle.ln_stats(x, 1e-5)
+    mu32, rstd32 = mu.astype(np.float32), rstd.astype(np.float32)
+    assert abs(np.abs(mu * rstd).mean() - mean_over_sigma) <= 0.1 * mean_over_sigma + 0.2  # the rows are what they claim
+    y32 = oracle.ln_apply(x, mu32, rstd32, g, b).astype(np.float64)
+    u = 2.0 ** -24
+    x64, g64, b64 = x.astype(np.float64), g.astype(np.float64), b.astype(np.float64)
+    # (a) same fp32 statistics, exact arithmetic
+    m64, r64 = mu32.astype(np.float64)[:, None], rstd32.astype(np.float64)[:, None]
+    n_same = x64 * r64 - m64 * r64
+    y_same = n_same * g64 + b64
+    bound_a = 1.01 * u * ((np.abs(m64 * r64) + np.abs(n_same)) * np.abs(g64) + np.abs(y_same))
+    assert np.all(np.abs(y32 - y_same) <= bound_a)
+    # (b) the fp64 LayerNorm (own statistics): add the rounding of mu and rstd to fp32
+    y_true = oracle.ln_f64(x, g64, b64, 1e-5)
+    n_true = (x64 - mu[:, None]) * rstd[:, None]
+    bound_b = bound_a + 1.01 * u * (np.abs(mu * rstd)[:, None] + 2 * np.abs(n_true)) * np.abs(g64)
+    assert np.all(np.abs(y32 - y_true) <= bound_b)
+    # the bound is what it says: of the order of (1 + |mu| / sigma) * 2^-24, far below a quantisation step
+    assert bound_b.max() <= (mean_over_sigma + 8) * 4 * u
+    # in code units: even at |mu| / sigma = 100 the error moves a value by < 1e-3 of a quantisation step
+    step = np.abs(y_true).max(axis=1, keepdims=True) / 127.0
+    assert (np.abs(y32 - y_true) / step).max() <= 1e-3
+
+
 # --------------------------------------------------------------------------- #
 # INT8 GEMM
 # --------------------------------------------------------------------------- #
