@@ -29,7 +29,7 @@ import numpy as np
 import torch
 
 WORKLOAD = 2  # OPT-13B-shaped prefill linears
-SAMPLE_ROWS_BASELINE = 1024
+SAMPLE_ROWS_BASELINE = 2048  # the whole config-2 problem
 SAMPLE_ROWS_REFERENCE = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per gemm_i8_kernel launch, mean over the four GEMMs of one step,
 # from the ncu capture summarised in profiles/gemm_i8_kernel__opt13b_prefill.md
@@ -149,21 +149,27 @@ def timed_rows(device, peaks):
     from paper_2211_10438_b200 import pipeline as pl
     rows = {}
 
-    def t(fn, n=10):
+    def t(fn, n=10, clocks=None):
         torch.cuda.synchronize()
         time.sleep(0.2)  # let the clocks recover from the previous row: every row starts from idle
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
+        sampler = None
+        if clocks is not None:  # rows of many milliseconds sag under the power cap: sample the SM clock beside them
+            sampler = ClockSampler(device.index or 0)
+            sampler.start()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         for _ in range(n):
             fn()
         b.record()
         torch.cuda.synchronize()
+        if sampler is not None:
+            clocks.update(sampler.stop())
         return a.elapsed_time(b) / n * 1e-3
 
-    ws = sq.new_workspace(max(1 << 20, sq.workspace_bytes(sq.SQ_OP_GEMM, 16, 49152, 49152)), device)
+    ws = sq.new_workspace(max(1 << 20, sq.workspace_bytes(sq.SQ_OP_LN_QUANT, 16384, 0, 20480)), device)
     # MT-NLG-shaped streaming rows (inputs 671 MB > L2)
     M, C = 16384, 20480
     x = torch.randn((M, C), device=device, dtype=torch.bfloat16)
@@ -177,12 +183,17 @@ def timed_rows(device, peaks):
     rows["quant_act_per_token_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
     s = t(lambda: sq.sq_ln_quant(x, g, b, 1e-5, "per_token", Xq=Xq, x_scale=xs, workspace=ws))
     rows["ln_quant_per_token_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    xs1 = torch.full((1,), 0.05, dtype=torch.float32, device=device)
+    s = t(lambda: sq.sq_ln_quant(x, g, b, 1e-5, "per_tensor_static", Xq=Xq, x_scale=xs1, workspace=ws))
+    rows["ln_quant_per_tensor_static_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
+    s = t(lambda: sq.sq_ln_quant(x, g, b, 1e-5, "per_tensor_dynamic", Xq=Xq, x_scale=xs1, workspace=ws))
+    rows["ln_quant_per_tensor_dynamic_16384x20480"] = {"GB/s": 5 * M * C / s / 1e9, "frac_hbm": 5 * M * C / s / 1e9 / peaks["hbm_gbs"],
+                                                       "us": s * 1e6}
     s = t(lambda: sq.sq_calib_absmax(x, a))
     rows["calib_absmax_16384x20480"] = {"GB/s": 2 * M * C / s / 1e9, "frac_hbm": 2 * M * C / s / 1e9 / peaks["hbm_gbs"]}
     # the other two activation granularities of Table 2: one step for the whole tensor, given
     # (static, 3 B/element) or found by a first pass over the tensor (dynamic, 5 B/element here:
     # 671 MB does not stay in L2 between the passes)
-    xs1 = torch.full((1,), 0.05, dtype=torch.float32, device=device)
     s = t(lambda: sq.sq_quant_act(x, "per_tensor_static", Xq=Xq, x_scale=xs1, workspace=ws))
     rows["quant_act_per_tensor_static_16384x20480"] = {"GB/s": 3 * M * C / s / 1e9, "frac_hbm": 3 * M * C / s / 1e9 / peaks["hbm_gbs"]}
     s = t(lambda: sq.sq_quant_act(x, "per_tensor_dynamic", Xq=Xq, x_scale=xs1, workspace=ws))
@@ -232,36 +243,48 @@ def timed_rows(device, peaks):
             "GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6,
             "cache_bytes_fp16_would_be": 2 * (byts - 4 * Bk * H * D)}
         del kc, vc
-    # decode-shaped GEMMs at GPT-3 / OPT-175B shapes (weights 453-604 MB > L2); per-token dynamic
-    # quantisation of the bf16 input runs in front of the GEMM and is inside the timed call
+    # decode-shaped GEMMs at GPT-3 / OPT-175B shapes (weights 453-604 MB > L2), bf16 activations in,
+    # bf16 out: per-token dynamic quantisation runs in the GEMM kernel's prologue (one launch per
+    # call, 50 timed calls per row); `gemm_alone_us` is the same GEMM on codes quantised beforehand
+    ws = sq.new_workspace(max(1 << 20, sq.workspace_bytes(sq.SQ_OP_GEMM_FUSED_QUANT, 16, 49152, 49152)), device)
     for name, (N, K) in (("qkv", (36864, 12288)), ("fc1", (49152, 12288)), ("fc2", (12288, 49152))):
         Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device=device)
         wsd = torch.rand(N, device=device) * 0.001
-        for Md in (1, 16):
+        for Md in (1, 2, 4, 8, 16):
             xd = torch.randn((Md, K), device=device, dtype=torch.bfloat16)
-            Xd = torch.empty((Md, K), dtype=torch.int8, device=device)
-            xsd = torch.empty(Md, dtype=torch.float32, device=device)
             Y = torch.empty((Md, N), dtype=torch.bfloat16, device=device)
-
-            def call():
-                sq.sq_quant_act(xd, "per_token", Xq=Xd, x_scale=xsd, workspace=ws)
-                sq.sq_w8a8_gemm(Xd, Wq, xsd, wsd, ws, out=Y)
-            s = t(call)
+            s = t(lambda: sq.sq_w8a8_gemm_fused_quant(xd, Wq, wsd, ws, "per_token", out=Y), n=50)
             byts = N * K + 3 * Md * K + 2 * Md * N
-            rows["decode_%s_M%d_%dx%d" % (name, Md, N, K)] = {
-                "GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6}
+            row = {"GB/s": byts / s / 1e9, "frac_hbm": byts / s / 1e9 / peaks["hbm_gbs"], "us": s * 1e6, "launches": 1}
+            if Md in (1, 16):
+                Xd, xsd = sq.sq_quant_act(xd, "per_token")
+                row["gemm_alone_us"] = t(lambda: sq.sq_w8a8_gemm(Xd, Wq, xsd, wsd, ws, out=Y), n=50) * 1e6
+            rows["decode_%s_M%d_%dx%d" % (name, Md, N, K)] = row
         del Wq
-    # MT-NLG-shaped prefill GEMM (FC1 81920 x 20480 at M = 4096): 13.7 TOP per launch
-    M5, N5, K5 = 4096, 81920, 20480
-    Wq = torch.randint(-127, 128, (N5, K5), dtype=torch.int8, device=device)
-    X5 = torch.randint(-127, 128, (M5, K5), dtype=torch.int8, device=device)
-    xs5 = torch.rand(M5, device=device) * 0.1
-    ws5 = torch.rand(N5, device=device) * 0.001
-    Y5 = torch.empty((M5, N5), dtype=torch.bfloat16, device=device)
-    s = t(lambda: sq.sq_w8a8_gemm(X5, Wq, xs5, ws5, ws, out=Y5), n=5)
-    rows["prefill_gemm_mtnlg_fc1_M4096"] = {"TOPS": 2 * M5 * N5 * K5 / s / 1e12, "us": s * 1e6,
-                                            "frac_of_2x_bf16_sustained": 2 * M5 * N5 * K5 / s / 1e12 / (2 * peaks["bf16_sustained"])}
-    del Wq, X5, Y5
+    # MT-NLG-shaped prefill sweep (config 5): the four GEMMs at M = 4096 / 8192 / 16384, bf16 out,
+    # per-token x per-channel step sizes.  Launches of 3 to 20 ms run into the power cap: the SM clock
+    # sampled during each row is reported, and the time scaled to the full clock beside it.
+    for name, (N5, K5) in (("qkv", (61440, 20480)), ("out_proj", (20480, 20480)), ("fc1", (81920, 20480)),
+                           ("fc2", (20480, 81920))):
+        Wq = torch.randint(-127, 128, (N5, K5), dtype=torch.int8, device=device)
+        ws5 = torch.rand(N5, device=device) * 0.001
+        for M5 in (4096, 8192, 16384):
+            X5 = torch.randint(-127, 128, (M5, K5), dtype=torch.int8, device=device)
+            xs5 = torch.rand(M5, device=device) * 0.1
+            Y5 = torch.empty((M5, N5), dtype=torch.bfloat16, device=device)
+            wsg = sq.new_workspace(sq.workspace_bytes(sq.SQ_OP_GEMM, M5, N5, K5), device)
+            ck = {}
+            s = t(lambda: sq.sq_w8a8_gemm(X5, Wq, xs5, ws5, wsg, out=Y5), n=5, clocks=ck)
+            tops = 2 * M5 * N5 * K5 / s / 1e12
+            mhz = ck.get("sm_mhz") or 0.0
+            rows["prefill_gemm_mtnlg_%s_M%d" % (name, M5)] = {
+                "TOPS": tops, "us": s * 1e6, "sm_mhz": mhz, "reasons": ck.get("reasons"),
+                "frac_of_2x_bf16_sustained": tops / (2 * peaks["bf16_sustained"]),
+                "frac_of_2x_bf16_burst": tops / (2 * peaks["bf16_burst"]),
+                "us_x_mhz_over_max": s * 1e6 * mhz / ck["sm_max_mhz"] if mhz and ck.get("sm_max_mhz") else None,
+                "status": sq.device_status(wsg)}
+            del X5, Y5, wsg
+        del Wq
     rows.update(block_rows(device))
     return rows
 
@@ -330,11 +353,13 @@ def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, 
     from paper_2211_10438_b200 import pipeline as pl
     from paper_2211_10438_b200 import binding as sq
     L_max = 2048
-    gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, dt)
-    gen.load_prompt(prompt_blk.qkv, S)
     x = pl.synth_device_activations(B, hid, dt, ch, fac, seed + 90, device)
     out = {}
-    for ctx in (S, L_max - 1):
+    # seven launches (residual adds in the GEMM epilogues) is the library's default; the five-launch form
+    # with the LayerNorm+quantise steps in the GEMM prologues is timed beside it
+    for fused, ctx in ((False, S), (False, L_max - 1), (True, S)):
+        gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, dt, fused=fused)
+        gen.load_prompt(prompt_blk.qkv, S)
         gen.ctx.fill_(ctx)
         gen.lens.fill_(ctx + 1)
         for _ in range(3):
@@ -348,7 +373,7 @@ def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, 
             g.replay()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n = 20
+        n = 50
         a.record()
         for _ in range(n):
             g.replay()
@@ -356,10 +381,10 @@ def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, 
         torch.cuda.synchronize()
         us = a.elapsed_time(b) / n * 1e3
         byts = gen.bytes_per_step(ctx * B)
-        out["opt30b_generation_b%d_ctx%d" % (B, ctx)] = {
+        out["opt30b_generation_b%d_ctx%d%s" % (B, ctx, "_five_launches" if fused else "")] = {
             "us_per_layer": us, "GB/s": byts / us / 1e3, "frac_hbm": byts / us / 1e3 / measured_peaks()["hbm_gbs"],
-            "status": sq.device_status(gen.ws)}
-        del g
+            "launches": gen.launches_per_step, "status": sq.device_status(gen.ws)}
+        del g, gen
     return out
 
 

@@ -70,7 +70,8 @@ typedef enum {
     SQ_OP_LN_QUANT = 1,
     SQ_OP_QUANT_WEIGHT = 2,
     SQ_OP_GEMM = 3,
-    SQ_OP_BMM = 4
+    SQ_OP_BMM = 4,
+    SQ_OP_GEMM_FUSED_QUANT = 5
 } sq_op;
 
 /* Largest reduction length for which |sum| <= 127*127*K stays inside INT32. */
@@ -268,6 +269,39 @@ sq_status sq_w8a8_gemm_residual(const int8_t* Xq, const int8_t* Wq, int64_t M, i
                                 int w_scale_is_per_channel, const void* bias, sq_dtype bias_dt,
                                 const void* residual, int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy,
                                 void* workspace, size_t ws_bytes, void* stream);
+
+/*
+ * The generation-stage W8A8 linear (M <= 32 tokens) with the activation quantiser INSIDE the GEMM
+ * kernel.  With a handful of tokens the layer is a single pass over the INT8 weights (the paper's
+ * appendix on weight-only quantisation: this stage is memory-bound), and a quantiser launched in
+ * front of it costs a tenth of that pass; here the kernel's first weight slices are already in
+ * flight while thread block r turns token row r into INT8 codes:
+ *     [ y = LayerNorm(x; gamma_hat, beta_hat, eps)      when gamma_hat != NULL, as sq_ln_quant ]
+ *     Delta_t = max_j |y[t, j]| / 127 (SQ_PER_TOKEN_DYNAMIC)   or   Delta = x_scale[0] (SQ_PER_TENSOR_STATIC)
+ *     Xq = clamp(round(y * (1 / Delta)), -127, 127)                                        (Eq. 1)
+ * followed by exactly the arithmetic of sq_w8a8_gemm / sq_w8a8_gemm_residual (Eq. 2, bias, ReLU,
+ * re-quantisation, residual add).  Codes and step sizes equal those of sq_quant_act (bit for bit)
+ * and of sq_ln_quant (bit for bit given the same row statistics; the statistics are a two-pass fp32
+ * reduction in another order, a tolerance quantity).
+ * X: [M, K] of x_dt (F16/BF16), contiguous, 16-byte aligned; K a multiple of 16, K <= SQ_MAX_K.
+ * gamma_hat, beta_hat: [K] of x_dt or NULL (beta_hat may be NULL alone).  g: SQ_PER_TOKEN_DYNAMIC or
+ * SQ_PER_TENSOR_STATIC; SQ_PER_TENSOR_DYNAMIC and M > 32 return SQ_ERR_UNSUPPORTED (use sq_quant_act /
+ * sq_ln_quant followed by sq_w8a8_gemm).  x_scale: static: [1] INPUT; dynamic: optional [M] OUTPUT
+ * (NULL keeps the step sizes in the workspace).  Xq_out: optional [M, K] int8 OUTPUT, 16-byte aligned
+ * (NULL keeps the codes in the workspace).  dbg_mean_rstd: optional [2 M] fp32, as in sq_ln_quant.
+ * residual (nullable): as in sq_w8a8_gemm_residual (then out_dt is F16/BF16, no ReLU / re-quantisation).
+ * out_dt: SQ_F16 / SQ_BF16 / SQ_I8.  Other arguments as sq_w8a8_gemm.
+ * workspace: sq_workspace_bytes(SQ_OP_GEMM_FUSED_QUANT, M, N, K) bytes, REQUIRED.  The thread blocks
+ * of the call meet once on a counter in it (bounded wait; on expiry SQ_ERR_TIMEOUT | 10 << 8 or
+ * | 11 << 8 in the status word), so two calls that can overlap on the GPU must not share a workspace.
+ */
+sq_status sq_w8a8_gemm_fused_quant(const void* X, sq_dtype x_dt, int64_t M, int64_t N, int64_t K,
+                                   const void* gamma_hat, const void* beta_hat, float eps, sq_act_gran g,
+                                   float* x_scale, int8_t* Xq_out, float* dbg_mean_rstd, const int8_t* Wq,
+                                   const float* w_scale, int w_scale_is_per_channel, const void* bias,
+                                   sq_dtype bias_dt, sq_epilogue_act act, const float* requant_mul,
+                                   int requant_is_per_channel, const void* residual, int64_t ld_res, void* Y,
+                                   sq_dtype out_dt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream);
 
 /*
  * INT8 batched matmul for attention (Fig. 6: the BMMs run in INT8):

@@ -20,7 +20,7 @@ SQ_F16, SQ_BF16, SQ_I8, SQ_I32 = 0, 1, 2, 3
 SQ_PER_TENSOR_STATIC, SQ_PER_TENSOR_DYNAMIC, SQ_PER_TOKEN_DYNAMIC = 0, 1, 2
 SQ_W_PER_TENSOR, SQ_W_PER_CHANNEL = 0, 1
 SQ_EPI_NONE, SQ_EPI_RELU = 0, 1
-SQ_OP_QUANT_ACT, SQ_OP_LN_QUANT, SQ_OP_QUANT_WEIGHT, SQ_OP_GEMM, SQ_OP_BMM = 0, 1, 2, 3, 4
+SQ_OP_QUANT_ACT, SQ_OP_LN_QUANT, SQ_OP_QUANT_WEIGHT, SQ_OP_GEMM, SQ_OP_BMM, SQ_OP_GEMM_FUSED_QUANT = 0, 1, 2, 3, 4, 5
 SQ_MAX_K = 133144
 SQ_NOALLOC_MAX_ROWS = 16384
 
@@ -28,7 +28,7 @@ EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm", "sq_w8a8_gemm_residual",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
            "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention",
-           "sq_token_absmax", "sq_clipped_absmax", "sq_selftest_row_wait"]
+           "sq_token_absmax", "sq_clipped_absmax", "sq_selftest_row_wait", "sq_w8a8_gemm_fused_quant"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -68,6 +68,8 @@ def lib():
                                    vp, i32, i64, vp, sz, vp]
         L.sq_w8a8_gemm_residual.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, i32, vp, i32, vp, i64, vp, i32, i64,
                                             vp, sz, vp]
+        L.sq_w8a8_gemm_fused_quant.argtypes = [vp, i32, i64, i64, i64, vp, vp, f32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32,
+                                               vp, i32, vp, i64, vp, i32, i64, vp, sz, vp]
         L.sq_w8a8_bmm.argtypes = [vp, vp, i64, i64, i64, i64, i64, c.POINTER(i64), c.POINTER(i64), i32, i32,
                                   f32, vp, vp, i32, c.POINTER(i64), vp, sz, vp]
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
@@ -227,6 +229,29 @@ def sq_w8a8_gemm_residual(Xq, Wq, x_scale, w_scale, workspace, residual, bias=No
         _ptr(w_scale), 1 if (w_scale is not None and w_scale.numel() > 1) else 0, _ptr(bias),
         _DT[bias.dtype] if bias is not None else SQ_F16, _ptr(residual), residual.stride(0),
         _ptr(out), _DT[out.dtype], out.stride(0), wp, wn, _stream()), "sq_w8a8_gemm_residual")
+    return out
+
+
+def sq_w8a8_gemm_fused_quant(X, Wq, w_scale, workspace, gran="per_token", x_scale=None, gamma_hat=None, beta_hat=None,
+                             eps=1e-5, Xq_out=None, dbg_mean_rstd=None, bias=None, relu=False, requant_mul=None,
+                             residual=None, out=None, out_dtype=None):
+    """Decode-shaped W8A8 linear (M <= 32) on 16-bit activations: Eq. 1 (optionally behind the folded
+    LayerNorm) runs in the GEMM kernel's prologue.  gran: "per_token" (x_scale: optional [M] output) or
+    "per_tensor_static" (x_scale: [1] input)."""
+    M, K = X.shape
+    N = Wq.shape[0]
+    g = GRAN[gran] if isinstance(gran, str) else gran
+    if out is None:
+        odt = out_dtype or (torch.int8 if requant_mul is not None else (residual.dtype if residual is not None else X.dtype))
+        out = torch.empty((M, N), dtype=odt, device=X.device)
+    wp, wn = _ws(workspace)
+    _check(lib().sq_w8a8_gemm_fused_quant(
+        _ptr(X), _DT[X.dtype], M, N, K, _ptr(gamma_hat), _ptr(beta_hat), float(eps), g, _ptr(x_scale), _ptr(Xq_out),
+        _ptr(dbg_mean_rstd), _ptr(Wq), _ptr(w_scale), 1 if w_scale.numel() > 1 else 0, _ptr(bias),
+        _DT[bias.dtype] if bias is not None else SQ_F16, SQ_EPI_RELU if relu else SQ_EPI_NONE, _ptr(requant_mul),
+        1 if (requant_mul is not None and requant_mul.numel() > 1) else 0, _ptr(residual),
+        residual.stride(0) if residual is not None else 0, _ptr(out), _DT[out.dtype], out.stride(0), wp, wn, _stream()),
+        "sq_w8a8_gemm_fused_quant")
     return out
 
 

@@ -29,6 +29,15 @@ def _stale(target, deps):
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def build_trace() -> str:
+    """Tuning build: libsq_trace.so, the same library with the decode-shaped GEMM's timestamp trace
+    compiled in (-DSQ_DEC_TRACE).  Never loaded by the binding unless LIB_PATH is pointed at it."""
+    out = os.path.join(HERE, "libsq_trace.so")
+    subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSQ_DEC_TRACE", "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out],
+                   check=True)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "sq.h"))
@@ -59,4 +68,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--trace" in sys.argv:
+        print(build_trace())
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

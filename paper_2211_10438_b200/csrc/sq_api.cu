@@ -71,6 +71,9 @@ size_t sq_workspace_bytes(sq_op op, int64_t M, int64_t N, int64_t K) {
             if (!(M > 0 && N > 0 && K > 0)) return kWsHeader;
             if (M <= 32) return decode_workspace_bytes(M, N);
             return gemm_workspace_bytes(M, N, K);
+        case SQ_OP_GEMM_FUSED_QUANT:  // the same + the codes and step sizes of the prologue quantiser
+            if (!(M > 0 && M <= 32 && N > 0 && K > 0)) return kWsHeader;
+            return decode_fused_workspace_bytes(M, N, K);
         case SQ_OP_QUANT_ACT:
         case SQ_OP_QUANT_WEIGHT:
         case SQ_OP_BMM: return kWsHeader;
@@ -241,6 +244,63 @@ sq_status sq_w8a8_gemm_residual(const int8_t* Xq, const int8_t* Wq, int64_t M, i
     if (!residual) return SQ_ERR_INVALID_ARG;
     return w8a8_gemm_impl(Xq, Wq, M, N, K, x_scale, x_scale_is_per_token, w_scale, w_scale_is_per_channel, bias, bias_dt,
                           SQ_EPI_NONE, nullptr, 0, nullptr, residual, ld_res, Y, out_dt, ldy, workspace, ws_bytes, stream);
+}
+
+sq_status sq_w8a8_gemm_fused_quant(const void* X, sq_dtype x_dt, int64_t M, int64_t N, int64_t K,
+                                   const void* gamma_hat, const void* beta_hat, float eps, sq_act_gran g,
+                                   float* x_scale, int8_t* Xq_out, float* dbg_mean_rstd, const int8_t* Wq,
+                                   const float* w_scale, int w_scale_is_per_channel, const void* bias,
+                                   sq_dtype bias_dt, sq_epilogue_act act, const float* requant_mul,
+                                   int requant_is_per_channel, const void* residual, int64_t ld_res, void* Y,
+                                   sq_dtype out_dt, int64_t ldy, void* workspace, size_t ws_bytes, void* stream) {
+    if (!is_act_dtype(x_dt) || (g != SQ_PER_TENSOR_STATIC && g != SQ_PER_TOKEN_DYNAMIC && g != SQ_PER_TENSOR_DYNAMIC))
+        return SQ_ERR_INVALID_ARG;
+    if (M < 0 || N < 0 || K < 0) return SQ_ERR_SHAPE;
+    if (out_dt < SQ_F16 || out_dt > SQ_I8 || (act != SQ_EPI_NONE && act != SQ_EPI_RELU)) return SQ_ERR_INVALID_ARG;
+    if (gamma_hat != nullptr && !(eps >= 0.0f)) return SQ_ERR_INVALID_ARG;
+    if (gamma_hat == nullptr && (beta_hat != nullptr || dbg_mean_rstd != nullptr)) return SQ_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return SQ_OK;
+    if (K == 0) return SQ_ERR_SHAPE;
+    // one step for the whole tensor would need a second meeting of the CTAs; beyond 32 tokens the
+    // quantiser is a pass of its own: both go through sq_quant_act / sq_ln_quant + sq_w8a8_gemm
+    if (M > 32 || g == SQ_PER_TENSOR_DYNAMIC || K > SQ_MAX_K) return SQ_ERR_UNSUPPORTED;
+    if (ldy < N) return SQ_ERR_SHAPE;
+    if (!X || !Wq || !Y || !w_scale) return SQ_ERR_INVALID_ARG;
+    if (g == SQ_PER_TENSOR_STATIC && !x_scale) return SQ_ERR_INVALID_ARG;
+    if ((out_dt == SQ_I8) != (requant_mul != nullptr)) return SQ_ERR_INVALID_ARG;
+    if (bias && !is_act_dtype(bias_dt)) return SQ_ERR_INVALID_ARG;
+    if (K % 16 != 0 || !aligned16(X) || !aligned16(Wq) || (Xq_out && !aligned16(Xq_out)) ||
+        (gamma_hat && !aligned16(gamma_hat)) || (beta_hat && !aligned16(beta_hat)))
+        return SQ_ERR_ALIGN;
+    if (residual) {
+        if (!is_act_dtype(out_dt)) return SQ_ERR_INVALID_ARG;
+        if (ld_res < N) return SQ_ERR_SHAPE;
+        if (!aligned16(residual) || ld_res % 8 != 0 || N % 8 != 0) return SQ_ERR_ALIGN;
+    }
+    if (!ws_ok(workspace, ws_bytes, sq_workspace_bytes(SQ_OP_GEMM_FUSED_QUANT, M, N, K))) return SQ_ERR_WORKSPACE;
+    GemmArgs a{};
+    a.ws_bytes = ws_bytes;
+    a.A = nullptr; a.B = Wq;
+    a.batch = 1; a.heads = 1; a.M = M; a.N = N; a.K = K;
+    a.strideA[0] = M * K; a.strideA[1] = M * K; a.strideA[2] = K;
+    a.strideB[0] = N * K; a.strideB[1] = N * K; a.strideB[2] = K;
+    a.x_scale = x_scale; a.x_per_row = g == SQ_PER_TOKEN_DYNAMIC;
+    a.w_scale = w_scale; a.w_per_col = w_scale_is_per_channel;
+    a.alpha = 1.0f;
+    a.bias = bias; a.bias_dt = bias_dt;
+    a.relu = act == SQ_EPI_RELU;
+    a.requant_mul = requant_mul; a.requant_per_col = requant_is_per_channel;
+    a.residual = residual; a.ld_res = ld_res;
+    a.C = Y; a.out_dt = out_dt;
+    a.strideC[2] = ldy;
+    a.status = reinterpret_cast<uint32_t*>(workspace);
+    a.x_raw = X; a.x_raw_dt = x_dt;
+    a.ln_gamma = gamma_hat; a.ln_beta = beta_hat; a.ln_eps = eps;
+    a.x_static = g == SQ_PER_TENSOR_STATIC;
+    a.xq_out = Xq_out;
+    a.xs_out = g == SQ_PER_TOKEN_DYNAMIC ? x_scale : nullptr;
+    a.ln_stats_out = dbg_mean_rstd;
+    return decode_gemm(a, workspace, ws_bytes, as_stream(stream));
 }
 
 sq_status sq_w8a8_bmm(const int8_t* A, const int8_t* B, int64_t batch, int64_t heads, int64_t M, int64_t N,

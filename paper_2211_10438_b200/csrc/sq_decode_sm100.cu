@@ -4,9 +4,10 @@
 //   * operands are swapped: 128 OUTPUT CHANNELS of W (128 x 128 bytes per K slice) ride on the
 //     MMA's M dimension and the tokens on its N dimension (tcgen05.mma.kind::i8, 128 x 16 x 32
 //     or 128 x 32 x 32), so no tile is padded from 16 to 128 rows and a stage is 18 or 20 KB;
-//   * the (128-channel tile, K block) pairs, tile-major, are cut into equal contiguous ranges,
-//     one per CTA ("stream-K"): every SM streams the same number of weight bytes whatever N
-//     and K are, at the price of tiles whose K range is shared by two or more CTAs;
+//   * every CTA gets the same number of K blocks whatever N and K are: as many whole 128-channel
+//     tiles as divide evenly among the CTAs, plus an equal contiguous range of the remaining
+//     tiles' (tile, K block) pairs, tile-major ("stream-K"), whose K ranges are then shared by
+//     two or more CTAs.  The shared part is done first, the whole tiles last;
 //   * a 10-stage TMA ring keeps ~180 KB of weights in flight per SM;
 //   * a CTA parks the partial accumulators of a shared tile in its own slot of the workspace
 //     with plain stores (INT32 partial sums add exactly in any order); the CTA that arrives
@@ -14,11 +15,15 @@
 //     (dequant, bias, ReLU, requant), writes Y and leaves the counter zeroed for the next call.
 //   * optionally the activation quantiser runs INSIDE this kernel (Eq. 1 per token, or with a given
 //     static step; optionally behind the folded LayerNorm): while every CTA's first weight slices
-//     are already in flight, CTA r quantises token row r (16-bit values -> INT8 codes + step size,
-//     written to scratch in the workspace), the CTAs meet on one counter, and only then are the
-//     activation slices fetched.  The quantiser's cost hides behind the first fill of the ring
-//     instead of being a launch of its own in front of the GEMM.
+//     are already in flight, CTA r pulls token row r into the top of its own ring with one bulk
+//     copy and quantises it (16-bit values -> INT8 codes + step size), the CTAs meet on one
+//     counter, and only then are the activation slices fetched.  The codes are parked in the
+//     workspace K block by K block, each block already in the 128-byte-swizzled image the MMA
+//     reads, so an activation slice is ONE contiguous bulk copy per stage instead of a strided
+//     box of 16 or 32 rows.  The quantiser's cost hides behind the first fill of the ring instead
+//     of being a launch of its own in front of the GEMM.
 // Every wait is bounded (status word, as in the prefill kernel).
+#include "sq_bulk.cuh"
 #include "sq_kernels.h"
 #include "sq_tcgen05.cuh"
 
@@ -29,6 +34,10 @@ namespace {
 using namespace tc;
 
 constexpr int DEC_THREADS = 192;      // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: epilogue
+constexpr int DEC_QUANT_THREADS = 256;  // prologue quantiser: the epilogue warps + 4 helper warps (more warps hide
+                                        // the latency of its dependent instruction chains; 12 would cap the kernel
+                                        // at 128 registers per thread and spill the 32-token epilogue)
+constexpr int DEC_THREADS_FUSED = 64 + DEC_QUANT_THREADS;
 constexpr int DEC_MAX_N = 32;         // most tokens this kernel takes
 constexpr int W_BYTES = BLOCK_M * BLOCK_K;  // 16 KB of weights per stage
 // DN = tokens per MMA (its N dimension): 16 or 32.  A stage holds 16 KB of weights and
@@ -39,16 +48,37 @@ struct DecCfg {
     static constexpr int STAGE = W_BYTES + X_BYTES;
     static constexpr int STAGES = 10;
     static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
-    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 5) * 8 + 64 + DN * 4 + 32;
+    static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 7) * 8 + 64 + DN * 4 + 64;
 };
+
+// Tuning aid, compiled out unless SQ_DEC_TRACE is defined (python -m paper_2211_10438_b200.build --trace
+// builds libsq_trace.so): one thread per role stores its SM's cycle counter at fixed points of a
+// CTA's life (reading the global nanosecond timer costs a fraction of a microsecond per read and
+// would inflate every interval; cycle counters of different SMs are not aligned, so only differences
+// within a CTA mean anything); sq_debug_decode_trace() copies the table of the last launch to the
+// host and clears it.
+#ifdef SQ_DEC_TRACE
+constexpr int kTraceSlots = 16, kTraceLaunches = 8;
+__device__ unsigned long long g_dec_trace[kTraceLaunches][256][kTraceSlots];  // the last 8 launches, round robin
+__device__ __forceinline__ void dec_trace(int launch, int slot) {
+    g_dec_trace[launch][blockIdx.x][slot] = (unsigned long long)clock64();
+}
+#define DEC_TRACE(slot) dec_trace(p.trace_id, slot)
+#else
+#define DEC_TRACE(slot) ((void)0)
+#endif
 
 struct DecParams {
     int M;
     int64_t N, K;
     int num_n, num_kb;
-    int64_t total_kb;    // num_n * num_kb: every (tile, K block) pair, tile-major
-    int range;           // K blocks per CTA: CTA g owns positions [g * range, (g + 1) * range)
+    int64_t total_kb;    // sk_tiles * num_kb: the (tile, K block) pairs of the shared tiles, tile-major
+    int range;           // of those, K blocks per CTA: CTA g owns positions [g * range, (g + 1) * range)
     int maxcount;        // most CTAs that share one tile
+    int trace_id;        // SQ_DEC_TRACE builds: which of the trace tables this launch writes
+    int l2_ahead;        // K blocks beyond the ring that a CTA pulls into L2 while it waits at its start
+    int sk_tiles;        // tiles [0, sk_tiles) are shared; tile sk_tiles + i * grid + g is whole tile i of CTA g
+    int whole_per_cta;
     const float* x_scale; int x_per_row;
     const float* w_scale; int w_per_col;
     float alpha;         // the tokens' common factor when x_scale == nullptr (batched-matmul calls)
@@ -69,10 +99,43 @@ struct DecParams {
     const void* ln_beta;    // nullable
     float ln_eps;
     int x_static;           // 1: Delta = x_scale[0] is given; 0: Delta_t = absmax(row t) / 127 -> xs_out[t]
-    int8_t* xq;             // [M, K] codes: written here, read back through the tensor map of X
+    int8_t* xq;             // [num_kb][DN][128] codes, K block by K block, each block in the swizzled
+                            // shared-memory image of a stage's activation slot
+    int8_t* xq_rows;        // nullable: [M, K] the same codes row-major (a caller who wants to see them)
+    int row_stages;         // ring stages a token row of x_raw (and the LayerNorm parameters behind it) occupy
+                            // while it is quantised; 0: they do not fit and are read from global memory
     float* xs_out;          // [M] step sizes (dynamic mode)
     float* stats_out;       // nullable [2 M]: mean and 1/sqrt(var + eps) of every row
     uint32_t* sync;         // [2]: rows quantised so far, CTAs past the meeting point; zero between calls
+};
+
+// A CTA's work in the order it is done: first its contiguous range of the SHARED tiles' (tile, K
+// block) pairs, then its whole tiles.  The shared tiles come first so that their fix-up (partial
+// sums parked, the last arriver adds them) runs in the epilogue warps while the CTA already streams
+// its next tile; what a CTA ends on is a whole tile with a plain epilogue.  (With every tile shared
+// and finished at the very end, each CTA spent 4.4 us between its last MMA and its exit.)
+struct DecWalk {
+    int64_t pos, end;
+    int whole_i;
+    __device__ __forceinline__ explicit DecWalk(const DecParams& p)
+        : pos((int64_t)blockIdx.x * p.range), end(min((int64_t)blockIdx.x * p.range + (int64_t)p.range, p.total_kb)), whole_i(0) {}
+    __device__ __forceinline__ bool next(const DecParams& p, int& ni, int& kb0, int& kb1) {
+        if (pos < end) {
+            ni = (int)(pos / p.num_kb);
+            kb0 = (int)(pos % p.num_kb);
+            kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
+            pos += kb1 - kb0;
+            return true;
+        }
+        if (whole_i < p.whole_per_cta) {
+            ni = p.sk_tiles + whole_i * (int)gridDim.x + (int)blockIdx.x;
+            ++whole_i;
+            kb0 = 0;
+            kb1 = p.num_kb;
+            return ni < p.num_n;
+        }
+        return false;
+    }
 };
 
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
@@ -85,24 +148,26 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
         : "memory");
 }
 __device__ __forceinline__ void dec_epi_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+__device__ __forceinline__ void dec_quant_sync() { asm volatile("bar.sync 3, %0;" ::"n"(DEC_QUANT_THREADS) : "memory"); }
 
 // ------------------------------------------------------------------------------------
-// The activation quantiser of the prologue: one token row per call, by the 128 epilogue threads.
+// The activation quantiser of the prologue: one token row per call, by DEC_QUANT_THREADS threads.
 // Arithmetic is the library's normative fp32 sequence (Eq. 1: Delta = max(m, 1e-5) / 127,
 // code = round(v * (1 / Delta)); LayerNorm: n = fma(x, rstd, -(mu * rstd)), y = fma(n, g, b),
 // statistics two-pass in fp32), so codes and step sizes equal those of sq_quant_act /
 // sq_ln_quant given the same statistics.
 // ------------------------------------------------------------------------------------
-constexpr int QV = 12;  // 16-byte vectors of the row a thread keeps in registers (rows up to 12 288 elements)
-
 template <bool IS_MAX>
-__device__ __forceinline__ float dec_epi_reduce(float v, float* red, int wq, int lane) {
+__device__ __forceinline__ float dec_quant_reduce(float v, float* red, int wq, int lane) {
+    constexpr int NW = DEC_QUANT_THREADS / 32;
     v = IS_MAX ? warp_max(v) : warp_sum(v);
     if (lane == 0) red[wq] = v;
-    dec_epi_sync();
-    const float a = red[0], b = red[1], c = red[2], d = red[3];
-    dec_epi_sync();  // `red` is rewritten by the next reduction
-    return IS_MAX ? fmaxf(fmaxf(a, b), fmaxf(c, d)) : (a + b) + (c + d);
+    dec_quant_sync();
+    float r = red[0];  // every thread folds the partials in the same order
+#pragma unroll
+    for (int i = 1; i < NW; ++i) r = IS_MAX ? fmaxf(r, red[i]) : r + red[i];
+    dec_quant_sync();  // `red` is rewritten by the next reduction
+    return r;
 }
 
 template <typename T>
@@ -110,61 +175,44 @@ __device__ __forceinline__ void dec_ln_vec(const uint4& xv, const uint4* g4, con
                                            float shift, float (&y)[8]) {
     float x[8], g[8], b[8];
     unpack8<T>(xv, x);
-    unpack8<T>(__ldg(g4 + v), g);
-    if (b4 != nullptr) unpack8<T>(__ldg(b4 + v), b);
+    unpack8<T>(g4[v], g);
+    if (b4 != nullptr) unpack8<T>(b4[v], b);
 #pragma unroll
     for (int k = 0; k < 8; ++k)
         y[k] = __fmaf_rn(__fmaf_rn(x[k], rstd, shift), g[k], b4 != nullptr ? b[k] : 0.0f);
 }
 
-template <typename T>
-__device__ void dec_quant_row(const DecParams& p, int row, int et, float* red) {
+// `src`: the row's 16-byte vectors, in shared memory (the usual case) or in global memory.
+// This code runs once per launch, so what it costs is fetching its instructions: with the passes
+// unrolled (or the row cached in registers by straight-line code) a 12 288-element row took 1.4 us
+// whatever the arithmetic was; as compact loops whose body is fetched once it takes a third of that.
+template <typename T, int DN>
+__device__ void dec_quant_row(const DecParams& p, int row, int et, const uint4* __restrict__ src,
+                              const uint4* __restrict__ g4, const uint4* __restrict__ b4, float static_delta, float* red) {
+    constexpr int NT = DEC_QUANT_THREADS;
     const int wq = et >> 5, lane = et & 31;
     const int nvec = (int)(p.K >> 3);
-    const uint4* src = reinterpret_cast<const uint4*>(static_cast<const T*>(p.x_raw) + (int64_t)row * p.K);
-    const uint4* g4 = reinterpret_cast<const uint4*>(p.ln_gamma);
-    const uint4* b4 = reinterpret_cast<const uint4*>(p.ln_beta);
-    const bool ln = p.ln_gamma != nullptr;
-    // the row comes from the kernel in front: read it through L2 (never a stale L1 line)
-    uint4 c[QV];
-#pragma unroll
-    for (int i = 0; i < QV; ++i) {
-        const int v = et + i * 128;
-        c[i] = v < nvec ? __ldcg(src + v) : make_uint4(0u, 0u, 0u, 0u);
-    }
+    const bool ln = g4 != nullptr;
     float rstd = 1.0f, shift = 0.0f;
     if (ln) {
         const float inv_C = __fdiv_rn(1.0f, (float)p.K);
         float sum = 0.0f;
-#pragma unroll
-        for (int i = 0; i < QV; ++i) {  // zero-filled vectors add nothing
+#pragma unroll 2
+        for (int v = et; v < nvec; v += NT) {
             float f[8];
-            unpack8<T>(c[i], f);
+            unpack8<T>(src[v], f);
             sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
         }
-        for (int v = et + QV * 128; v < nvec; v += 128) {
-            float f[8];
-            unpack8<T>(__ldcg(src + v), f);
-            sum += ((f[0] + f[1]) + (f[2] + f[3])) + ((f[4] + f[5]) + (f[6] + f[7]));
-        }
-        const float mu = dec_epi_reduce<false>(sum, red, wq, lane) * inv_C;
+        const float mu = dec_quant_reduce<false>(sum, red, wq, lane) * inv_C;
         float ss = 0.0f;
-#pragma unroll
-        for (int i = 0; i < QV; ++i) {
-            if (et + i * 128 < nvec) {
-                float f[8];
-                unpack8<T>(c[i], f);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) { const float d = f[k] - mu; ss = fmaf(d, d, ss); }
-            }
-        }
-        for (int v = et + QV * 128; v < nvec; v += 128) {
+#pragma unroll 2
+        for (int v = et; v < nvec; v += NT) {
             float f[8];
-            unpack8<T>(__ldcg(src + v), f);
+            unpack8<T>(src[v], f);
 #pragma unroll
             for (int k = 0; k < 8; ++k) { const float d = f[k] - mu; ss = fmaf(d, d, ss); }
         }
-        ss = dec_epi_reduce<false>(ss, red, wq, lane);
+        ss = dec_quant_reduce<false>(ss, red, wq, lane);
         rstd = rsqrt_refined(ss * inv_C + p.ln_eps);
         shift = -__fmul_rn(mu, rstd);
         if (p.stats_out != nullptr && et == 0) {
@@ -174,58 +222,53 @@ __device__ void dec_quant_row(const DecParams& p, int row, int et, float* red) {
     }
     float delta;
     if (p.x_static) {
-        delta = __ldg(p.x_scale);
+        delta = static_delta;
     } else {
         float m = 0.0f;
         if (ln) {
-#pragma unroll
-            for (int i = 0; i < QV; ++i) {
-                const int v = et + i * 128;
-                if (v < nvec) {
-                    float y[8];
-                    dec_ln_vec<T>(c[i], g4, b4, v, rstd, shift, y);
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(y[k]));
-                }
-            }
-            for (int v = et + QV * 128; v < nvec; v += 128) {
+#pragma unroll 2
+            for (int v = et; v < nvec; v += NT) {
                 float y[8];
-                dec_ln_vec<T>(__ldcg(src + v), g4, b4, v, rstd, shift, y);
+                dec_ln_vec<T>(src[v], g4, b4, v, rstd, shift, y);
 #pragma unroll
                 for (int k = 0; k < 8; ++k) m = fmaxf(m, fabsf(y[k]));
             }
         } else {
-            uint32_t pm = 0u;  // |x| and max are exact on the packed 16-bit values
-#pragma unroll
-            for (int i = 0; i < QV; ++i) {
-                pm = Act<T>::absmax2(pm, c[i].x); pm = Act<T>::absmax2(pm, c[i].y);
-                pm = Act<T>::absmax2(pm, c[i].z); pm = Act<T>::absmax2(pm, c[i].w);
+            uint32_t pm0 = 0u, pm1 = 0u;  // |x| and max are exact on the packed 16-bit values
+#pragma unroll 2
+            for (int v = et; v < nvec; v += NT) {
+                const uint4 x = src[v];
+                pm0 = Act<T>::absmax2(pm0, x.x); pm1 = Act<T>::absmax2(pm1, x.y);
+                pm0 = Act<T>::absmax2(pm0, x.z); pm1 = Act<T>::absmax2(pm1, x.w);
             }
-            for (int v = et + QV * 128; v < nvec; v += 128) {
-                const uint4 x = __ldcg(src + v);
-                pm = Act<T>::absmax2(pm, x.x); pm = Act<T>::absmax2(pm, x.y);
-                pm = Act<T>::absmax2(pm, x.z); pm = Act<T>::absmax2(pm, x.w);
-            }
-            m = Act<T>::hmax_of2(pm);
+            m = fmaxf(Act<T>::hmax_of2(pm0), Act<T>::hmax_of2(pm1));
         }
-        m = dec_epi_reduce<true>(m, red, wq, lane);
+        m = dec_quant_reduce<true>(m, red, wq, lane);
+        if (et == 0) DEC_TRACE(13);
         delta = step_size(m);
         if (et == 0) p.xs_out[row] = delta;
     }
     const float inv = recip_step(delta);
-    uint2* dst = reinterpret_cast<uint2*>(p.xq + (int64_t)row * p.K);
-    auto emit = [&](const uint4& xv, int v) {
+    uint2* rows_out = p.xq_rows != nullptr ? reinterpret_cast<uint2*>(p.xq_rows + (int64_t)row * p.K) : nullptr;
+    int8_t* const blk_row = p.xq + (size_t)row * BLOCK_K;
+    const int sw = row & 7;
+    const float lo = p.x_static ? kRoundMagic - 127.0f : -INFINITY, hi = p.x_static ? kRoundMagic + 127.0f : INFINITY;
+#pragma unroll 2
+    for (int v = et; v < nvec; v += NT) {
         float y[8];
-        if (ln) dec_ln_vec<T>(xv, g4, b4, v, rstd, shift, y);
-        else unpack8<T>(xv, y);
-        dst[v] = p.x_static ? quant8<true>(y, inv) : quant8<false>(y, inv);  // a given step may be exceeded: saturate
-    };
+        if (ln) dec_ln_vec<T>(src[v], g4, b4, v, rstd, shift, y);
+        else unpack8<T>(src[v], y);
+        uint32_t cdw[8];
 #pragma unroll
-    for (int i = 0; i < QV; ++i) {
-        const int v = et + i * 128;
-        if (v < nvec) emit(c[i], v);
+        for (int k = 0; k < 8; ++k)  // round(y * inv) in one FMA; a given static step may be exceeded: saturate
+            cdw[k] = __float_as_uint(fminf(fmaxf(__fmaf_rn(y[k], inv, kRoundMagic), lo), hi));
+        const uint2 q = make_uint2(pack4(cdw[0], cdw[1], cdw[2], cdw[3]), pack4(cdw[4], cdw[5], cdw[6], cdw[7]));
+        // vector v = bytes 8v .. 8v+7 of the row: K block kb, 16-byte chunk j of its 128-byte slice;
+        // the slice of token `row` sits where a 128-byte-swizzled tensor copy would have put it
+        const int kb = v >> 4, j = (v >> 1) & 7, half = v & 1;
+        *reinterpret_cast<uint2*>(blk_row + (size_t)kb * (DN * BLOCK_K) + ((j ^ sw) << 4) + half * 8) = q;
+        if (rows_out != nullptr) rows_out[v] = q;
     }
-    for (int v = et + QV * 128; v < nvec; v += 128) emit(__ldcg(src + v), v);
 }
 
 __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* ptr) {
@@ -291,8 +334,9 @@ __device__ __forceinline__ void dec_finish(const DecParams& p, const int32_t (&a
     }
 }
 
-template <int DN>
-__global__ void __launch_bounds__(DEC_THREADS, 1)
+// FUSED: the activation quantiser runs in the prologue (8 helper warps more; see the file header).
+template <int DN, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? DEC_THREADS_FUSED : DEC_THREADS, 1)
 decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                    const DecParams p) {
     constexpr int DEC_N = DN, DEC_STAGE = DecCfg<DN>::STAGE, DEC_STAGES = DecCfg<DN>::STAGES;
@@ -304,12 +348,14 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     uint64_t* tmem_full = empty_bar + DEC_STAGES;
     uint64_t* tmem_empty = tmem_full + 2;
     uint64_t* x_ready = tmem_empty + 2;  // prologue quantiser: every token row has been written
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(x_ready + 1);
+    uint64_t* x_row_bar = x_ready + 1;   // prologue quantiser: this CTA's token row has landed in the ring
+    uint64_t* x_ln_bar = x_row_bar + 1;  // prologue quantiser: the LayerNorm parameters have landed in the ring
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(x_ln_bar + 1);
     volatile uint32_t* abort_flag = tmem_holder + 1;
     volatile uint32_t* epi_go = tmem_holder + 2;
     volatile uint32_t* epi_last = tmem_holder + 3;
     float* s_xs = reinterpret_cast<float*>(tmem_holder + 4);  // [DN] the tokens' step sizes
-    float* s_red = s_xs + DEC_N;                              // [4] reduction scratch of the prologue quantiser
+    float* s_red = s_xs + DEC_N;                              // [8] reduction scratch of the prologue quantiser
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -325,6 +371,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             mbar_init(tmem_empty + s, 128);
         }
         mbar_init(x_ready, 1);
+        mbar_init(x_row_bar, 1);
+        mbar_init(x_ln_bar, 1);
         *abort_flag = 0u;
         *epi_go = 0u;
         *epi_last = 0u;
@@ -341,33 +389,60 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
     if (warp == 0) {
         // ============================ TMA producer ============================
         if (lane == 0) {
+            DEC_TRACE(0);
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            // The weights are static, the activations come from the kernel in front (the per-token
-            // quantiser): fill the ring with weight slices first, wait for the predecessor, then
-            // add the activation slices of those stages.
-            int prefetched = 0;
+            // The weights are static, the activations come from the kernel in front (or from this
+            // kernel's own quantiser): fill the ring with weight slices first, wait for the
+            // predecessor (and for the quantiser), then add the activation slices of those stages.
+            // A CTA that quantises a token row keeps the top of its ring free for that row.
+            constexpr bool fused = FUSED;
+            const uint64_t stream_once = l2_policy_evict_first();
+            auto load_x = [&](uint8_t* sx, uint64_t* bar, int kb) {
+                if (fused)  // one contiguous, pre-swizzled block per K block
+                    bulk::bulk_load(sx, p.xq + (size_t)kb * DecCfg<DN>::X_BYTES, DecCfg<DN>::X_BYTES, bar);
+                else
+                    tma_load_4d<1>(sx, &tmap_x, bar, kb * BLOCK_K, 0, 0, 0);
+            };
             bool waited = false;
-            int64_t pos = (int64_t)blockIdx.x * p.range;
-            const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
-            for (; ok && pos < end;) {
-                const int ni = (int)(pos / p.num_kb);
-                const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
-                pos += kb1 - kb0;
+            DecWalk walk(p);
+            int ni, kb0, kb1;
+            while (ok && walk.next(p, ni, kb0, kb1)) {
                 int kb = kb0;
                 if (!waited) {
-                    const int n_pre = min(DEC_STAGES, kb1 - kb0);
+                    int n_pre = min(DEC_STAGES, kb1 - kb0);
+                    if (fused && (int)blockIdx.x < p.M) n_pre = max(0, min(n_pre, DEC_STAGES - p.row_stages));
                     for (int i = 0; i < n_pre; ++i) {
                         mbar_expect_tx(full_bar + i, DEC_STAGE);
-                        tma_load_4d<1>(smem + i * DEC_STAGE, &tmap_w, full_bar + i, (kb0 + i) * BLOCK_K, ni * BLOCK_M, 0, 0);
+                        tma_load_4d_policy(smem + i * DEC_STAGE, &tmap_w, full_bar + i, (kb0 + i) * BLOCK_K, ni * BLOCK_M, 0, 0,
+                                           stream_once);
                     }
+                    // The weights are static and this lane is about to wait (for the launch in front, then
+                    // for the quantiser): meanwhile the next slices of this CTA's stream go to L2, so that
+                    // HBM keeps working through the gap between two launches.
+                    {
+                        DecWalk ahead(p);
+                        int ni2, a2, b2, idx = 0;
+                        const int stop = n_pre + p.l2_ahead;
+                        while (idx < stop && ahead.next(p, ni2, a2, b2))
+                            for (int k2 = a2; k2 < b2 && idx < stop; ++k2, ++idx)
+                                if (idx >= n_pre) tma_prefetch_l2_4d(&tmap_w, k2 * BLOCK_K, ni2 * BLOCK_M, 0, 0);
+                    }
+                    DEC_TRACE(1);
                     pdl_wait();
+                    DEC_TRACE(2);
+#ifdef SQ_DEC_TRACE
+                    {  // one global-timer read per CTA relates the launches of a chain to each other
+                        unsigned long long t;
+                        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+                        g_dec_trace[p.trace_id][blockIdx.x][4] = t;
+                    }
+#endif
                     // with the quantiser in the prologue the codes of X exist once every CTA's rows are done
-                    if (p.x_raw != nullptr && !(ok = mbar_wait(x_ready, 0u, abort_flag, p.status, 11))) break;
-                    for (int i = 0; i < n_pre; ++i)
-                        tma_load_4d<1>(smem + i * DEC_STAGE + W_BYTES, &tmap_x, full_bar + i, (kb0 + i) * BLOCK_K, 0, 0, 0);
-                    prefetched = n_pre;
+                    if (fused && !(ok = mbar_wait(x_ready, 0u, abort_flag, p.status, 11))) break;
+                    DEC_TRACE(3);
+                    for (int i = 0; i < n_pre; ++i) load_x(smem + i * DEC_STAGE + W_BYTES, full_bar + i, kb0 + i);
                     waited = true;
                     kb = kb0 + n_pre;
                     stage = n_pre % DEC_STAGES;
@@ -377,12 +452,11 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 6))) break;
                     uint8_t* sw = smem + stage * DEC_STAGE;
                     mbar_expect_tx(full_bar + stage, DEC_STAGE);
-                    tma_load_4d<1>(sw, &tmap_w, full_bar + stage, kb * BLOCK_K, ni * BLOCK_M, 0, 0);
-                    tma_load_4d<1>(sw + W_BYTES, &tmap_x, full_bar + stage, kb * BLOCK_K, 0, 0, 0);
+                    tma_load_4d_policy(sw, &tmap_w, full_bar + stage, kb * BLOCK_K, ni * BLOCK_M, 0, 0, stream_once);
+                    load_x(sw + W_BYTES, full_bar + stage, kb);
                     if (++stage == DEC_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
-            (void)prefetched;
         }
     } else if (warp == 1) {
         // ============================ MMA issuer ==============================
@@ -393,16 +467,17 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
-            int64_t pos = (int64_t)blockIdx.x * p.range;
-            const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
-            for (; ok && pos < end;) {
-                const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
-                pos += kb1 - kb0;
+            DecWalk walk(p);
+            int ni, kb0, kb1;
+            while (ok && walk.next(p, ni, kb0, kb1)) {
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 7))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * DEC_N);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 8))) break;
+#ifdef SQ_DEC_TRACE
+                    if (g_dec_trace[p.trace_id][blockIdx.x][5] == 0ull) DEC_TRACE(5);
+#endif
                     tcgen05_fence_after();
                     const uint32_t sw = smem_u32(smem + stage * DEC_STAGE);
                     const uint32_t sx = sw + W_BYTES;
@@ -415,41 +490,87 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                 }
                 if (!ok) break;
                 umma_commit<1>(tmem_full + slot);
+                DEC_TRACE(6);
                 slot ^= 1;
                 if (slot == 0) slot_phase ^= 1u;
             }
         }
     } else {
         // ============================ epilogue (warps 2-5) ====================
-        pdl_wait();  // x_scale and the split-K scratch belong to earlier kernels until here
+        float static_delta = 0.0f;
+        if constexpr (FUSED) {
+            // The folded LayerNorm parameters are static: a CTA that will quantise a token row pulls them
+            // into the top of its ring (behind the row's own place) before it waits for the launch in front
+            if (threadIdx.x == 64 && p.ln_gamma != nullptr && p.row_stages > 0 && (int)blockIdx.x < p.M) {
+                uint8_t* top = smem + (DEC_STAGES - p.row_stages) * DEC_STAGE;
+                const uint32_t rb = (uint32_t)(p.K * 2);
+                mbar_expect_tx(x_ln_bar, p.ln_beta != nullptr ? 2 * rb : rb);
+                bulk::bulk_load(top + rb, p.ln_gamma, rb, x_ln_bar);
+                if (p.ln_beta != nullptr) bulk::bulk_load(top + 2 * rb, p.ln_beta, rb, x_ln_bar);
+            }
+            // ... and a static step is a calibrated constant: fetched now, it is there when the row lands
+            // (read after the wait, one L2 miss queued behind every CTA's weight prefetch cost 3-5 us)
+            if (p.x_static) static_delta = __ldg(p.x_scale);
+        }
+        pdl_wait();  // a dynamic x_scale and the split-K scratch belong to earlier kernels until here
+        if (threadIdx.x == 64) DEC_TRACE(7);
         const int quarter = warp & 3;           // TMEM lanes this warp may read
         const int ch = quarter * 32 + lane;     // output channel within the tile
         const int et = threadIdx.x - 64;        // 0..127
         bool x_ok = true;
-        if (p.x_raw != nullptr) {
-            // ---- activation quantiser: CTA r takes token rows r, r + grid, ... ----
+        if constexpr (FUSED) {
+            // ---- activation quantiser (warps 2-9): CTA r takes token rows r, r + grid, ... ----
             uint32_t done = 0;
+            bool row_ok = true;
             for (int row = (int)blockIdx.x; row < p.M; row += (int)gridDim.x, ++done) {
-                if (p.x_is_bf16) dec_quant_row<__nv_bfloat16>(p, row, et, s_red);
-                else dec_quant_row<__half>(p, row, et, s_red);
+                const uint8_t* grow = static_cast<const uint8_t*>(p.x_raw) + (size_t)row * (size_t)p.K * 2;
+                const uint4* src = reinterpret_cast<const uint4*>(grow);
+                const uint4* g4 = reinterpret_cast<const uint4*>(p.ln_gamma);
+                const uint4* b4 = reinterpret_cast<const uint4*>(p.ln_beta);
+                if (p.row_stages > 0) {
+                    // the row lands in the top stages of the ring (the producer lane leaves them
+                    // alone until the meeting below) with one bulk copy
+                    uint8_t* rowbuf = smem + (DEC_STAGES - p.row_stages) * DEC_STAGE;
+                    const uint32_t rb = (uint32_t)(p.K * 2);
+                    if (et == 0) {
+                        mbar_expect_tx(x_row_bar, rb);
+                        bulk::bulk_load(rowbuf, grow, rb, x_row_bar);
+                        bool ok = mbar_wait(x_row_bar, done & 1u, abort_flag, p.status, 12);
+                        if (ok && g4 != nullptr && done == 0) ok = mbar_wait(x_ln_bar, 0u, abort_flag, p.status, 13);
+                        *epi_go = ok ? 1u : 0u;
+                    }
+                    if (g4 != nullptr) {
+                        g4 = reinterpret_cast<const uint4*>(rowbuf + rb);
+                        if (b4 != nullptr) b4 = reinterpret_cast<const uint4*>(rowbuf + 2 * rb);
+                    }
+                    dec_quant_sync();
+                    if (et == 0) DEC_TRACE(8);
+                    row_ok = *epi_go != 0u;
+                    src = reinterpret_cast<const uint4*>(rowbuf);
+                    if (!row_ok) break;  // the copy never landed (same outcome in every thread)
+                }
+                if (p.x_is_bf16) dec_quant_row<__nv_bfloat16, DEC_N>(p, row, et, src, g4, b4, static_delta, s_red);
+                else dec_quant_row<__half, DEC_N>(p, row, et, src, g4, b4, static_delta, s_red);
+                dec_quant_sync();  // everyone is done with the row buffer (and with epi_go)
             }
-            if (done) __threadfence();  // this thread's codes are visible device-wide before the count moves
-            dec_epi_sync();
             if (et == 0) {
+                DEC_TRACE(14);
                 if (done) {
-                    asm volatile("fence.proxy.async.global;" ::: "memory");  // they will be read by bulk-tensor copies
+                    // the barrier above ordered every thread's stores before this fence: the count moves
+                    // only once this CTA's codes are visible device-wide (also to bulk copies)
+                    __threadfence();
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
                     atomicAdd(p.sync, done);
                 }
+                DEC_TRACE(15);
                 // meet: all M rows written (bounded, like every other wait of the kernel)
                 const long long t0 = clock64();
-                bool ok = true;
-                while (ld_acquire_gpu(p.sync) < (uint32_t)p.M) {
-                    if (*abort_flag || (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) {
-                        ok = false;
-                        break;
-                    }
+                bool ok = row_ok;
+                while (ok && ld_acquire_gpu(p.sync) < (uint32_t)p.M) {
+                    if (*abort_flag || (unsigned long long)(clock64() - t0) > (unsigned long long)kWaitCycles) ok = false;
                 }
                 if (ok) {
+                    DEC_TRACE(10);
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                     mbar_arrive(x_ready);  // the producer lane may fetch activation slices now
                 } else {
@@ -464,21 +585,19 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
                     p.sync[1] = 0u;
                 }
             }
-            dec_epi_sync();
+            dec_quant_sync();
             x_ok = *epi_go != 0u;
-            dec_epi_sync();  // epi_go is rewritten in the loop below
         }
+        if (warp < 6) {  // the helper warps of the quantiser are done; the four epilogue warps go on
+        dec_epi_sync();  // (epi_go is rewritten in the loop below)
         // step sizes: the caller's, or the ones the prologue just wrote (read through L2)
         if (et < DEC_N) s_xs[et] = (et < p.M && p.x_scale) ? __ldcg(p.x_scale + (p.x_per_row ? et : 0)) : p.alpha;
         dec_epi_sync();
         int slot = 0;
         uint32_t slot_phase = 0;
-        int64_t pos = (int64_t)blockIdx.x * p.range;
-        const int64_t end = min(pos + (int64_t)p.range, p.total_kb);
-        while (x_ok && pos < end) {
-            const int ni = (int)(pos / p.num_kb);
-            const int kb0 = (int)(pos % p.num_kb), kb1 = (int)min((int64_t)p.num_kb, kb0 + (end - pos));
-            pos += kb1 - kb0;
+        DecWalk walk(p);
+        int ni, kb0, kb1;
+        while (x_ok && walk.next(p, ni, kb0, kb1)) {
             const int64_t col = (int64_t)ni * BLOCK_M + ch;
             const DecChan chan = dec_chan(p, col);  // in flight while the K blocks stream
             uint16_t res[DEC_N];
@@ -486,6 +605,9 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             if (et == 0) *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 9) ? 1u : 0u;
             dec_epi_sync();
             if (*epi_go == 0u) break;
+#ifdef SQ_DEC_TRACE
+            if (et == 0 && g_dec_trace[p.trace_id][blockIdx.x][11] == 0ull) DEC_TRACE(11);
+#endif
             tcgen05_fence_after();
             int32_t acc[DEC_N];
 #pragma unroll
@@ -543,6 +665,8 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             }
             dec_epi_sync();  // epi_go / epi_last are rewritten by thread 0 in the next round
         }
+        if (et == 0) DEC_TRACE(12);
+        }  // warp < 6
     }
 
     __syncwarp();
@@ -562,40 +686,61 @@ constexpr int kMinKbPerCta = 4;       // below this a CTA's fixed costs outweigh
 constexpr int kMaxCtas = 256;         // bound used by the workspace formula
 constexpr int64_t kMaxSharedTiles = (int64_t)kDecCounterBytes / 4;
 
-struct DecPlan { int ctas, range, maxcount; };
+// K blocks beyond its ring that a CTA pulls into L2 while it waits at its start (8 x 16 KB x 148 CTAs =
+// 19 MB).  Measured on the GPT-3 shapes, back-to-back calls: 0 -> 8 blocks gains 1.5 to 2 us per call
+// (12288 x 49152, 16 tokens: 95.6 -> 93.5 us), 16 the same, 32 and 64 lose it again (the lines are
+// evicted before they are used, and the activations with them).
+constexpr int kL2AheadBlocks = 8;
+
+struct DecPlan { int ctas, range, maxcount, sk_tiles, whole_per_cta; };
 DecPlan plan_decode(int num_n, int num_kb, int sms, bool may_share) {
-    const int64_t total = (int64_t)num_n * num_kb;
-    DecPlan pl;
+    DecPlan pl{};
+    const int ctas_max = std::min(sms, kMaxCtas);
     if (!may_share) {  // whole tiles only
-        const int ctas = (int)std::min<int64_t>(num_n, sms);
-        const int tiles_per = (num_n + ctas - 1) / ctas;
-        pl.range = tiles_per * num_kb;
-        pl.ctas = (num_n + tiles_per - 1) / tiles_per;
+        pl.ctas = std::min(num_n, ctas_max);
+        pl.whole_per_cta = (num_n + pl.ctas - 1) / pl.ctas;
+        pl.sk_tiles = 0;
+        pl.range = 0;
         pl.maxcount = 1;
         return pl;
     }
-    int64_t ctas = std::min<int64_t>(std::min(sms, kMaxCtas), std::max<int64_t>(1, total / kMinKbPerCta));
-    pl.range = (int)((total + ctas - 1) / ctas);
-    pl.ctas = (int)((total + pl.range - 1) / pl.range);
+    // as many whole tiles per CTA as divide evenly; the remaining tiles (fewer than CTAs) are shared:
+    // their (tile, K block) pairs are cut into equal contiguous ranges
+    pl.whole_per_cta = num_n / ctas_max;
+    pl.sk_tiles = num_n - pl.whole_per_cta * ctas_max;
+    const int64_t sk_total = (int64_t)pl.sk_tiles * num_kb;
+    if (sk_total == 0) {
+        pl.ctas = ctas_max;
+        pl.range = 0;
+        pl.maxcount = 1;
+        return pl;
+    }
+    const int64_t sk_ctas = std::min<int64_t>(ctas_max, std::max<int64_t>(1, sk_total / kMinKbPerCta));
+    pl.range = (int)((sk_total + sk_ctas - 1) / sk_ctas);
+    pl.ctas = pl.whole_per_cta > 0 ? ctas_max : (int)((sk_total + pl.range - 1) / pl.range);
     pl.maxcount = (num_kb + pl.range - 2) / pl.range + 1;
     return pl;
 }
 
-template <int DN>
+template <int DN, bool FUSED>
 sq_status launch_decode(const GemmArgs& a, const DecParams& p, int ctas, cudaStream_t st) {
     CUtensorMap mw, mx;
     int s0, s1, s2;
     if (!make_map(&mw, a.B, 1, a.K, a.N, 1, 1, a.K, 0, 0, BLOCK_K, BLOCK_M, &s0, &s1, &s2)) return SQ_ERR_CUDA;
-    const void* x_codes = p.x_raw != nullptr ? static_cast<const void*>(p.xq) : static_cast<const void*>(a.A);
+    // (with the quantiser in the prologue the activation slices come by plain bulk copies: the
+    // map of X is then a placeholder over the weights)
+    const void* x_codes = p.x_raw != nullptr ? static_cast<const void*>(a.B) : static_cast<const void*>(a.A);
     if (!make_map(&mx, x_codes, 1, a.K, a.M, 1, 1, a.K, 0, 0, BLOCK_K, DN, &s0, &s1, &s2)) return SQ_ERR_CUDA;
     static bool attr_set[64] = {false};  // per instantiation and device
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(decode_gemm_kernel<DN>, cudaFuncAttributeMaxDynamicSharedMemorySize, DecCfg<DN>::SMEM));
+        SQ_CUDA_OK(cudaFuncSetAttribute(decode_gemm_kernel<DN, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        DecCfg<DN>::SMEM));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    return launch_pdl(decode_gemm_kernel<DN>, dim3((unsigned)ctas), dim3(DEC_THREADS), (size_t)DecCfg<DN>::SMEM, st, 1, mw, mx, p);
+    return launch_pdl(decode_gemm_kernel<DN, FUSED>, dim3((unsigned)ctas), dim3(FUSED ? DEC_THREADS_FUSED : DEC_THREADS),
+                      (size_t)DecCfg<DN>::SMEM, st, 1, mw, mx, p);
 }
 
 }  // namespace
@@ -610,7 +755,8 @@ size_t decode_workspace_bytes(int64_t M, int64_t N) {
 // The same plus what the prologue quantiser writes: 256 bytes of step sizes, then the [M, K] codes.
 static size_t round256(size_t v) { return (v + 255) & ~(size_t)255; }
 size_t decode_fused_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-    return round256(decode_workspace_bytes(M, N)) + 256 + round256((size_t)M * (size_t)K);
+    const size_t num_kb = (size_t)((K + BLOCK_K - 1) / BLOCK_K), dn = M <= 16 ? 16 : 32;
+    return round256(decode_workspace_bytes(M, N)) + 256 + num_kb * dn * BLOCK_K;
 }
 
 // Up to 32 tokens the activation slices are a small addition to the weight stream and this kernel
@@ -631,9 +777,17 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.num_kb = (int)((a.K + BLOCK_K - 1) / BLOCK_K);
     const bool may_share = ws_bytes >= decode_workspace_bytes(a.M, a.N) && p.num_n <= kMaxSharedTiles;
     const DecPlan plan = plan_decode(p.num_n, p.num_kb, sm_count(), may_share);
-    p.total_kb = (int64_t)p.num_n * p.num_kb;
+    p.total_kb = (int64_t)plan.sk_tiles * p.num_kb;
     p.range = plan.range;
     p.maxcount = plan.maxcount;
+    p.l2_ahead = kL2AheadBlocks;
+    p.trace_id = 0;
+#ifdef SQ_DEC_TRACE
+    static int trace_launch = 0;
+    p.trace_id = (trace_launch++) & 7;
+#endif
+    p.sk_tiles = plan.sk_tiles;
+    p.whole_per_cta = plan.whole_per_cta;
     p.x_scale = a.x_scale; p.x_per_row = a.x_per_row;
     p.w_scale = a.w_scale; p.w_per_col = a.w_per_col;
     p.alpha = a.alpha;
@@ -648,16 +802,33 @@ sq_status decode_gemm(const GemmArgs& a, void* workspace, size_t ws_bytes, cudaS
     p.x_raw = a.x_raw; p.x_is_bf16 = a.x_raw_dt == SQ_BF16;
     p.ln_gamma = a.ln_gamma; p.ln_beta = a.ln_beta; p.ln_eps = a.ln_eps;
     p.x_static = a.x_static;
-    p.xq = nullptr; p.xs_out = nullptr; p.stats_out = a.ln_stats_out; p.sync = nullptr;
+    p.xq = nullptr; p.xq_rows = nullptr; p.row_stages = 0; p.xs_out = nullptr; p.stats_out = a.ln_stats_out; p.sync = nullptr;
     if (a.x_raw != nullptr) {  // the caller (sq_api.cu) has checked that the workspace holds the scratch
         char* scratch = static_cast<char*>(workspace) + round256(decode_workspace_bytes(a.M, a.N));
         p.xs_out = a.xs_out != nullptr ? a.xs_out : reinterpret_cast<float*>(scratch);
-        p.xq = a.xq_out != nullptr ? a.xq_out : reinterpret_cast<int8_t*>(scratch + 256);
+        p.xq = reinterpret_cast<int8_t*>(scratch + 256);
+        p.xq_rows = a.xq_out;
+        // a token row (2 K bytes) is quantised out of the top stages of its CTA's ring when it fits
+        const int64_t stage_bytes = a.M <= 16 ? DecCfg<16>::STAGE : DecCfg<32>::STAGE;
+        const int64_t parts = a.ln_gamma == nullptr ? 1 : (a.ln_beta == nullptr ? 2 : 3);  // row [+ gamma [+ beta]]
+        const int64_t need = (parts * 2 * a.K + stage_bytes - 1) / stage_bytes;
+        p.row_stages = need <= DecCfg<16>::STAGES ? (int)need : 0;
         p.sync = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kWsSyncOff);
         if (!a.x_static) { p.x_scale = p.xs_out; p.x_per_row = 1; }
     }
-    if (a.M <= 16) return launch_decode<16>(a, p, plan.ctas, st);
-    return launch_decode<32>(a, p, plan.ctas, st);
+    if (a.x_raw != nullptr)
+        return a.M <= 16 ? launch_decode<16, true>(a, p, plan.ctas, st) : launch_decode<32, true>(a, p, plan.ctas, st);
+    return a.M <= 16 ? launch_decode<16, false>(a, p, plan.ctas, st) : launch_decode<32, false>(a, p, plan.ctas, st);
 }
 
 }  // namespace sq
+
+#ifdef SQ_DEC_TRACE
+// Copies the timestamps of the last eight decode-shaped launches to host_out[8 * 256 * 16] and clears them.
+extern "C" int sq_debug_decode_trace(unsigned long long* host_out) {
+    if (cudaMemcpyFromSymbol(host_out, sq::g_dec_trace, sizeof(sq::g_dec_trace)) != cudaSuccess) return 1;
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, sq::g_dec_trace) != cudaSuccess) return 1;
+    return cudaMemset(addr, 0, sizeof(sq::g_dec_trace)) == cudaSuccess ? 0 : 1;
+}
+#endif

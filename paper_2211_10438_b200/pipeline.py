@@ -254,14 +254,25 @@ class DecoderBlockStatic:
 
 class DecoderBlockDecode:
     """Generation stage of DecoderBlockStatic: one new token per sequence against an INT8 KV cache,
-    as nine libsq launches: LN1+quantise -> QKV GEMM (INT8 out) -> attention of the new token over
-    the cache, which also appends its k, v (INT8 out) -> out-proj GEMM -> residual ->
-    LN2+quantise -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM -> residual (the add folded into the GEMM
-    epilogue measured the same time here, so the two small launches stay).  Same `lin` / `steps` as the
-    prompt block.  `ctx` (int32 device tensor [B]) counts the positions each sequence has cached."""
+    as seven libsq launches: LN1 + static quantiser -> QKV GEMM (INT8 out) -> attention of the new
+    token over the cache, which also appends its k, v (INT8 out) -> out-proj GEMM with the residual
+    add in its epilogue -> LN2 + static quantiser -> FC1 GEMM (+ReLU, INT8 out) -> FC2 GEMM with the
+    residual add in its epilogue.
+    `fused=True` moves both LayerNorm+quantise steps into the prologues of the GEMMs that consume
+    them (five launches).  Measured on B200 (OPT-30B shapes, batch 16, one CUDA graph per step): inside
+    a chain of dependent launches the separate quantiser kernel overlaps the GEMM's own start-up and
+    the seven-launch form is the faster one (158 against 164 us per layer); for a GEMM called on its
+    own the fused form wins.  `fuse_residual=False` keeps the residual adds as kernels of their own
+    (nine launches with `fused=False`: 161 us).  Same `lin` / `steps` as the prompt block.  `ctx`
+    (int32 device tensor [B]) counts the positions each sequence has cached.  `keep_codes` also
+    writes the LayerNorm codes of the fused form to x1q / x2q so that a checker can look at them."""
 
-    def __init__(self, lin, steps, B, H, d, L_max, act_dtype, eps=1e-5):
+    def __init__(self, lin, steps, B, H, d, L_max, act_dtype, eps=1e-5, fused=False, keep_codes=False,
+                 fuse_residual=True):
         self.lin, self.B, self.H, self.d, self.L_max, self.dt, self.eps = lin, B, H, d, L_max, act_dtype, eps
+        self.fused = fused and B <= 32
+        self.fuse_residual = fuse_residual
+        self.keep_codes = keep_codes
         dev = lin["qkv"].Wq.device
         hid, ffn = H * d, lin["fc1"].Wq.shape[0]
         self.hid = hid
@@ -284,10 +295,11 @@ class DecoderBlockDecode:
         self.v_cache = torch.zeros((B, H, L_max // 4, d, 4), dtype=torch.int8, device=dev)
         self.ctx = torch.zeros(B, dtype=torch.int32, device=dev)
         self.lens = torch.ones(B, dtype=torch.int32, device=dev)  # ctx + 1: what the new token attends over
-        need = max([sq.workspace_bytes(sq.SQ_OP_GEMM, B, l.Wq.shape[0], l.Wq.shape[1]) for l in lin.values()] +
+        op = sq.SQ_OP_GEMM_FUSED_QUANT if self.fused else sq.SQ_OP_GEMM
+        need = max([sq.workspace_bytes(op, B, l.Wq.shape[0], l.Wq.shape[1]) for l in lin.values()] +
                    [sq.workspace_bytes(sq.SQ_OP_LN_QUANT, B, 0, hid)])
         self.ws = sq.new_workspace(need, dev)
-        self.launches_per_step = 9
+        self.launches_per_step = 9 - (2 if self.fused else 0) - (2 if self.fuse_residual else 0)
 
     def load_prompt(self, qkv_codes, S):
         """Fill the cache from a prompt pass's QKV code buffer [B*S, 3*H*d]; every sequence then holds S positions."""
@@ -300,24 +312,45 @@ class DecoderBlockDecode:
         (default: the cache capacity).  Returns the block output [B, H*d]."""
         L, s, B, H, d = self.lin, self.s, self.B, self.H, self.d
         max_len = self.L_max if max_len is None else max_len
-        sq.sq_ln_quant(x, L["qkv"].gamma_hat, L["qkv"].beta_hat, self.eps, "per_tensor_static", Xq=self.x1q,
-                       x_scale=s["d_ln1"], workspace=self.ws)
-        sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
-                        requant_mul=self.r_qkv, out=self.qkv)
-        hid = self.hid  # the attention kernel takes the new k, v rows from the QKV buffer and caches them
+        hid = self.hid
+        if self.fused:
+            sq.sq_w8a8_gemm_fused_quant(x, L["qkv"].Wq, L["qkv"].w_scale, self.ws, "per_tensor_static", x_scale=s["d_ln1"],
+                                        gamma_hat=L["qkv"].gamma_hat, beta_hat=L["qkv"].beta_hat, eps=self.eps,
+                                        Xq_out=self.x1q if self.keep_codes else None, bias=L["qkv"].bias,
+                                        requant_mul=self.r_qkv, out=self.qkv)
+        else:
+            sq.sq_ln_quant(x, L["qkv"].gamma_hat, L["qkv"].beta_hat, self.eps, "per_tensor_static", Xq=self.x1q,
+                           x_scale=s["d_ln1"], workspace=self.ws)
+            sq.sq_w8a8_gemm(self.x1q, L["qkv"].Wq, s["d_ln1"], L["qkv"].w_scale, self.ws, bias=L["qkv"].bias,
+                            requant_mul=self.r_qkv, out=self.qkv)
+        # the attention kernel takes the new k, v rows from the QKV buffer and caches them
         sq.sq_w8a8_decode_attention(self.qkv, self.k_cache, self.v_cache, self.lens, B, H, d, self.L_max, max_len,
                                     self.alpha_qk, self.alpha_pv, self.ws, requant_mul=self.r_attn, out=self.attn,
                                     k_new=self.qkv[:, hid:], v_new=self.qkv[:, 2 * hid:])
-        sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
-                        bias=L["out_proj"].bias, out=self.proj)
-        sq.sq_residual_add(x, self.proj, out=self.h)
-        sq.sq_ln_quant(self.h, L["fc1"].gamma_hat, L["fc1"].beta_hat, self.eps, "per_tensor_static", Xq=self.x2q,
-                       x_scale=s["d_ln2"], workspace=self.ws)
-        sq.sq_w8a8_gemm(self.x2q, L["fc1"].Wq, s["d_ln2"], L["fc1"].w_scale, self.ws, bias=L["fc1"].bias, relu=True,
-                        requant_mul=self.r_fc1, out=self.f1q)
-        sq.sq_w8a8_gemm(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, bias=L["fc2"].bias,
-                        out=self.fc2)
-        sq.sq_residual_add(self.h, self.fc2, out=self.y)
+        if self.fuse_residual:
+            sq.sq_w8a8_gemm_residual(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws, x,
+                                     bias=L["out_proj"].bias, out=self.h)
+        else:
+            sq.sq_w8a8_gemm(self.attn, L["out_proj"].Wq, s["d_attn"], L["out_proj"].w_scale, self.ws,
+                            bias=L["out_proj"].bias, out=self.proj)
+            sq.sq_residual_add(x, self.proj, out=self.h)
+        if self.fused:
+            sq.sq_w8a8_gemm_fused_quant(self.h, L["fc1"].Wq, L["fc1"].w_scale, self.ws, "per_tensor_static", x_scale=s["d_ln2"],
+                                        gamma_hat=L["fc1"].gamma_hat, beta_hat=L["fc1"].beta_hat, eps=self.eps,
+                                        Xq_out=self.x2q if self.keep_codes else None, bias=L["fc1"].bias, relu=True,
+                                        requant_mul=self.r_fc1, out=self.f1q)
+        else:
+            sq.sq_ln_quant(self.h, L["fc1"].gamma_hat, L["fc1"].beta_hat, self.eps, "per_tensor_static", Xq=self.x2q,
+                           x_scale=s["d_ln2"], workspace=self.ws)
+            sq.sq_w8a8_gemm(self.x2q, L["fc1"].Wq, s["d_ln2"], L["fc1"].w_scale, self.ws, bias=L["fc1"].bias, relu=True,
+                            requant_mul=self.r_fc1, out=self.f1q)
+        if self.fuse_residual:
+            sq.sq_w8a8_gemm_residual(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, self.h,
+                                     bias=L["fc2"].bias, out=self.y)
+        else:
+            sq.sq_w8a8_gemm(self.f1q, L["fc2"].Wq, s["d_fc1"], L["fc2"].w_scale, self.ws, bias=L["fc2"].bias,
+                            out=self.fc2)
+            sq.sq_residual_add(self.h, self.fc2, out=self.y)
         if advance:  # bookkeeping of the sequence lengths, not part of the arithmetic
             torch._foreach_add_([self.ctx, self.lens], 1)
         return self.y

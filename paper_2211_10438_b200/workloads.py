@@ -5,7 +5,7 @@
 Meant for profilers and quick timing: every workload allocates its operands with a seeded
 generator, calls the entry point `--calls` times on the current CUDA device, synchronises, checks
 the device status word and prints the mean time per call (CUDA events, after one untimed call).
-Names: decode_gemm, attention, kv_attention, ln_quant, quant_act.
+Names: gemm, decode_gemm, generation_block, attention, kv_attention, ln_quant, quant_act.
 """
 import argparse
 
@@ -32,20 +32,99 @@ def _gen(seed=0x5EED):
     return g
 
 
+def _codes(shape, values, g):
+    """INT8 operand codes of a given value class: what the tensor cores draw depends on the data."""
+    if values == "zeros":
+        return torch.zeros(shape, dtype=torch.int8, device="cuda")
+    if values == "ones":
+        return torch.ones(shape, dtype=torch.int8, device="cuda")
+    if values == "tri":  # small codes, triangular around zero: what a smoothed LLM activation quantises to, mostly
+        a = torch.randint(-8, 9, shape, dtype=torch.int8, device="cuda", generator=g)
+        return a + torch.randint(-8, 9, shape, dtype=torch.int8, device="cuda", generator=g)
+    return torch.randint(-127, 128, shape, dtype=torch.int8, device="cuda", generator=g)  # "full"
+
+
+def gemm(args):
+    """Prefill-shaped W8A8 GEMM (default: the OPT-13B FC1 of config 2), bf16 output, per-token x
+    per-channel step sizes.  --values picks the operand value class (the power the tensor cores draw,
+    and with it the sustained clock, depends on the data), --no-split withholds the scratch the
+    K split of a partly filled last wave needs, --int-mm times torch._int_mm (cuBLASLt, INT32
+    output, no epilogue) on the same operands for context."""
+    g = _gen()
+    for M in args.M:
+        N, K = args.N, args.K
+        X = _codes((M, K), args.values, g)
+        Wq = _codes((N, K), args.values, g)
+        xs = torch.rand(M, device="cuda", generator=g) * 0.1
+        wsc = torch.rand(N, device="cuda", generator=g) * 1e-3
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = sq.new_workspace(256 if args.no_split else sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K))
+        us = _time(lambda: sq.sq_w8a8_gemm(X, Wq, xs, wsc, ws, out=Y), args.calls)
+        line = "gemm M=%d N=%d K=%d values=%s%s: %.1f us, %.0f TOPS" % (
+            M, N, K, args.values, " no-split" if args.no_split else "", us, 2.0 * M * N * K / us / 1e6)
+        if args.int_mm:
+            Wt = Wq.t()
+            us2 = _time(lambda: torch._int_mm(X, Wt), args.calls)
+            line += "; torch._int_mm %.1f us, %.0f TOPS" % (us2, 2.0 * M * N * K / us2 / 1e6)
+        print(line)
+        if sq.device_status(ws) != 0:
+            raise SystemExit("device status word = %d" % sq.device_status(ws))
+        del X, Wq, Y
+    return sq.new_workspace(256)
+
+
 def decode_gemm(args):
-    """Decode-shaped W8A8 GEMM: M tokens against an [N, K] INT8 weight (default: GPT-3 FC1)."""
+    """Decode-shaped W8A8 GEMM: M tokens against an [N, K] INT8 weight (default: GPT-3 FC1).
+    --fused: bf16 activations in, per-token quantisation in the kernel's prologue."""
     g = _gen()
     N, K = args.N, args.K
     Wq = torch.randint(-127, 128, (N, K), dtype=torch.int8, device="cuda", generator=g)
     w_scale = torch.rand(N, device="cuda", generator=g) * 1e-3
-    ws = sq.new_workspace(max(sq.workspace_bytes(sq.SQ_OP_GEMM, M, N, K) for M in args.M))
+    ws = sq.new_workspace(max(sq.workspace_bytes(sq.SQ_OP_GEMM_FUSED_QUANT, M, N, K) for M in args.M))
     for M in args.M:
-        X = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda", generator=g)
-        xs = torch.rand(M, device="cuda", generator=g)
         Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-        us = _time(lambda: sq.sq_w8a8_gemm(X, Wq, xs, w_scale, ws, out=Y), args.calls)
-        print("decode_gemm M=%d N=%d K=%d: %.1f us, %.0f GB/s of weights" % (M, N, K, us, N * K / us / 1e3))
+        if args.fused:
+            x = torch.randn((M, K), dtype=torch.bfloat16, device="cuda", generator=g)
+            us = _time(lambda: sq.sq_w8a8_gemm_fused_quant(x, Wq, w_scale, ws, "per_token", out=Y), args.calls)
+        else:
+            X = torch.randint(-127, 128, (M, K), dtype=torch.int8, device="cuda", generator=g)
+            xs = torch.rand(M, device="cuda", generator=g)
+            us = _time(lambda: sq.sq_w8a8_gemm(X, Wq, xs, w_scale, ws, out=Y), args.calls)
+        print("decode_gemm%s M=%d N=%d K=%d: %.1f us, %.0f GB/s of weights" % (
+            " (quantiser in the prologue)" if args.fused else "", M, N, K, us, N * K / us / 1e3))
     return ws
+
+
+def generation_block(args):
+    """One generation-stage step of the OPT-30B-shaped static W8A8 block (hidden 7168, 56 heads,
+    FFN 28672; batch --B, context --S cached positions): random INT8 weights and cache, fixed
+    static steps.  Seven launches per step; --fused: five (the LayerNorm+quantise steps run in the
+    prologues of the GEMMs that consume them)."""
+    from . import pipeline as pl
+    g = _gen()
+    H, d, hid, ffn, B = 56, 128, 7168, 28672, args.B
+    dt = torch.float16
+    lin = {}
+    for name, (N, K) in (("qkv", (3 * hid, hid)), ("out_proj", (hid, hid)), ("fc1", (ffn, hid)), ("fc2", (hid, ffn))):
+        lin[name] = pl.PreparedLinear(name, torch.randint(-127, 128, (N, K), dtype=torch.int8, device="cuda", generator=g),
+                                      torch.rand(N, device="cuda", generator=g) * 1e-3,
+                                      (torch.randn(N, device="cuda", generator=g) * 0.01).to(dt), name == "fc1")
+    for name in ("qkv", "fc1"):
+        lin[name].gamma_hat = (1 + 0.1 * torch.randn(hid, device="cuda", generator=g)).to(dt)
+        lin[name].beta_hat = (0.1 * torch.randn(hid, device="cuda", generator=g)).to(dt)
+    steps = dict(d_ln1=0.05, d_q=0.02, d_k=0.02, d_v=0.02, d_attn=0.01, d_ln2=0.05, d_fc1=0.02)
+    L_max = 2048
+    blk = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, dt, fused=args.fused)
+    blk.k_cache.random_(-100, 100, generator=g)
+    blk.v_cache.random_(-100, 100, generator=g)
+    blk.ctx.fill_(args.S)
+    blk.lens.fill_(args.S + 1)
+    x = torch.randn((B, hid), device="cuda", dtype=dt, generator=g)
+    us = _time(lambda: blk.step(x, advance=False), args.calls)
+    byts = blk.bytes_per_step(args.S * B)
+    print("generation_block B=%d ctx=%d, %d launches per step: %.1f us per step (stream, no graph), %.0f GB/s of weights + cache"
+          % (B, args.S, blk.launches_per_step, us, byts / us / 1e3))
+    return blk.ws
 
 
 def attention(args):
@@ -111,11 +190,17 @@ def quant_act(args):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("name", choices=["decode_gemm", "attention", "kv_attention", "ln_quant", "quant_act"])
+    ap.add_argument("name", choices=["gemm", "decode_gemm", "generation_block", "attention", "kv_attention", "ln_quant",
+                                     "quant_act"])
     ap.add_argument("--calls", type=int, default=20)
-    ap.add_argument("--M", type=lambda s: [int(v) for v in s.split(",")], default=[1, 16], help="decode_gemm: token counts")
-    ap.add_argument("--N", type=int, default=49152)
-    ap.add_argument("--K", type=int, default=12288)
+    ap.add_argument("--M", type=lambda s: [int(v) for v in s.split(",")], default=None,
+                    help="token counts (decode_gemm: 1,16; gemm: 2048)")
+    ap.add_argument("--N", type=int, default=None, help="output channels (decode_gemm: 49152; gemm: 20480)")
+    ap.add_argument("--K", type=int, default=None, help="input channels (decode_gemm: 12288; gemm: 5120)")
+    ap.add_argument("--values", choices=["full", "tri", "ones", "zeros"], default="full", help="gemm: operand value class")
+    ap.add_argument("--no-split", action="store_true", help="gemm: no scratch for the K split of the last wave")
+    ap.add_argument("--int-mm", action="store_true", help="gemm: also time torch._int_mm (cuBLASLt) for context")
+    ap.add_argument("--fused", action="store_true", help="decode_gemm / generation_block: quantiser inside the GEMM")
     ap.add_argument("--B", type=int, default=None, help="batch (attention: 4, kv_attention: 16)")
     ap.add_argument("--H", type=int, default=None, help="heads (attention: 56, kv_attention: 96)")
     ap.add_argument("--S", type=int, default=512)
@@ -126,6 +211,12 @@ def main(argv=None):
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise SystemExit("needs a CUDA device: the library has no CPU fallback")
+    if args.M is None:
+        args.M = [2048] if args.name == "gemm" else [1, 16]
+    if args.N is None:
+        args.N = 20480 if args.name == "gemm" else 49152
+    if args.K is None:
+        args.K = 5120 if args.name == "gemm" else 12288
     if args.B is None:
         args.B = 4 if args.name == "attention" else 16
     if args.H is None:

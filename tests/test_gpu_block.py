@@ -156,8 +156,9 @@ def test_host_streamed_block_matches_sequential_steps():
         assert torch.equal(o.view(torch.int16), w.view(torch.int16))
 
 
+@pytest.mark.parametrize("fused,fuse_residual", [(True, True), (False, True), (False, False)])
 @pytest.mark.parametrize("dtype", ["f16", "bf16"])
-def test_generation_stage_block_against_oracle(dtype):
+def test_generation_stage_block_against_oracle(dtype, fused, fuse_residual):
     """Prompt pass of 128 tokens with the prompt block, cache filled from its QKV codes, then three
     generated tokens through the generation-stage block; each step against the oracle's generation
     block, which walks its own caches (oracle prompt codes -> oracle cache)."""
@@ -180,7 +181,8 @@ def test_generation_stage_block_against_oracle(dtype):
     steps = {k: p[k] for k in ("d_ln1", "d_q", "d_k", "d_v", "d_attn", "d_ln2", "d_fc1")}
     blk = pl.DecoderBlockStatic(lin, steps, B, S, H, d, tdt)
     blk.forward(dev(x, dtype))
-    gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, tdt)
+    gen = pl.DecoderBlockDecode(lin, steps, B, H, d, L_max, tdt, fused=fused, fuse_residual=fuse_residual, keep_codes=True)
+    assert gen.launches_per_step == 9 - 2 * fused - 2 * fuse_residual
     gen.load_prompt(blk.qkv, S)
 
     def codes_close(name, got, ref, max_frac):
