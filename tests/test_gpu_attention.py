@@ -1,14 +1,16 @@
 """GPU parity of the fused causal INT8 attention kernel against the oracle's unfused definition
 (Q.K^T -> fp32 scores -> causal softmax -> P = round(127 p) -> P.V -> requant).
-The kernel sums each softmax row in a different order (online, tile by tile), so a P code that sits
-on a rounding boundary may differ by one and move an output code by one: compared by code distance
-and mismatch fraction, and against the library's own unfused chain."""
+The kernel sums each softmax row in a different order (online, tile by tile) and never writes P, so
+a P code whose exact value sits on a rounding boundary may be either neighbour.  Every output code
+must lie in the interval that the admissible P matrices allow (parity.attention_codes_valid); where
+no P code is ambiguous that interval is the oracle's single value."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from helpers import dev, host
+from parity import attention_codes_valid
 from paper_2211_10438_b200 import binding as sq
 from paper_2211_10438_b200 import synth
 
@@ -43,10 +45,17 @@ def test_fused_attention_against_oracle_chain(B, H, S):
     sq.sq_w8a8_attention(qd, B, H, S, d, alpha_qk, alpha_pv, dev(r), out, ws)
     torch.cuda.synchronize()
     assert sq.device_status(ws) == 0
-    got = host(out).astype(np.int32)
-    diff = np.abs(got - want.astype(np.int32))
-    assert diff.max() <= 2, "output codes differ by %d" % diff.max()
-    assert (diff != 0).mean() <= 5e-3, "%.4f of output codes differ" % (diff != 0).mean()
+    got = host(out).reshape(B, S, H, d)
+    v5 = qkv.reshape(B, S, 3, H, d)
+    for b in range(B):
+        for h in range(H):
+            q, k, v = (np.ascontiguousarray(v5[b, :, i, h]) for i in range(3))
+            _, scores = oracle.w8a8_bmm(q[None], k[None], float(alpha_qk), out_dtype="f32")
+            amb, multi, differ = attention_codes_valid(got[b, :, h], scores[0], np.arange(1, S + 1), v, alpha_pv,
+                                                       requant_mul=r, P_oracle=P[b, h])
+            # few P codes are ambiguous, and an output differs from the oracle's own only where the
+            # ambiguity leaves more than one valid value
+            assert amb <= 2e-3 and differ <= multi
     assert np.abs(want).max() > 20  # the comparison is not vacuous
     # the library's own unfused chain (fp16 scores) stays close: it differs by the score rounding only
     hid, row = H * d, 3 * H * d
