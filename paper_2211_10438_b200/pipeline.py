@@ -361,12 +361,16 @@ class DecoderBlockDecode:
         return w + 2 * self.H * self.d * (ctx_sum + self.B)
 
 
-def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
+def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5, clip_frac=0.0):
     """Static per-tensor steps for DecoderBlockStatic from calibration batches (each [B*S, H*d]):
-    the block is walked with DYNAMIC steps and floating-point intermediates, and the running
-    maximum of every tensor that will later be quantised statically is kept (Section 5.1:
-    smoothing factors and static steps are calibrated once, offline).  Every tensor operation is
-    a libsq call; only the final max-over-batches of a handful of scalars is host bookkeeping."""
+    the block is walked with DYNAMIC steps and floating-point intermediates, and for every tensor
+    that will later be quantised statically the absolute maximum of each calibration token is kept
+    (Section 5.1: smoothing factors and static steps are calibrated once, offline).  At the end the
+    static step of a tensor is Eq. 1's step of the largest token maximum over all batches, the
+    `clip_frac` largest tokens set aside first (Section 5.2; 0 = none).  Every tensor operation and
+    every step size is a libsq call (sq_token_absmax, sq_clipped_absmax); the host only moves the
+    resulting scalars.  LN1 / LN2 outputs are never materialised in floating point: their static step
+    is the largest of the per-batch steps the dynamic per-tensor quantiser found (no clipping there)."""
     dev = lin["qkv"].Wq.device
     M, hid, ffn = B * S, H * d, lin["fc1"].Wq.shape[0]
     row = 3 * hid
@@ -379,21 +383,24 @@ def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
     proj, h = e((M, hid), act_dtype), e((M, hid), act_dtype)
     x2q, xs2 = e((M, hid), torch.int8), e(1, torch.float32)
     f1 = e((M, ffn), act_dtype)
-    mx = {k: 0.0 for k in ("d_ln1", "d_q", "d_k", "d_v", "d_attn", "d_ln2", "d_fc1")}
+    names = ("d_ln1", "d_q", "d_k", "d_v", "d_attn", "d_ln2", "d_fc1")
+    token_max = {k: [] for k in names}   # per tensor: the token maxima of every batch (device tensors)
     t32 = lambda v: torch.tensor(v, dtype=torch.float32)
-    step = lambda absmax: float(torch.clamp(t32(absmax), min=1e-5) / t32(127.0))
 
-    def tensor_absmax(t, lo=0, hi=None):
-        a = torch.zeros(t.shape[1], dtype=torch.float32, device=dev)
-        sq.sq_calib_absmax(t, a)
-        return float(a[lo:hi].max())
+    def step_of(token_absmax):
+        """Eq. 1's step of the largest token maximum (libsq; one device scalar read back)."""
+        _, st = sq.sq_clipped_absmax(token_absmax, 0)
+        return float(st.item())
 
     for x in calib_batches:
         sq.sq_ln_quant(x, lin["qkv"].gamma_hat, lin["qkv"].beta_hat, eps, "per_tensor_dynamic", Xq=x1q, x_scale=xs,
                        workspace=ws)
         sq.sq_w8a8_gemm(x1q, lin["qkv"].Wq, xs, lin["qkv"].w_scale, ws, bias=lin["qkv"].bias, out=qkv_f)
-        d_ln1 = float(xs.item())
-        dq, dk, dv = (step(tensor_absmax(qkv_f, i * hid, (i + 1) * hid)) for i in range(3))
+        token_max["d_ln1"].append(xs.clone())  # the batch's own step (LN1's output is never materialised)
+        tm = [sq.sq_token_absmax(qkv_f[:, i * hid:(i + 1) * hid]) for i in range(3)]
+        for k, v in zip(("d_q", "d_k", "d_v"), tm):
+            token_max[k].append(v)
+        dq, dk, dv = (step_of(v) for v in tm)
         one = t32(1.0)
         r = torch.cat([torch.full((hid,), float(one / t32(v))) for v in (dq, dk, dv)]).to(torch.float32).to(dev)
         sq.sq_w8a8_gemm(x1q, lin["qkv"].Wq, xs, lin["qkv"].w_scale, ws, bias=lin["qkv"].bias, requant_mul=r, out=qkv_q)
@@ -403,7 +410,9 @@ def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
         sq.sq_softmax_quant_p(scores, P)
         sq.sq_w8a8_bmm(P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
                        float(t32(dv) / t32(127.0)), attn_f, (S * hid, d, hid), ws)
-        d_attn = step(tensor_absmax(attn_f))
+        ta = sq.sq_token_absmax(attn_f)
+        token_max["d_attn"].append(ta)
+        d_attn = step_of(ta)
         ra = torch.tensor([float(one / t32(d_attn))], dtype=torch.float32, device=dev)
         sq.sq_w8a8_bmm(P, flat[2 * hid:], B, H, S, d, S, (H * S * S, S * S, S), (S * row, d, row), True,
                        float(t32(dv) / t32(127.0)), attn_q, (S * hid, d, hid), ws, requant_mul=ra)
@@ -412,9 +421,17 @@ def calibrate_static_steps(lin, calib_batches, B, S, H, d, act_dtype, eps=1e-5):
         sq.sq_residual_add(x, proj, out=h)
         sq.sq_ln_quant(h, lin["fc1"].gamma_hat, lin["fc1"].beta_hat, eps, "per_tensor_dynamic", Xq=x2q, x_scale=xs2,
                        workspace=ws)
+        token_max["d_ln2"].append(xs2.clone())
         sq.sq_w8a8_gemm(x2q, lin["fc1"].Wq, xs2, lin["fc1"].w_scale, ws, bias=lin["fc1"].bias, relu=True, out=f1)
-        d_fc1 = step(tensor_absmax(f1))
-        for k, v in (("d_ln1", d_ln1), ("d_q", dq), ("d_k", dk), ("d_v", dv), ("d_attn", d_attn),
-                     ("d_ln2", float(xs2.item())), ("d_fc1", d_fc1)):
-            mx[k] = max(mx[k], v)
-    return mx
+        token_max["d_fc1"].append(sq.sq_token_absmax(f1))
+    out = {}
+    for k in names:
+        allmax = torch.cat(token_max[k])
+        if k in ("d_ln1", "d_ln2"):  # per-batch steps: the static step is the largest of them (a selection, no arithmetic)
+            largest, _ = sq.sq_clipped_absmax(allmax, 0)
+            out[k] = float(largest.item())
+        else:
+            n_clip = int(clip_frac * allmax.numel() + 0.5)
+            _, st = sq.sq_clipped_absmax(allmax, n_clip)
+            out[k] = float(st.item())
+    return out
