@@ -38,6 +38,15 @@ def build_trace() -> str:
     return out
 
 
+def build_issue_only() -> str:
+    """Ceiling build: libsq_issue_only.so, in which the prefill GEMM loads no operand and stores no result
+    (-DSQ_GEMM_ISSUE_ONLY): what the tensor pipe sustains on its own.  For `workloads gemm --lib ...` only."""
+    out = os.path.join(HERE, "libsq_issue_only.so")
+    subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSQ_GEMM_ISSUE_ONLY", "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out],
+                   check=True)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "sq.h"))
@@ -70,5 +79,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
 if __name__ == "__main__":
     if "--trace" in sys.argv:
         print(build_trace())
+    elif "--issue-only" in sys.argv:
+        print(build_issue_only())
     else:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

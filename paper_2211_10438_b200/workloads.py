@@ -193,6 +193,7 @@ def main(argv=None):
     ap.add_argument("name", choices=["gemm", "decode_gemm", "generation_block", "attention", "kv_attention", "ln_quant",
                                      "quant_act"])
     ap.add_argument("--calls", type=int, default=20)
+    ap.add_argument("--lib", default=None, help="path of another build of the library (libsq_issue_only.so, libsq_trace.so)")
     ap.add_argument("--M", type=lambda s: [int(v) for v in s.split(",")], default=None,
                     help="token counts (decode_gemm: 1,16; gemm: 2048)")
     ap.add_argument("--N", type=int, default=None, help="output channels (decode_gemm: 49152; gemm: 20480)")
@@ -221,6 +222,8 @@ def main(argv=None):
         args.B = 4 if args.name == "attention" else 16
     if args.H is None:
         args.H = 56 if args.name == "attention" else 96
+    if args.lib:
+        sq.LIB_PATH = args.lib
     sq.lib()
     ws = globals()[args.name](args)
     status = sq.device_status(ws)
