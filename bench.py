@@ -457,6 +457,62 @@ def run_reference(args):
     }))
 
 
+def run_tensor_parallel(args, device, world, rank, dist):
+    """ONE config-2 block (the same seeded weights on every rank) cut over the ranks: QKV / FC1 by output
+    channels, out-proj / FC2 by input channels, two max-all-reduces of [M] token maxima and two INT32
+    sum-all-reduces of [M, hidden] partial sums per step over NCCL.  Total work is fixed: strong scaling."""
+    from paper_2211_10438_b200 import binding as sq
+    from paper_2211_10438_b200 import tensor_parallel as tp
+    wl, block, x_in, attn_out, offline_s = build_block(device, seed_offset=0)  # identical on every rank
+    lin = block.lin
+    hd = wl.head_dim
+    tpb = tp.TensorParallelLinears(lin, block.M, wl.hidden, hd, torch.bfloat16, world, rank)
+    attn_slice = attn_out[:, tpb.head_lo:tpb.head_hi].contiguous()
+    ops_total = block.gemm_ops()
+    del block
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        tpb.step(x_in, attn_slice)
+    barrier()
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        tpb.step(x_in, attn_slice)
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1) * 1e-3], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    elapsed = float(t.item())
+    clocks = sampler.stop()
+    status = sq.device_status(tpb.ws)
+    if status != 0:
+        raise SystemExit("device status word = %d" % status)
+    if rank == 0:
+        print(json.dumps({
+            "metric": "W8A8 linear-layer throughput (4 GEMMs + activation quantisation)",
+            "value": ops_total * args.steps / elapsed / 1e12, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": "opt13b-prefill (config 2): hidden 5120, M=2048 tokens, bf16 activations, per-token dynamic "
+                                   "act / per-channel weight INT8, one block cut over the ranks",
+                       "parallelism": "tp%d" % world,
+                       "l2": "per-rank working set exceeds L2 up to 4 ranks; no flush"},
+            "clocks": clocks, "gpu_launches": (12 if world >= 1 else 0) * args.steps,
+            "exchange_bytes_per_rank_per_step": tpb.exchanged_bytes(),
+            "offline_setup_s": offline_s}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -465,6 +521,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-rows", action="store_true", help="skip the isolated per-row timings")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tp", action="store_true",
+                    help="with --gpus N: ONE config-2 block cut over the N ranks (tensor parallel, strong scaling) "
+                         "instead of N independent replicas")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps == 50 and args.warmup == 5:
@@ -486,6 +545,8 @@ def main():
     from paper_2211_10438_b200 import binding as sq
     sq.lib()  # fail loudly if the extension is missing
     peaks = measured_peaks()
+    if args.tp:
+        return run_tensor_parallel(args, device, world, rank, dist)
     wl, block, x_in, attn_out, offline_s = build_block(device, seed_offset=1000 * rank)
 
     def barrier():

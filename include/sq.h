@@ -175,6 +175,35 @@ sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_
                        size_t ws_bytes, void* stream);
 
 /*
+ * Two pieces for tensor-parallel serving of the W8A8 linears (Section 5.3 runs the larger models
+ * with FasterTransformer's tensor parallelism over up to 8 GPUs: QKV / FC1 split by output
+ * channels, out-proj / FC2 split by INPUT channels, partial results summed across GPUs).
+ *
+ * sq_quant_act_given_absmax: Eq. 1 per token when a token's channels are spread over several ranks.
+ * The per-token maximum must then be the maximum over ALL ranks' slices, or the ranks' codes would
+ * have different step sizes and their INT32 partial sums could not be added.  Each rank takes
+ * sq_token_absmax of its slice, the ranks exchange a max-all-reduce of those [M] values, and this
+ * call quantises the local slice with Delta_t = max(row_absmax[t], 1e-5) / 127 (written to
+ * x_scale[t]; identical on every rank).  X: [M, C] slice, contiguous; row_absmax: [M] fp32 INPUT.
+ * With row_absmax the slice's own maxima this is sq_quant_act(SQ_PER_TOKEN_DYNAMIC), bit for bit.
+ *
+ * sq_dequant_acc: Eq. 2 on INT32 accumulators that already sit in memory -- what the epilogue of
+ * sq_w8a8_gemm / sq_w8a8_gemm_residual computes, operation for operation, as a pass of its own:
+ *     y = fma((float)acc[t, o], x_scale[t] * w_scale[o], bias[o]), ReLU, then round to F16 / BF16
+ *     (optionally + residual, as in sq_w8a8_gemm_residual) or clamp(round(y * requant_mul)) to I8.
+ * A row-parallel layer runs sq_w8a8_gemm with out_dt = SQ_I32 on every rank (raw partial sums),
+ * the ranks add them with an INT32 sum-all-reduce (exact: the result is bit for bit that of the
+ * unsharded layer), and this call dequantises the sum once.  acc: [M, N] int32, row stride ld_acc
+ * (a multiple of 4), 16-byte aligned; N a multiple of 8; Y: row stride ldy a multiple of 8.
+ */
+sq_status sq_quant_act_given_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* row_absmax,
+                                    int8_t* Xq, float* x_scale, void* workspace, size_t ws_bytes, void* stream);
+sq_status sq_dequant_acc(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* x_scale,
+                         int x_scale_is_per_token, const float* w_scale, int w_scale_is_per_channel, const void* bias,
+                         sq_dtype bias_dt, sq_epilogue_act act, const float* requant_mul, int requant_is_per_channel,
+                         const void* residual, int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy, void* stream);
+
+/*
  * Fused LayerNorm (with the smoothing factor already folded into gamma_hat, beta_hat by
  * sq_fold_ln_weight) + Eq. 1, one pass over X:
  *     mu_t, var_t = mean and biased variance of row t: fp32, one pass -- per-thread (mean, sum of

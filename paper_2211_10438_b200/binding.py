@@ -28,7 +28,7 @@ EXPORTS = ["sq_status_str", "sq_workspace_bytes", "sq_calib_absmax", "sq_smooth_
            "sq_fold_ln_weight", "sq_quant_weight", "sq_quant_act", "sq_ln_quant", "sq_w8a8_gemm", "sq_w8a8_gemm_residual",
            "sq_w8a8_bmm", "sq_softmax_quant_p", "sq_residual_add", "sq_ln_quant_tensor_noalloc",
            "sq_selftest_bounded_wait", "sq_w8a8_attention", "sq_kv_cache_write", "sq_w8a8_decode_attention",
-           "sq_token_absmax", "sq_clipped_absmax", "sq_selftest_row_wait", "sq_w8a8_gemm_fused_quant"]
+           "sq_token_absmax", "sq_clipped_absmax", "sq_selftest_row_wait", "sq_w8a8_gemm_fused_quant", "sq_quant_act_given_absmax", "sq_dequant_acc"]
 
 _DT = {torch.float16: SQ_F16, torch.bfloat16: SQ_BF16, torch.int8: SQ_I8, torch.int32: SQ_I32}
 GRAN = {"per_tensor_static": SQ_PER_TENSOR_STATIC, "per_tensor_dynamic": SQ_PER_TENSOR_DYNAMIC,
@@ -70,6 +70,8 @@ def lib():
                                             vp, sz, vp]
         L.sq_w8a8_gemm_fused_quant.argtypes = [vp, i32, i64, i64, i64, vp, vp, f32, i32, vp, vp, vp, vp, vp, i32, vp, i32, i32,
                                                vp, i32, vp, i64, vp, i32, i64, vp, sz, vp]
+        L.sq_quant_act_given_absmax.argtypes = [vp, i32, i64, i64, vp, vp, vp, vp, sz, vp]
+        L.sq_dequant_acc.argtypes = [vp, i64, i64, i64, vp, i32, vp, i32, vp, i32, i32, vp, i32, vp, i64, vp, i32, i64, vp]
         L.sq_w8a8_bmm.argtypes = [vp, vp, i64, i64, i64, i64, i64, c.POINTER(i64), c.POINTER(i64), i32, i32,
                                   f32, vp, vp, i32, c.POINTER(i64), vp, sz, vp]
         L.sq_softmax_quant_p.argtypes = [vp, i32, i64, i64, vp, vp]
@@ -182,6 +184,36 @@ def sq_quant_act(X, gran, col_mul=None, Xq=None, x_scale=None, workspace=None):
     _check(lib().sq_quant_act(_ptr(X), _DT[X.dtype], M, C, g, _ptr(col_mul), _ptr(Xq), _ptr(x_scale), wp,
                               wn, _stream()), "sq_quant_act")
     return Xq, x_scale
+
+
+def sq_quant_act_given_absmax(X, row_absmax, Xq=None, x_scale=None, workspace=None):
+    """Per-token Eq. 1 with the token maxima given (agreed on across tensor-parallel ranks) -> (Xq, x_scale[M])."""
+    M, C = X.shape
+    if Xq is None:
+        Xq = torch.empty((M, C), dtype=torch.int8, device=X.device)
+    if x_scale is None:
+        x_scale = torch.empty(M, dtype=torch.float32, device=X.device)
+    wp, wn = _ws(workspace)
+    _check(lib().sq_quant_act_given_absmax(_ptr(X), _DT[X.dtype], M, C, _ptr(row_absmax), _ptr(Xq), _ptr(x_scale), wp, wn,
+                                           _stream()), "sq_quant_act_given_absmax")
+    return Xq, x_scale
+
+
+def sq_dequant_acc(acc, x_scale, w_scale, bias=None, relu=False, requant_mul=None, residual=None, out=None,
+                   out_dtype=torch.float16):
+    """Eq. 2 on an INT32 accumulator matrix [M, N] (the sum of tensor-parallel partial sums)."""
+    M, N = acc.shape
+    if out is None:
+        odt = torch.int8 if requant_mul is not None else (residual.dtype if residual is not None else out_dtype)
+        out = torch.empty((M, N), dtype=odt, device=acc.device)
+    _check(lib().sq_dequant_acc(
+        _ptr(acc), acc.stride(0), M, N, _ptr(x_scale), 1 if x_scale.numel() > 1 else 0, _ptr(w_scale),
+        1 if w_scale.numel() > 1 else 0, _ptr(bias), _DT[bias.dtype] if bias is not None else SQ_F16,
+        SQ_EPI_RELU if relu else SQ_EPI_NONE, _ptr(requant_mul),
+        1 if (requant_mul is not None and requant_mul.numel() > 1) else 0, _ptr(residual),
+        residual.stride(0) if residual is not None else 0, _ptr(out), _DT[out.dtype], out.stride(0), _stream()),
+        "sq_dequant_acc")
+    return out
 
 
 def sq_ln_quant(X, gamma_hat, beta_hat, eps, gran, Xq=None, x_scale=None, dbg_mean_rstd=None,

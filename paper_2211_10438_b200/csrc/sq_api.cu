@@ -163,6 +163,40 @@ sq_status sq_quant_act(const void* X, sq_dtype dt, int64_t M, int64_t C, sq_act_
                              as_stream(stream));
 }
 
+sq_status sq_quant_act_given_absmax(const void* X, sq_dtype dt, int64_t M, int64_t C, const float* row_absmax,
+                                    int8_t* Xq, float* x_scale, void* workspace, size_t ws_bytes, void* stream) {
+    if (!is_act_dtype(dt)) return SQ_ERR_INVALID_ARG;
+    if (M < 0 || C < 0) return SQ_ERR_SHAPE;
+    if (M == 0 || C == 0) return SQ_OK;
+    if (!X || !Xq || !x_scale || !row_absmax) return SQ_ERR_INVALID_ARG;
+    if (C % 8 != 0 || !aligned16(X) || (reinterpret_cast<uintptr_t>(Xq) & 7) != 0) return SQ_ERR_ALIGN;
+    uint32_t* status = ws_ok(workspace, ws_bytes, sizeof(uint32_t)) ? static_cast<uint32_t*>(workspace) : nullptr;
+    return row_quant(X, dt, M, C, nullptr, nullptr, nullptr, 0.0f, false, ROW_GIVEN_ROW_ABSMAX, Xq, x_scale,
+                     const_cast<float*>(row_absmax), nullptr, 0, status, as_stream(stream));
+}
+
+sq_status sq_dequant_acc(const int32_t* acc, int64_t ld_acc, int64_t M, int64_t N, const float* x_scale,
+                         int x_scale_is_per_token, const float* w_scale, int w_scale_is_per_channel, const void* bias,
+                         sq_dtype bias_dt, sq_epilogue_act act, const float* requant_mul, int requant_is_per_channel,
+                         const void* residual, int64_t ld_res, void* Y, sq_dtype out_dt, int64_t ldy, void* stream) {
+    if (M < 0 || N < 0) return SQ_ERR_SHAPE;
+    if (out_dt < SQ_F16 || out_dt > SQ_I8 || (act != SQ_EPI_NONE && act != SQ_EPI_RELU)) return SQ_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return SQ_OK;
+    if (!acc || !Y || !x_scale || !w_scale) return SQ_ERR_INVALID_ARG;
+    if ((out_dt == SQ_I8) != (requant_mul != nullptr)) return SQ_ERR_INVALID_ARG;
+    if (bias && !is_act_dtype(bias_dt)) return SQ_ERR_INVALID_ARG;
+    if (residual && (out_dt == SQ_I8 || act != SQ_EPI_NONE)) return SQ_ERR_INVALID_ARG;
+    if (ld_acc < N || ldy < N || (residual && ld_res < N)) return SQ_ERR_SHAPE;
+    const int64_t out_vec = out_dt == SQ_I8 ? 8 : 8;  // 8 outputs per store: 8 or 16 bytes
+    if (N % 8 != 0 || ld_acc % 4 != 0 || ldy % out_vec != 0 || !aligned16(acc) ||
+        (reinterpret_cast<uintptr_t>(Y) & (out_dt == SQ_I8 ? 7 : 15)) != 0 ||
+        (residual && (!aligned16(residual) || ld_res % 8 != 0)))
+        return SQ_ERR_ALIGN;
+    DequantArgs a{acc, ld_acc, M, N, x_scale, x_scale_is_per_token, w_scale, w_scale_is_per_channel, bias, bias_dt,
+                  act == SQ_EPI_RELU, requant_mul, requant_is_per_channel, residual, ld_res, Y, out_dt, ldy};
+    return dequant_acc(a, as_stream(stream));
+}
+
 sq_status sq_ln_quant(const void* X, sq_dtype dt, int64_t M, int64_t C, const void* gamma_hat,
                       const void* beta_hat, float eps, sq_act_gran g, int8_t* Xq, float* x_scale,
                       float* dbg_mean_rstd, void* workspace, size_t ws_bytes, void* stream) {

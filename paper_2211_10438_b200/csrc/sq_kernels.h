@@ -14,7 +14,9 @@ enum RowMode {
     ROW_DYNAMIC = 0,          // Delta_row = absmax(row)/127, written to scale[row]
     ROW_GIVEN_SCALE = 1,      // Delta = scale[0], an input (static)
     ROW_FROM_ABSMAX_WORD = 2, // Delta = step_size(*absmax_word); scale[0] receives it
-    ROW_ABSMAX_ONLY = 3       // no codes: atomically fold the row's absmax into *absmax_word
+    ROW_ABSMAX_ONLY = 3,      // no codes: atomically fold the row's absmax into *absmax_word
+    ROW_GIVEN_ROW_ABSMAX = 4  // Delta_row = step_size(absmax_word[row]), an INPUT array [M] (a maximum agreed on
+                              // across tensor-parallel ranks); written to scale[row]; larger values saturate
 };
 
 // Workspace layout (bytes).  Word 0 is the sticky device status.
@@ -47,6 +49,16 @@ sq_status softmax_quant_p(const void* scores, sq_dtype dt, int64_t n_mat, int64_
                           cudaStream_t st);
 sq_status residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out,
                        cudaStream_t st);
+// Eq. 2 (+ bias, ReLU, re-quantisation, residual add) on INT32 accumulators that already sit in memory
+struct DequantArgs {
+    const int32_t* acc; int64_t ld_acc; int64_t M, N;
+    const float* x_scale; int x_per_row; const float* w_scale; int w_per_col;
+    const void* bias; sq_dtype bias_dt; int relu;
+    const float* requant_mul; int requant_per_col;
+    const void* residual; int64_t ld_res;
+    void* Y; sq_dtype out_dt; int64_t ldy;
+};
+sq_status dequant_acc(const DequantArgs& a, cudaStream_t st);
 
 // Batched INT8 GEMM on the tensor cores (tcgen05, kind::i8) with the fused epilogue.
 struct GemmArgs {

@@ -354,10 +354,13 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
             }
             delta = step_size(m);
             if (gt == 0) scale[row] = delta;
+        } else if (mode == ROW_GIVEN_ROW_ABSMAX) {  // the row's maximum was agreed on elsewhere (all ranks' slices)
+            delta = step_size(__ldg(absmax_word + row));
+            if (gt == 0) scale[row] = delta;
         }
         const float inv = recip_step(delta);
         uint2* qrow = reinterpret_cast<uint2*>(Xq + row * C);
-        if (mode == ROW_GIVEN_SCALE) {  // a calibrated step may be exceeded at run time: saturate
+        if (mode == ROW_GIVEN_SCALE || mode == ROW_GIVEN_ROW_ABSMAX) {  // a given step may be exceeded: saturate
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 const int v = gt + i * GROUP;

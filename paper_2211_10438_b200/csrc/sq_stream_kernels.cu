@@ -519,6 +519,9 @@ row_quant_kernel(const T* __restrict__ X, int64_t M, int64_t C, const float* __r
         if (lead) scale[row] = delta;
     } else if (mode == ROW_GIVEN_SCALE) {
         delta = __ldg(scale);
+    } else if (mode == ROW_GIVEN_ROW_ABSMAX) {
+        delta = step_size(__ldg(absmax_word + row));
+        if (lead) scale[row] = delta;
     } else {  // ROW_FROM_ABSMAX_WORD
         delta = step_size(__ldg(absmax_word));
         if (row == 0 && lead) scale[0] = delta;
@@ -715,6 +718,63 @@ __global__ void residual_add_kernel(const uint4* __restrict__ a, const uint4* __
         for (int k = 0; k < 8; ++k) r[k] = Act<T>::from_float(__fadd_rn(fa[k], fb[k]));
         out[i] = *reinterpret_cast<uint4*>(r);
     }
+}
+
+// Eq. 2 on a matrix of INT32 accumulators that already sits in memory: the epilogue of the GEMM
+// kernels as a pass of its own.  Tensor-parallel row-parallel layers need it: every rank's GEMM
+// leaves raw partial sums, the ranks add them exactly as integers, and the sum is dequantised once.
+// Same arithmetic, operation for operation, as the fused epilogues.  One thread = 8 columns.
+template <typename T>
+__global__ void __launch_bounds__(256)
+dequant_acc_kernel(const DequantArgs a) {
+    pdl_wait();
+    pdl_launch_dependents();
+    const int64_t nvec = a.N >> 3;
+    const int64_t total = a.M * nvec;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / nvec, col = (i - row * nvec) << 3;
+        const int4* src = reinterpret_cast<const int4*>(a.acc + row * a.ld_acc + col);
+        const int4 lo = __ldcs(src), hi = __ldcs(src + 1);
+        const int32_t acc[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+        const float xs = __ldg(a.x_scale + (a.x_per_row ? row : 0));
+        float y[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float ws = __ldg(a.w_scale + (a.w_per_col ? col + k : 0));
+            const float bs = a.bias == nullptr ? 0.0f
+                             : (a.bias_dt == SQ_BF16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.bias)[col + k])
+                                                     : __half2float(static_cast<const __half*>(a.bias)[col + k]));
+            float v = __fmaf_rn(__int2float_rn(acc[k]), __fmul_rn(xs, ws), bs);
+            if (a.relu) v = fmaxf(v, 0.0f);
+            y[k] = v;
+        }
+        if (a.out_dt == SQ_I8) {
+            uint32_t c[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) c[k] = quant_code(y[k], __ldg(a.requant_mul + (a.requant_per_col ? col + k : 0)));
+            *reinterpret_cast<uint2*>(static_cast<int8_t*>(a.Y) + row * a.ldy + col) =
+                make_uint2(pack4(c[0], c[1], c[2], c[3]), pack4(c[4], c[5], c[6], c[7]));
+        } else {
+            if (a.residual != nullptr) {  // round to the output type, then the residual add (rounded by the store)
+                float r[8];
+                unpack8<T>(__ldg(reinterpret_cast<const uint4*>(static_cast<const T*>(a.residual) + row * a.ld_res + col)), r);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) y[k] = __fadd_rn(Act<T>::to_float(Act<T>::from_float(y[k])), r[k]);
+            }
+            __align__(16) T o[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = Act<T>::from_float(y[k]);
+            *reinterpret_cast<uint4*>(static_cast<T*>(a.Y) + row * a.ldy + col) = *reinterpret_cast<const uint4*>(o);
+        }
+    }
+}
+
+sq_status dequant_acc(const DequantArgs& a, cudaStream_t st) {
+    const int64_t total = a.M * (a.N >> 3);
+    const unsigned grid = (unsigned)std::min<int64_t>((total + 255) / 256, 16LL * sm_count());
+    if (a.out_dt == SQ_BF16)
+        return launch_pdl(dequant_acc_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, 1, a);
+    return launch_pdl(dequant_acc_kernel<__half>, dim3(grid), dim3(256), 0, st, 1, a);  // also SQ_I8 (T unused there)
 }
 
 sq_status residual_add(const void* a, const void* b, sq_dtype dt, int64_t n, void* out,
