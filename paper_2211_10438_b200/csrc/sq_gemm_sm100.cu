@@ -83,15 +83,28 @@ struct Params {
     int split, kb_per_piece;
     int32_t* part;
     uint32_t* counters;
+    // N split of the last wave, for reductions too short for the K split (nsplit == 1: none): unit
+    // full_tiles + t * nsplit + i is column part i (BLOCK_N / nsplit wide, the whole K range) of tile
+    // full_tiles + t.  No exchange is needed; the A tile is simply fetched once per part.
+    int nsplit;
 };
 
-// unit id -> tile and K-block range; piece < 0 for a whole tile (kb1 is then the tile's own count)
-__device__ __forceinline__ void unit_of(uint32_t u, const Params& p, uint32_t& tile, int& kb0, int& kb1, int& piece) {
+// unit id -> tile and K-block range; piece < 0 for a whole tile (kb1 is then the tile's own count);
+// npart >= 0: the unit is column part npart of its tile (whole K range)
+__device__ __forceinline__ void unit_of(uint32_t u, const Params& p, uint32_t& tile, int& kb0, int& kb1, int& piece,
+                                        int& npart) {
+    npart = -1;
     if (u < p.full_tiles) {
         tile = u; kb0 = 0; kb1 = -1; piece = -1;
         return;
     }
     const uint32_t r = u - p.full_tiles;
+    if (p.nsplit > 1) {
+        const uint32_t t = r / (uint32_t)p.nsplit;
+        npart = (int)(r - t * (uint32_t)p.nsplit);
+        tile = p.full_tiles + t; kb0 = 0; kb1 = -1; piece = -1;
+        return;
+    }
     const uint32_t t = r / (uint32_t)p.split;
     piece = (int)(r - t * (uint32_t)p.split);
     tile = p.full_tiles + t;
@@ -369,7 +382,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
 template <int BLOCK_N, int CG, int EW>
 __global__ void __launch_bounds__(EW * 32 + 64, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const __grid_constant__ CUtensorMap tmap_c, const Params p) {
+               const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bp, const Params p) {
     using C = Cfg<BLOCK_N, CG, EW>;
     extern __shared__ uint8_t smem_raw[];
     // identical layout in both CTAs of a pair (the MMA addresses both with one descriptor)
@@ -423,8 +436,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             bool ok = true;
             for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
                 uint32_t tile;
-                int kb0, kb1, piece;
-                unit_of(u, p, tile, kb0, kb1, piece);
+                int kb0, kb1, piece, npart;
+                unit_of(u, p, tile, kb0, kb1, piece, npart);
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -433,7 +446,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 int ca[4] = {0, 0, 0, 0}, cb[4] = {0, 0, 0, 0};
                 ca[p.a_slot_row] = (mi * CG + rank) * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
                 cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
-                const int b_row0 = ni * BLOCK_N + rank * C::B_ROWS;  // this CTA's share of the B tile
+                // this CTA's share of the B tile (of the column part, whose own map has a smaller box)
+                const int part_rows = npart >= 0 ? C::B_ROWS / p.nsplit : C::B_ROWS;
+                const int b_row0 = ni * BLOCK_N + (npart >= 0 ? npart * (BLOCK_N / p.nsplit) : 0) + rank * part_rows;
+                const CUtensorMap* mapb = npart >= 0 ? &tmap_bp : &tmap_b;
+                const uint32_t stage_tx = (uint32_t)(C::A_BYTES + part_rows * BLOCK_K) * CG;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
                     uint8_t* sa = stage_base + stage * C::STAGE_BYTES;
@@ -446,7 +463,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                     continue;
 #endif
-                    if (rank == 0) mbar_expect_tx(full_bar + stage, C::STAGE_BYTES * CG);
+                    if (rank == 0) mbar_expect_tx(full_bar + stage, stage_tx);
                     ca[0] = kb * BLOCK_K;
                     tma_load_4d<CG>(sa, &tmap_a, full_bar + stage, ca[0], ca[1], ca[2], ca[3]);
                     if (p.b_is_kn) {  // B stored [K, N]: x walks N, the row slot walks K
@@ -456,7 +473,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         cb[0] = kb * BLOCK_K;
                         cb[p.b_slot_row] = b_row0;
                     }
-                    tma_load_4d<CG>(sb, &tmap_b, full_bar + stage, cb[0], cb[1], cb[2], cb[3]);
+                    tma_load_4d<CG>(sb, mapb, full_bar + stage, cb[0], cb[1], cb[2], cb[3]);
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -474,12 +491,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             bool ok = true;
             for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
                 uint32_t tile;
-                int kb0, kb1, piece;
-                unit_of(u, p, tile, kb0, kb1, piece);
+                int kb0, kb1, piece, npart;
+                unit_of(u, p, tile, kb0, kb1, piece, npart);
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
                 if (piece < 0) kb1 = tile_num_kb(p, mi, BLOCK_M * CG);
+                const uint32_t idesc_u = npart >= 0 ? make_idesc(BLOCK_M * CG, BLOCK_N / p.nsplit, p.b_is_kn) : idesc;
                 if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
@@ -492,7 +510,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
                         const uint64_t adesc = make_smem_desc(sa + k * UMMA_K, 16);
                         const uint64_t bdesc = make_smem_desc(sb + k * b_kstep, p.b_is_kn ? 16384u : 16u);
-                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc_u, (kb > kb0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit<CG>(empty_bar + stage);  // frees the stage (in both CTAs) once these MMAs retire
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
@@ -515,15 +533,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         uint32_t slot_phase = 0;
         for (uint32_t u = first_tile; u < p.total_units; u += tile_step) {
             uint32_t tile;
-            int kb0, kb1, piece;
-            unit_of(u, p, tile, kb0, kb1, piece);
+            int kb0, kb1, piece, npart;
+            unit_of(u, p, tile, kb0, kb1, piece, npart);
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
             if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
             const int b = bh / p.heads, h = bh - b * p.heads;
-            const int64_t col0 = (int64_t)ni * BLOCK_N;
+            const int width = npart >= 0 ? BLOCK_N / p.nsplit : BLOCK_N;  // columns of this unit
+            const int64_t col0 = (int64_t)ni * BLOCK_N + (npart >= 0 ? npart * width : 0);
             // stage this tile's per-column constants
-            for (int c = et; c < BLOCK_N; c += C::EPI_THREADS) {
+            for (int c = et; c < width; c += C::EPI_THREADS) {
                 const int64_t col = col0 + c;
                 const bool in = col < p.N;
                 float ws = 1.0f, rq = 1.0f, bs = 0.0f;
@@ -542,7 +561,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 const int64_t prow = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
                 if (prow < p.M) {
                     const char* base = reinterpret_cast<const char*>(static_cast<const uint16_t*>(p.residual) + prow * p.ld_res + col0);
-                    const int64_t bytes = 2 * min((int64_t)BLOCK_N, p.N - col0);
+                    const int64_t bytes = 2 * min((int64_t)width, p.N - col0);
                     for (int64_t off = half * 128; off < bytes; off += (EW == 8 ? 256 : 128))
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
                 }
@@ -561,10 +580,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             // split the tile's 32-column chunks between the two warps of this lane quarter, in whole
             // store groups (a staged TMA store covers 128 bytes of a row = 1, 2 or 4 chunks)
             const int cps = p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2);
-            const int groups = (BLOCK_N / 32 + cps - 1) / cps;
+            const int groups = (width / 32 + cps - 1) / cps;
             const int g_split = EW == 8 ? (groups + 1) / 2 : groups;
             const int cc_begin = half == 0 ? 0 : g_split * cps;
-            const int cc_end = half == 0 ? min(g_split * cps, BLOCK_N / 32) : BLOCK_N / 32;
+            const int cc_end = half == 0 ? min(g_split * cps, width / 32) : width / 32;
             if (EW == 8 || piece < 0) {  // (the eight-warp configuration serves short reductions: never split)
                 epilogue_slot<BLOCK_N, false, EW == 8>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
                                        c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
@@ -757,9 +776,30 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
             p.part = reinterpret_cast<int32_t*>(ws + kWsHeader + kDecCounterBytes);
         }
     }
+    // N split of the last wave: plain GEMMs whose reduction is too short for the K split.  With R tiles left
+    // over after the full waves, cutting each into 2 or 4 column parts that still fit ONE round shortens the
+    // last wave to a half or a quarter of a tile time; the parts need no exchange, only the A tile again.
+    // Measured on B200 (full-range codes): 2048 x 5120 x 5120 50.6 -> 47.2 us, 2048 x 15360 x 5120 112.6 -> 111.7,
+    // 512 x 28672 x 7168 87.4 -> 85.4, 512 x 21504 x 7168 67.8 -> 66.7 (quarters; halves gain about half of that).
+    p.nsplit = 1;
+    CUtensorMap mbp = mb;  // placeholder unless the split is taken
+    if (BLOCK_N == 256 && CG == 2 && p.split == 1 && a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn) {
+        const int64_t G = sm_count() / CG;
+        const int64_t R = (int64_t)p.total_tiles % G;
+        const int max_ns = a.out_dt == SQ_I8 ? 2 : 4;  // a staged store row is 128 bytes: a part must fill it
+        const int ns = (p.total_tiles > G && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
+        if (ns > 1) {
+            if (!make_map(&mbp, a.B, 1, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0], BLOCK_K,
+                          C::B_ROWS / ns, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch))
+                return SQ_ERR_CUDA;
+            p.nsplit = ns;
+            p.full_tiles = (uint32_t)(p.total_tiles - R);
+            p.total_units = p.full_tiles + (uint32_t)R * (uint32_t)ns;
+        }
+    }
     const int groups = (int)std::min<int64_t>((int64_t)p.total_units, sm_count() / CG);
     return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
-                      (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, p);
+                      (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
 }
 
 // Short reductions (few K slices per tile) are bound by draining the accumulators: give them
