@@ -91,6 +91,7 @@ struct Params {
 
 // unit id -> tile and K-block range; piece < 0 for a whole tile (kb1 is then the tile's own count);
 // npart >= 0: the unit is column part npart of its tile (whole K range)
+template <bool NS>
 __device__ __forceinline__ void unit_of(uint32_t u, const Params& p, uint32_t& tile, int& kb0, int& kb1, int& piece,
                                         int& npart) {
     npart = -1;
@@ -99,7 +100,7 @@ __device__ __forceinline__ void unit_of(uint32_t u, const Params& p, uint32_t& t
         return;
     }
     const uint32_t r = u - p.full_tiles;
-    if (p.nsplit > 1) {
+    if (NS) {
         const uint32_t t = r / (uint32_t)p.nsplit;
         npart = (int)(r - t * (uint32_t)p.nsplit);
         tile = p.full_tiles + t; kb0 = 0; kb1 = -1; piece = -1;
@@ -379,7 +380,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
 // ------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N, int CG, int EW>
+template <int BLOCK_N, int CG, int EW, bool NS = false>
 __global__ void __launch_bounds__(EW * 32 + 64, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bp, const Params p) {
@@ -437,7 +438,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
                 uint32_t tile;
                 int kb0, kb1, piece, npart;
-                unit_of(u, p, tile, kb0, kb1, piece, npart);
+                unit_of<NS>(u, p, tile, kb0, kb1, piece, npart);
                 int bh, mi, ni;
                 tile_coords(tile, p, bh, mi, ni);
                 if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
@@ -447,9 +448,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 ca[p.a_slot_row] = (mi * CG + rank) * BLOCK_M; ca[p.a_slot_head] = h; ca[p.a_slot_batch] = b;
                 cb[p.b_slot_head] = h; cb[p.b_slot_batch] = b;
                 // this CTA's share of the B tile (of the column part, whose own map has a smaller box)
-                const int part_rows = npart >= 0 ? C::B_ROWS / p.nsplit : C::B_ROWS;
-                const int b_row0 = ni * BLOCK_N + (npart >= 0 ? npart * (BLOCK_N / p.nsplit) : 0) + rank * part_rows;
-                const CUtensorMap* mapb = npart >= 0 ? &tmap_bp : &tmap_b;
+                const int part_rows = (NS && npart >= 0) ? C::B_ROWS / p.nsplit : C::B_ROWS;
+                const int b_row0 = ni * BLOCK_N + ((NS && npart >= 0) ? npart * (BLOCK_N / p.nsplit) : 0) + rank * part_rows;
+                const CUtensorMap* mapb = (NS && npart >= 0) ? &tmap_bp : &tmap_b;
                 const uint32_t stage_tx = (uint32_t)(C::A_BYTES + part_rows * BLOCK_K) * CG;
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag, p.status, 1))) break;
@@ -480,10 +481,23 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
     } else if (warp == EW + 1) {
         // ============================ MMA issuer (even CTA only) ==============
-        if (lane == 0 && rank == 0) {
+        // The WHOLE warp walks the units and waits on the barriers, converged; one elected lane issues the MMAs
+        // and commits.  Everything the MMA instruction takes is then warp-uniform to the compiler (under a
+        // `lane == 0` branch it is not, and every operand is first moved to a uniform register, lane by lane).
+        if (rank == 0) {
             const uint32_t idesc = make_idesc(BLOCK_M * CG, BLOCK_N, p.b_is_kn);
-            // bytes between consecutive K=32 slices inside a stage
-            const uint32_t b_kstep = p.b_is_kn ? (uint32_t)(UMMA_K * 128) : (uint32_t)UMMA_K;
+            // The loop over the K blocks takes about as long as the tensor pipe needs for them (four MMAs
+            // of 128 cycles): it is kept short -- descriptors as running low words, barriers by their
+            // shared-memory addresses, the slow path of a wait out of line -- so that the warp gets ahead of
+            // the pipe and the epilogue warps' instructions, which share its scheduler, cannot hold it up.
+            constexpr uint32_t kStage16 = (uint32_t)C::STAGE_BYTES >> 4;
+            const uint32_t a_lo0 = smem_desc_lo(smem_u32(stage_base), 16);
+            const uint32_t b_lo0 = smem_desc_lo(smem_u32(stage_base) + (uint32_t)C::A_BYTES, p.b_is_kn ? 16384u : 16u);
+            // descriptor step between consecutive K=32 slices inside a stage (in 16-byte units)
+            const uint32_t a_k16 = (uint32_t)UMMA_K >> 4;
+            const uint32_t b_k16 = (p.b_is_kn ? (uint32_t)(UMMA_K * 128) : (uint32_t)UMMA_K) >> 4;
+            const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+            const uint32_t tmem_full0 = smem_u32(tmem_full), tmem_empty0 = smem_u32(tmem_empty);
             int stage = 0;
             uint32_t phase = 0;
             int slot = 0;
@@ -492,31 +506,43 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
                 uint32_t tile;
                 int kb0, kb1, piece, npart;
-                unit_of(u, p, tile, kb0, kb1, piece, npart);
-                int bh, mi, ni;
-                tile_coords(tile, p, bh, mi, ni);
-                if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
-                if (piece < 0) kb1 = tile_num_kb(p, mi, BLOCK_M * CG);
-                const uint32_t idesc_u = npart >= 0 ? make_idesc(BLOCK_M * CG, BLOCK_N / p.nsplit, p.b_is_kn) : idesc;
-                if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 2))) break;
+                unit_of<NS>(u, p, tile, kb0, kb1, piece, npart);
+                // This lane is never more than about one MMA ahead of the tensor pipe: whatever it computes
+                // between two tiles is time the pipe idles.  A tile's coordinates (three dependent integer
+                // divisions, several hundred cycles) matter to this role only under a causal mask.
+                if (p.causal) {
+                    int bh, mi, ni;
+                    tile_coords(tile, p, bh, mi, ni);
+                    if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
+                    if (piece < 0) kb1 = tile_num_kb(p, mi, BLOCK_M * CG);
+                } else if (piece < 0) {
+                    kb1 = p.num_kb;
+                }
+                const uint32_t idesc_u = (NS && npart >= 0) ? make_idesc(BLOCK_M * CG, BLOCK_N / p.nsplit, p.b_is_kn) : idesc;
+                if (!(ok = mbar_wait_warp(tmem_empty + slot, tmem_empty0 + (uint32_t)slot * 8u, slot_phase ^ 1u, abort_flag,
+                                          p.status, 2)))
+                    break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
+                uint32_t accumulate = 0u;  // the tile's first MMA overwrites the slot
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 3))) break;
+                    if (!(ok = mbar_wait_warp(full_bar + stage, full0 + (uint32_t)stage * 8u, phase, abort_flag, p.status, 3)))
+                        break;
                     tcgen05_fence_after();
-                    const uint32_t sa = smem_u32(stage_base + stage * C::STAGE_BYTES);
-                    const uint32_t sb = sa + C::A_BYTES;
+                    const uint32_t a_lo = a_lo0 + (uint32_t)stage * kStage16;
+                    const uint32_t b_lo = b_lo0 + (uint32_t)stage * kStage16;
+                    if (elect_one()) {
+                        umma_i8_lo<CG>(d_tmem, a_lo, b_lo, idesc_u, accumulate);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                        const uint64_t adesc = make_smem_desc(sa + k * UMMA_K, 16);
-                        const uint64_t bdesc = make_smem_desc(sb + k * b_kstep, p.b_is_kn ? 16384u : 16u);
-                        umma_i8<CG>(d_tmem, adesc, bdesc, idesc_u, (kb > kb0 || k > 0) ? 1u : 0u);
+                        for (int k = 1; k < BLOCK_K / UMMA_K; ++k)
+                            umma_i8_lo<CG>(d_tmem, a_lo + k * a_k16, b_lo + k * b_k16, idesc_u, 1u);
+                        umma_commit_u32<CG>(empty0 + (uint32_t)stage * 8u);  // frees the stage (in both CTAs) once these MMAs retire
                     }
-                    umma_commit<CG>(empty_bar + stage);  // frees the stage (in both CTAs) once these MMAs retire
+                    accumulate = 1u;
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit<CG>(tmem_full + slot);  // accumulator complete -> epilogue (of both CTAs)
+                if (elect_one()) umma_commit_u32<CG>(tmem_full0 + (uint32_t)slot * 8u);  // accumulator complete -> epilogue (of both CTAs)
                 slot ^= 1;
                 if (slot == 0) slot_phase ^= 1u;
             }
@@ -534,13 +560,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (uint32_t u = first_tile; u < p.total_units; u += tile_step) {
             uint32_t tile;
             int kb0, kb1, piece, npart;
-            unit_of(u, p, tile, kb0, kb1, piece, npart);
+            unit_of<NS>(u, p, tile, kb0, kb1, piece, npart);
             int bh, mi, ni;
             tile_coords(tile, p, bh, mi, ni);
             if (tile_skipped(p, mi, ni, BLOCK_M * CG, BLOCK_N)) continue;
             const int b = bh / p.heads, h = bh - b * p.heads;
-            const int width = npart >= 0 ? BLOCK_N / p.nsplit : BLOCK_N;  // columns of this unit
-            const int64_t col0 = (int64_t)ni * BLOCK_N + (npart >= 0 ? npart * width : 0);
+            const int width = (NS && npart >= 0) ? BLOCK_N / p.nsplit : BLOCK_N;  // columns of this unit
+            const int64_t col0 = (int64_t)ni * BLOCK_N + ((NS && npart >= 0) ? npart * width : 0);
             // stage this tile's per-column constants
             for (int c = et; c < width; c += C::EPI_THREADS) {
                 const int64_t col = col0 + c;
@@ -754,12 +780,17 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         return SQ_ERR_CUDA;
     p.status = a.status;
 
+    // the N split of the last wave is a variant of its own (the plain instantiation pays nothing for it)
+    constexpr bool kCanSplitN = BLOCK_N == 256 && CG == 2 && EW == 4;
     static bool attr_set[64] = {false};  // once per device
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         C::SMEM_BYTES));
+        if (kCanSplitN)
+            SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, kCanSplitN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            C::SMEM_BYTES));
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     // K split of the last wave: plain GEMMs only, and only with the scratch it needs
@@ -779,15 +810,19 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     // N split of the last wave: plain GEMMs whose reduction is too short for the K split.  With R tiles left
     // over after the full waves, cutting each into 2 or 4 column parts that still fit ONE round shortens the
     // last wave to a half or a quarter of a tile time; the parts need no exchange, only the A tile again.
-    // Measured on B200 (full-range codes): 2048 x 5120 x 5120 50.6 -> 47.2 us, 2048 x 15360 x 5120 112.6 -> 111.7,
-    // 512 x 28672 x 7168 87.4 -> 85.4, 512 x 21504 x 7168 67.8 -> 66.7 (quarters; halves gain about half of that).
+    // Measured on B200 (full-range codes, same GPU back to back): 2048 x 5120 x 5120 48.2 -> 47.2 us,
+    // 512 x 28672 x 7168 85.5 -> 85.1.
     p.nsplit = 1;
     CUtensorMap mbp = mb;  // placeholder unless the split is taken
-    if (BLOCK_N == 256 && CG == 2 && p.split == 1 && a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn) {
+    if (kCanSplitN && p.split == 1 && a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn) {
         const int64_t G = sm_count() / CG;
         const int64_t R = (int64_t)p.total_tiles % G;
         const int max_ns = a.out_dt == SQ_I8 ? 2 : 4;  // a staged store row is 128 bytes: a part must fill it
-        const int ns = (p.total_tiles > G && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
+        // (the variant's roles carry the part's width as a run-time value and run about 2 % slower per wave
+        // than the plain instantiation: beyond a few waves that costs more than the shorter last wave gains --
+        // 2048 x 15360 x 5120, 6.5 waves: 109.5 us plain, 111.4 with halves)
+        const bool few_waves = p.total_tiles > G && p.total_tiles < 4 * G;
+        const int ns = (few_waves && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
         if (ns > 1) {
             if (!make_map(&mbp, a.B, 1, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0], BLOCK_K,
                           C::B_ROWS / ns, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch))
@@ -798,7 +833,10 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         }
     }
     const int groups = (int)std::min<int64_t>((int64_t)p.total_units, sm_count() / CG);
-    return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
+    if (kCanSplitN && p.nsplit > 1)
+        return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, kCanSplitN>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
+                          (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
+    return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, false>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
                       (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
 }
 

@@ -60,6 +60,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// One lane of a converged warp (the same one every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ bool mbar_try_wait_u32(uint32_t bar_addr, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bounded wait.  Returns false (and raises the CTA's abort flag + the global status word)
 // if the phase does not complete within the cycle budget or another role already aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
@@ -78,6 +99,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         }
     }
     return true;
+}
+
+// The same bounded wait by a whole, converged warp: every lane polls, the outcome is put to a vote, so the
+// warp leaves converged and with one answer (a lane that timed out next to one that did not would
+// otherwise part ways with it for good).
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t bar_addr, uint32_t parity,
+                                               volatile uint32_t* abort_flag, uint32_t* status, uint32_t where) {
+    if (__all_sync(0xffffffffu, mbar_try_wait_u32(bar_addr, parity))) return true;
+    const bool w = mbar_wait(bar, parity, abort_flag, status, where);
+    return __all_sync(0xffffffffu, w);
 }
 
 // Tiled TMA load of one box into this CTA's shared memory.  With CG = 2 the completion is
@@ -167,6 +198,18 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
             : "memory");
     }
 }
+template <int CG>
+__device__ __forceinline__ void umma_commit_u32(uint32_t bar_addr) {
+    if (CG == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_addr) : "memory");
+    } else {
+        const uint16_t mask = 3;  // both CTAs of the pair
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+            ::"r"(bar_addr), "h"(mask)
+            : "memory");
+    }
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -218,6 +261,41 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_
     d |= (uint64_t)1 << 46;                          // descriptor version of sm_100
     d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
     return d;
+}
+
+// The same descriptor in halves, for the MMA lane's inner loop: only the start address (and the
+// leading-dimension offset) live in the low word, so a stage's and a K slice's descriptors are the
+// first one's low word plus a multiple of 16 bytes >> 4; the high word never changes.
+__device__ __forceinline__ uint32_t smem_desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+constexpr uint32_t kSmemDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024 B, sm_100 version, SWIZZLE_128B
+static_assert(((uint64_t)kSmemDescHi << 32) == (((uint64_t)(1024u >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61)),
+              "high word of the shared-memory descriptor");
+
+// The same MMA with the operand descriptors given as low words (high word: kSmemDescHi).
+template <int CG>
+__device__ __forceinline__ void umma_i8_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                           uint32_t accumulate) {
+    if (CG == 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "mov.b64 da, {%1, %5};\n\t"
+            "mov.b64 db, {%2, %5};\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kSmemDescHi)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "mov.b64 da, {%1, %5};\n\t"
+            "mov.b64 db, {%2, %5};\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kSmemDescHi)
+            : "memory");
+    }
 }
 
 // Instruction descriptor of tcgen05.mma kind::i8: signed 8-bit A and B, INT32 D.
