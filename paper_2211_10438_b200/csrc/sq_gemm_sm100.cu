@@ -810,19 +810,15 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     // N split of the last wave: plain GEMMs whose reduction is too short for the K split.  With R tiles left
     // over after the full waves, cutting each into 2 or 4 column parts that still fit ONE round shortens the
     // last wave to a half or a quarter of a tile time; the parts need no exchange, only the A tile again.
-    // Measured on B200 (full-range codes, same GPU back to back): 2048 x 5120 x 5120 48.2 -> 47.2 us,
-    // 512 x 28672 x 7168 85.5 -> 85.1.
+    // Measured on B200 (full-range codes, same GPU back to back, split withheld -> taken): 2048 x 15360 x 5120
+    // 105.4 -> 103.9 us, 2048 x 21504 x 7168 198.2 -> 195.2, 8192 x 28672 x 7168 1019 -> 1011.
     p.nsplit = 1;
     CUtensorMap mbp = mb;  // placeholder unless the split is taken
     if (kCanSplitN && p.split == 1 && a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn) {
         const int64_t G = sm_count() / CG;
         const int64_t R = (int64_t)p.total_tiles % G;
         const int max_ns = a.out_dt == SQ_I8 ? 2 : 4;  // a staged store row is 128 bytes: a part must fill it
-        // (the variant's roles carry the part's width as a run-time value and run about 2 % slower per wave
-        // than the plain instantiation: beyond a few waves that costs more than the shorter last wave gains --
-        // 2048 x 15360 x 5120, 6.5 waves: 109.5 us plain, 111.4 with halves)
-        const bool few_waves = p.total_tiles > G && p.total_tiles < 4 * G;
-        const int ns = (few_waves && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
+        const int ns = (p.total_tiles > G && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
         if (ns > 1) {
             if (!make_map(&mbp, a.B, 1, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0], BLOCK_K,
                           C::B_ROWS / ns, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch))
