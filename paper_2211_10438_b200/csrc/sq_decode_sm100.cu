@@ -460,8 +460,15 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
         }
     } else if (warp == 1) {
         // ============================ MMA issuer ==============================
-        if (lane == 0) {
+        // The whole warp walks the tiles and waits on the barriers, converged; one elected lane issues the
+        // MMAs and the commits (their operands are then warp-uniform values to the compiler).
+        {
             const uint32_t idesc = make_idesc(BLOCK_M, DEC_N, 0);
+            constexpr uint32_t kStage16 = (uint32_t)DEC_STAGE >> 4;
+            const uint32_t w_lo0 = smem_desc_lo(smem_u32(smem), 16);
+            const uint32_t x_lo0 = smem_desc_lo(smem_u32(smem) + (uint32_t)W_BYTES, 16);
+            const uint32_t full0 = smem_u32(full_bar), empty0 = smem_u32(empty_bar);
+            const uint32_t tmem_full0 = smem_u32(tmem_full), tmem_empty0 = smem_u32(tmem_empty);
             int stage = 0;
             uint32_t phase = 0;
             int slot = 0;
@@ -470,27 +477,36 @@ decode_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_cons
             DecWalk walk(p);
             int ni, kb0, kb1;
             while (ok && walk.next(p, ni, kb0, kb1)) {
-                if (!(ok = mbar_wait(tmem_empty + slot, slot_phase ^ 1u, abort_flag, p.status, 7))) break;
+                if (!(ok = mbar_wait_warp(tmem_empty + slot, tmem_empty0 + (uint32_t)slot * 8u, slot_phase ^ 1u, abort_flag,
+                                          p.status, 7)))
+                    break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * DEC_N);
+                uint32_t accumulate = 0u;  // the tile's first MMA overwrites the slot
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag, p.status, 8))) break;
+                    if (!(ok = mbar_wait_warp(full_bar + stage, full0 + (uint32_t)stage * 8u, phase, abort_flag, p.status, 8)))
+                        break;
 #ifdef SQ_DEC_TRACE
-                    if (g_dec_trace[p.trace_id][blockIdx.x][5] == 0ull) DEC_TRACE(5);
+                    if (lane == 0 && g_dec_trace[p.trace_id][blockIdx.x][5] == 0ull) DEC_TRACE(5);
 #endif
                     tcgen05_fence_after();
-                    const uint32_t sw = smem_u32(smem + stage * DEC_STAGE);
-                    const uint32_t sx = sw + W_BYTES;
+                    const uint32_t w_lo = w_lo0 + (uint32_t)stage * kStage16;
+                    const uint32_t x_lo = x_lo0 + (uint32_t)stage * kStage16;
+                    if (elect_one()) {
+                        umma_i8_lo<1>(d_tmem, w_lo, x_lo, idesc, accumulate);
 #pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_i8<1>(d_tmem, make_smem_desc(sw + k * UMMA_K, 16), make_smem_desc(sx + k * UMMA_K, 16),
-                                   idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-                    umma_commit<1>(empty_bar + stage);
+                        for (int k = 1; k < BLOCK_K / UMMA_K; ++k)
+                            umma_i8_lo<1>(d_tmem, w_lo + k * (UMMA_K >> 4), x_lo + k * (UMMA_K >> 4), idesc, 1u);
+                        umma_commit_u32<1>(empty0 + (uint32_t)stage * 8u);
+                    }
+                    accumulate = 1u;
                     if (++stage == DEC_STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit<1>(tmem_full + slot);
-                DEC_TRACE(6);
+                if (elect_one()) umma_commit_u32<1>(tmem_full0 + (uint32_t)slot * 8u);
+#ifdef SQ_DEC_TRACE
+                if (lane == 0) DEC_TRACE(6);
+#endif
                 slot ^= 1;
                 if (slot == 0) slot_phase ^= 1u;
             }
