@@ -158,23 +158,31 @@ __device__ __forceinline__ int tile_num_kb(const Params& p, int mi, int tile_m) 
 // ------------------------------------------------------------------------------------
 // FIX: this CTA arrived last for a K-split tile: the other pieces' partial sums (fix_count slots,
 // fix_stride ints apart, fix_base already at this thread's row) are added to the accumulators first.
-template <int BLOCK_N, bool FIX = false, bool EW8 = false>
+template <int BLOCK_N, bool FIX = false, bool EW8 = false, bool PLAIN16 = false>
 __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
                                               uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
                                               int h, int64_t c_off, const float* s_wscale,
                                               const float* s_bias, const float* s_requant, int lane,
                                               int cc_begin, int cc_end, const int32_t* fix_base = nullptr,
                                               int fix_count = 0, int fix_mine = 0, size_t fix_stride = 0) {
+    // PLAIN16: the instantiation for the plain linear layer -- 16-bit output through staged TMA stores, vector
+    // scales / bias, no residual, no row maxima.  The generic body carries every output type and option in one
+    // unrolled loop; its code size alone (instruction fetch, 255 registers) made a slot take 11 000 cycles
+    // where this one takes under 7 000.
+    const int out_dt = PLAIN16 ? (p.out_dt == SQ_F16 ? (int)SQ_F16 : (int)SQ_BF16) : p.out_dt;
+    const bool c_tma = PLAIN16 || p.c_tma;
+    const void* const residual = PLAIN16 ? nullptr : p.residual;
+    float* const row_absmax_out = PLAIN16 ? nullptr : p.row_absmax_out;
     const bool row_ok = row < p.M;
     float xs = p.alpha;
     if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
     float row_max = 0.0f;
     // 32-column chunks per 128-byte staging row: 1 (int32), 2 (fp16/bf16), 4 (int8)
-    const int chunks_per_store = p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2);
+    const int chunks_per_store = out_dt == SQ_I32 ? 1 : (out_dt == SQ_I8 ? 4 : 2);
     const int pieces = 8 / chunks_per_store;  // 16-byte pieces one chunk contributes to the row
     int cc_coord[4] = {0, 0, 0, 0};
     cc_coord[p.c_slot_row] = row0_warp; cc_coord[p.c_slot_head] = h; cc_coord[p.c_slot_batch] = b;
-    const bool scalar_scale = p.w_scale == nullptr && p.bias == nullptr;  // attention BMMs: y = acc * alpha
+    const bool scalar_scale = !PLAIN16 && p.w_scale == nullptr && p.bias == nullptr;  // attention BMMs: y = acc * alpha
 #pragma unroll 1
     for (int cc = cc_begin; cc < cc_end; ++cc) {
         uint32_t r[32];
@@ -199,7 +207,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
         // ---- Eq. 2 on the chunk; w[] receives the packed output words ----
         uint32_t w[32];
         int nwords;
-        if (p.out_dt == SQ_I32) {
+        if (out_dt == SQ_I32) {
 #pragma unroll
             for (int j = 0; j < 32; ++j) w[j] = r[j];
             nwords = 32;
@@ -221,22 +229,22 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                     y[j] = v;
                 }
             }
-            if (p.row_absmax_out) {
+            if (row_absmax_out) {
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
                     if (j < ncols) row_max = fmaxf(row_max, fabsf(y[j]));
             }
-            if (p.residual && !p.c_tma) {
+            if (residual && !c_tma) {
                 // the block's residual connection: round y to the output type first, then add the
                 // residual element in fp32 (the final rounding below is the 16-bit add's rounding)
                 const uint4* rrow = reinterpret_cast<const uint4*>(
-                    static_cast<const uint16_t*>(p.residual) + (row_ok ? row : 0) * p.ld_res + col0 + cc * 32);
+                    static_cast<const uint16_t*>(residual) + (row_ok ? row : 0) * p.ld_res + col0 + cc * 32);
 #pragma unroll
                 for (int v = 0; v < 4; ++v) {
                     if (row_ok && 8 * v < ncols) {  // N is a multiple of 8: whole vectors only
                         const uint4 rv = __ldg(rrow + v);
                         float rf[8];
-                        if (p.out_dt == SQ_BF16) {
+                        if (out_dt == SQ_BF16) {
                             unpack8<__nv_bfloat16>(rv, rf);
 #pragma unroll
                             for (int k = 0; k < 8; ++k)
@@ -250,7 +258,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                     }
                 }
             }
-            if (p.out_dt == SQ_I8) {
+            if (out_dt == SQ_I8) {
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
                     w[v] = pack4(quant_code(y[4 * v], s_requant[cc * 32 + 4 * v]),
@@ -258,7 +266,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                                  quant_code(y[4 * v + 2], s_requant[cc * 32 + 4 * v + 2]),
                                  quant_code(y[4 * v + 3], s_requant[cc * 32 + 4 * v + 3]));
                 nwords = 8;
-            } else if (p.out_dt == SQ_BF16) {
+            } else if (out_dt == SQ_BF16) {
 #pragma unroll
                 for (int v = 0; v < 16; ++v) {
                     __nv_bfloat162 t = __halves2bfloat162(__float2bfloat16_rn(y[2 * v]), __float2bfloat16_rn(y[2 * v + 1]));
@@ -274,7 +282,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                 nwords = 16;
             }
         }
-        if (p.c_tma) {
+        if (c_tma) {
             // ---- staged TMA store: lane = row of the 32 x 128-byte staging tile ----
             const int sub = cc % chunks_per_store;
             uint8_t* buf = stg;
@@ -293,7 +301,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
             }
             if (sub == chunks_per_store - 1) {
                 const int64_t gcol = col0 + (int64_t)(cc - sub) * 32;  // first column of the staged group
-                if (p.residual) {
+                if (residual) {
                     // The residual connection, on the staged tile (32 rows x 64 rounded outputs): the
                     // warp walks it in the layout of the global rows -- 8 lanes per row, 16 bytes per
                     // lane -- so that the residual arrives in whole 128-byte lines, adds in fp32 and
@@ -309,7 +317,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                     for (int i = 0; i < RB; ++i) {
                         const int64_t rr = (int64_t)row0_warp + 4 * (i0 + i) + (lane >> 3);
                         rv[i] = (rr < p.M && rcol < p.N)  // N is a multiple of 8: whole vectors only
-                                    ? __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(p.residual) +
+                                    ? __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(residual) +
                                                                            rr * p.ld_res + rcol))
                                     : make_uint4(0u, 0u, 0u, 0u);
                     }
@@ -319,7 +327,7 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
                         uint4* cell = reinterpret_cast<uint4*>(buf + r * 128 + ((piece_c ^ (r & 7)) << 4));
                         float a[8], b[8];
                         uint4 o;
-                        if (p.out_dt == SQ_BF16) {
+                        if (out_dt == SQ_BF16) {
                             unpack8<__nv_bfloat16>(*cell, a);
                             unpack8<__nv_bfloat16>(rv[i], b);
                             __nv_bfloat162 t0 = __halves2bfloat162(__float2bfloat16_rn(a[0] + b[0]), __float2bfloat16_rn(a[1] + b[1]));
@@ -356,12 +364,12 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
         // ---- direct stores (unaligned C) ----
         if (!row_ok || ncols <= 0) continue;
         const bool full = ncols >= 32;
-        if (p.out_dt == SQ_I32) {
+        if (out_dt == SQ_I32) {
             int32_t* out = static_cast<int32_t*>(p.C) + c_off + cc * 32;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
                 if (full || j < ncols) out[j] = (int32_t)w[j];
-        } else if (p.out_dt == SQ_I8) {
+        } else if (out_dt == SQ_I8) {
             int8_t* out = static_cast<int8_t*>(p.C) + c_off + cc * 32;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
@@ -374,13 +382,13 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
         }
         (void)nwords;
     }
-    if (p.row_absmax_out && row_ok) atomic_max_nonneg(p.row_absmax_out + row, row_max);
+    if (row_absmax_out && row_ok) atomic_max_nonneg(row_absmax_out + row, row_max);
 }
 
 // ------------------------------------------------------------------------------------
 // The kernel
 // ------------------------------------------------------------------------------------
-template <int BLOCK_N, int CG, int EW, bool NS = false>
+template <int BLOCK_N, int CG, int EW, bool NS = false, bool PLAIN16 = false>
 __global__ void __launch_bounds__(EW * 32 + 64, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_bp, const Params p) {
@@ -581,7 +589,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
                 s_wscale[c] = ws; s_bias[c] = bs; s_requant[c] = rq;
             }
-            if (p.residual) {
+            if (!PLAIN16 && p.residual) {
                 // pull this thread's row of the residual tile into L2 while the tile's MMAs still run:
                 // under a saturated memory system a demand load in the epilogue waits microseconds
                 const int64_t prow = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
@@ -605,13 +613,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int row0_warp = (mi * CG + rank) * BLOCK_M + quarter * 32;
             // split the tile's 32-column chunks between the two warps of this lane quarter, in whole
             // store groups (a staged TMA store covers 128 bytes of a row = 1, 2 or 4 chunks)
-            const int cps = p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2);
+            const int cps = PLAIN16 ? 2 : (p.out_dt == SQ_I32 ? 1 : (p.out_dt == SQ_I8 ? 4 : 2));
             const int groups = (width / 32 + cps - 1) / cps;
             const int g_split = EW == 8 ? (groups + 1) / 2 : groups;
             const int cc_begin = half == 0 ? 0 : g_split * cps;
             const int cc_end = half == 0 ? min(g_split * cps, width / 32) : width / 32;
             if (EW == 8 || piece < 0) {  // (the eight-warp configuration serves short reductions: never split)
-                epilogue_slot<BLOCK_N, false, EW == 8>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
+                epilogue_slot<BLOCK_N, false, EW == 8, PLAIN16>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
                                        c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
             } else {
                 // K piece of a split tile: park the accumulators, then see who is last
@@ -637,7 +645,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 epi_bar_sync<C::EPI_THREADS>();
                 if (*epi_last != 0u) {
                     __threadfence();
-                    epilogue_slot<BLOCK_N, true>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b,
+                    epilogue_slot<BLOCK_N, true, false, PLAIN16>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b,
                                                  h, c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end,
                                                  tile_slots, p.split, piece, (size_t)CG * kTileInts);
                     if (et == 0) p.counters[rem * CG + rank] = 0u;  // hand the counter back zeroed
@@ -780,17 +788,27 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         return SQ_ERR_CUDA;
     p.status = a.status;
 
-    // the N split of the last wave is a variant of its own (the plain instantiation pays nothing for it)
-    constexpr bool kCanSplitN = BLOCK_N == 256 && CG == 2 && EW == 4;
+    // Variants of the main configuration, each an instantiation of its own so that the others pay nothing for
+    // it: the N split of the last wave, and the plain linear layer's epilogue (16-bit output through staged
+    // TMA stores, vector scales or bias, no residual, no row maxima).
+    constexpr bool kMain = BLOCK_N == 256 && CG == 2 && EW == 4;
+    constexpr bool kCanSplitN = kMain;
+    const bool plain16 = kMain && (a.out_dt == SQ_F16 || a.out_dt == SQ_BF16) && p.c_tma && a.residual == nullptr &&
+                         a.row_absmax_out == nullptr && (a.w_scale != nullptr || a.bias != nullptr);
     static bool attr_set[64] = {false};  // once per device
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         C::SMEM_BYTES));
-        if (kCanSplitN)
-            SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, kCanSplitN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            C::SMEM_BYTES));
+        if (kMain) {
+            SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, kMain, false>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+            SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, false, kMain>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+            SQ_CUDA_OK(cudaFuncSetAttribute(gemm_i8_kernel<BLOCK_N, CG, EW, kMain, kMain>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        }
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     // K split of the last wave: plain GEMMs only, and only with the scratch it needs
@@ -829,11 +847,14 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         }
     }
     const int groups = (int)std::min<int64_t>((int64_t)p.total_units, sm_count() / CG);
-    if (kCanSplitN && p.nsplit > 1)
-        return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, kCanSplitN>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
-                          (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
-    return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, false>, dim3((unsigned)(groups * CG)), dim3(C::NUM_THREADS),
-                      (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
+    const dim3 grid((unsigned)(groups * CG)), block(C::NUM_THREADS);
+    if (kMain && p.nsplit > 1 && plain16)
+        return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, kMain, kMain>, grid, block, (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
+    if (kMain && p.nsplit > 1)
+        return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, kMain, false>, grid, block, (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
+    if (kMain && plain16)
+        return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, false, kMain>, grid, block, (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
+    return launch_pdl(gemm_i8_kernel<BLOCK_N, CG, EW, false, false>, grid, block, (size_t)C::SMEM_BYTES, st, CG, ma, mb, mc, mbp, p);
 }
 
 // Short reductions (few K slices per tile) are bound by draining the accumulators: give them
