@@ -30,10 +30,10 @@ def _stale(target, deps):
 
 
 def build_trace() -> str:
-    """Tuning build: libsq_trace.so, the same library with the decode-shaped GEMM's timestamp trace
-    compiled in (-DSQ_DEC_TRACE).  Never loaded by the binding unless LIB_PATH is pointed at it."""
+    """Tuning build: libsq_trace.so, the same library with the timestamp traces of the decode-shaped GEMM
+    (-DSQ_DEC_TRACE) and of the prefill GEMM's MMA warp (-DSQ_GEMM_TRACE) compiled in.  Never loaded by the binding unless LIB_PATH is pointed at it."""
     out = os.path.join(HERE, "libsq_trace.so")
-    subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSQ_DEC_TRACE", "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out],
+    subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSQ_DEC_TRACE", "-DSQ_GEMM_TRACE", "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out],
                    check=True)
     return out
 

@@ -49,6 +49,21 @@ struct Cfg {
     static_assert(B_ROWS % 8 == 0, "B tile must be whole 8-row swizzle groups");
 };
 
+// Tuning build only (python -m paper_2211_10438_b200.build --trace: -DSQ_GEMM_TRACE): the MMA warp of every
+// even CTA records, in SM cycles, what it spends per tile -- index arithmetic before the tile, the wait for
+// the accumulator slot, the loop over the K blocks -- and, once, cycles and nanoseconds from its first MMA to
+// its last commit (their ratio is the SM clock the launch actually ran at); epilogue warp 0 records how long
+// it takes to drain the fourth tile's slot.  sq_debug_gemm_trace() copies the table of the last launch out.
+#ifdef SQ_GEMM_TRACE
+constexpr int kGemmTraceTiles = 16;
+__device__ unsigned long long g_gemm_trace[160][kGemmTraceTiles + 1][4];
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#endif
+
 struct Params {
     int64_t M, N, K;
     int heads, batch;
@@ -511,6 +526,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int slot = 0;
             uint32_t slot_phase = 0;
             bool ok = true;
+#ifdef SQ_GEMM_TRACE
+            int trace_tile = 0;
+            long long trace_prev_end = clock64(), trace_first = 0;
+            unsigned long long trace_first_ns = 0;
+#endif
             for (uint32_t u = first_tile; ok && u < p.total_units; u += tile_step) {
                 uint32_t tile;
                 int kb0, kb1, piece, npart;
@@ -527,12 +547,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     kb1 = p.num_kb;
                 }
                 const uint32_t idesc_u = (NS && npart >= 0) ? make_idesc(BLOCK_M * CG, BLOCK_N / p.nsplit, p.b_is_kn) : idesc;
+#ifdef SQ_GEMM_TRACE
+                const long long trace_decoded = clock64();
+#endif
                 if (!(ok = mbar_wait_warp(tmem_empty + slot, tmem_empty0 + (uint32_t)slot * 8u, slot_phase ^ 1u, abort_flag,
                                           p.status, 2)))
                     break;
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(slot * C::SLOT_COLS);
                 uint32_t accumulate = 0u;  // the tile's first MMA overwrites the slot
+#ifdef SQ_GEMM_TRACE
+                const long long trace_start = clock64();
+                if (trace_tile == 0) { trace_first = trace_start; trace_first_ns = global_timer_ns(); }
+#endif
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!(ok = mbar_wait_warp(full_bar + stage, full0 + (uint32_t)stage * 8u, phase, abort_flag, p.status, 3)))
                         break;
@@ -551,6 +578,25 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
                 if (!ok) break;
                 if (elect_one()) umma_commit_u32<CG>(tmem_full0 + (uint32_t)slot * 8u);  // accumulator complete -> epilogue (of both CTAs)
+#ifdef SQ_GEMM_TRACE
+                {
+                    const long long trace_end = clock64();
+                    if (lane == 0) {
+                        if (trace_tile < kGemmTraceTiles) {
+                            unsigned long long* tr = g_gemm_trace[blockIdx.x][trace_tile];
+                            tr[0] = (unsigned long long)(trace_decoded - trace_prev_end);
+                            tr[1] = (unsigned long long)(trace_start - trace_decoded);
+                            tr[2] = (unsigned long long)(trace_end - trace_start);
+                            tr[3] = (unsigned long long)(kb1 - kb0);
+                        }
+                        unsigned long long* tr = g_gemm_trace[blockIdx.x][kGemmTraceTiles];
+                        tr[0] = (unsigned long long)(trace_end - trace_first);
+                        tr[1] = global_timer_ns() - trace_first_ns;
+                    }
+                    ++trace_tile;
+                    trace_prev_end = trace_end;
+                }
+#endif
                 slot ^= 1;
                 if (slot == 0) slot_phase ^= 1u;
             }
@@ -565,6 +611,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int quarter = warp & 3, half = warp >> 2;
         int slot = 0;
         uint32_t slot_phase = 0;
+#ifdef SQ_GEMM_TRACE
+        int trace_tile = 0;
+        long long trace_go = 0;
+#endif
         for (uint32_t u = first_tile; u < p.total_units; u += tile_step) {
             uint32_t tile;
             int kb0, kb1, piece, npart;
@@ -605,6 +655,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             epi_bar_sync<C::EPI_THREADS>();  // constants staged; outcome of the wait visible to all epilogue threads
             if (*epi_go == 0u) break;
             tcgen05_fence_after();
+#ifdef SQ_GEMM_TRACE
+            trace_go = clock64();
+#endif
 
             const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
             const int64_t c_off = (int64_t)b * p.c_stride_batch + (int64_t)h * p.c_stride_head +
@@ -652,6 +705,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 }
             }
 
+#ifdef SQ_GEMM_TRACE
+            if (threadIdx.x == 0 && trace_tile == 3) g_gemm_trace[blockIdx.x][kGemmTraceTiles][2] = (unsigned long long)(clock64() - trace_go);
+            ++trace_tile;
+#endif
             // accumulator slot drained: hand it back to the MMA warp (in the even CTA)
             tcgen05_fence_before();
             if (CG == 1) mbar_arrive(tmem_empty + slot); else mbar_arrive_even_cta(tmem_empty + slot);
@@ -922,3 +979,16 @@ sq_status gemm_i8(const GemmArgs& a, cudaStream_t st) {
 }
 
 }  // namespace sq
+
+#ifdef SQ_GEMM_TRACE
+// [160 CTAs][16 tiles + 1][4] 64-bit words: per tile (index arithmetic, wait for the accumulator slot, K loop:
+// SM cycles; K blocks); last row: cycles and nanoseconds from the CTA's first MMA to its last commit, cycles
+// epilogue warp 0 took to drain the fourth tile's slot, 0.  Copies the table out and clears it.
+extern "C" int sq_debug_gemm_trace(unsigned long long* host_out) {
+    const size_t bytes = sizeof(unsigned long long) * 160 * (sq::kGemmTraceTiles + 1) * 4;
+    if (cudaMemcpyFromSymbol(host_out, sq::g_gemm_trace, bytes) != cudaSuccess) return 1;
+    void* dev = nullptr;
+    if (cudaGetSymbolAddress(&dev, sq::g_gemm_trace) != cudaSuccess || cudaMemset(dev, 0, bytes) != cudaSuccess) return 1;
+    return 0;
+}
+#endif

@@ -69,8 +69,36 @@ def gemm(args):
         print(line)
         if sq.device_status(ws) != 0:
             raise SystemExit("device status word = %d" % sq.device_status(ws))
+        if args.trace:
+            _print_gemm_trace()
         del X, Wq, Y
     return sq.new_workspace(256)
+
+
+def _print_gemm_trace():
+    """The MMA warps' cycle counts of the last launch (needs --lib .../libsq_trace.so)."""
+    import ctypes
+
+    import numpy as np
+    tiles = 16
+    buf = (ctypes.c_ulonglong * (160 * (tiles + 1) * 4))()
+    fn = getattr(sq.lib(), "sq_debug_gemm_trace", None)
+    if fn is None:
+        raise SystemExit("--trace needs the trace build: python -m paper_2211_10438_b200.build --trace, then --lib .../libsq_trace.so")
+    if fn(buf) != 0:
+        raise SystemExit("sq_debug_gemm_trace failed")
+    t = np.frombuffer(buf, dtype=np.uint64).reshape(160, tiles + 1, 4).astype(np.float64)
+    t = t[t[:, tiles, 1] > 0]                       # CTAs whose MMA warp ran (the even CTA of every pair)
+    n_tiles = (t[:, :tiles, 3] > 0).sum(axis=1)
+    later = np.concatenate([t[i, 1:int(n_tiles[i]), :] for i in range(len(t)) if n_tiles[i] > 1] or [np.zeros((0, 4))])
+    span_cyc, span_ns, epi = t[:, tiles, 0], t[:, tiles, 1], t[:, tiles, 2]
+    print("  MMA warp, %d CTA pairs, %d-%d tiles each; per tile after the first (mean, SM cycles): index arithmetic %.0f, "
+          "wait for the accumulator slot %.0f, K loop %.0f = %.1f per K block of 4 MMAs (128 cycles each at full rate)"
+          % (len(t), n_tiles.min(), n_tiles.max(), later[:, 0].mean(), later[:, 1].mean(), later[:, 2].mean(),
+             (later[:, 2] / later[:, 3]).mean()))
+    print("  first MMA -> last commit: median %.1f us, %.0f cycles: SM clock during the launch %.0f MHz; "
+          "epilogue warp 0 drains the fourth tile's slot in %.0f cycles"
+          % (np.median(span_ns) / 1e3, np.median(span_cyc), np.median(span_cyc / span_ns * 1e3), np.median(epi[epi > 0]) if (epi > 0).any() else 0))
 
 
 def decode_gemm(args):
@@ -201,6 +229,7 @@ def main(argv=None):
     ap.add_argument("--values", choices=["full", "tri", "ones", "zeros"], default="full", help="gemm: operand value class")
     ap.add_argument("--no-split", action="store_true", help="gemm: no scratch for the K split of the last wave")
     ap.add_argument("--int-mm", action="store_true", help="gemm: also time torch._int_mm (cuBLASLt) for context")
+    ap.add_argument("--trace", action="store_true", help="gemm: print the MMA warps' cycle counts (trace build given with --lib)")
     ap.add_argument("--fused", action="store_true", help="decode_gemm / generation_block: quantiser inside the GEMM")
     ap.add_argument("--B", type=int, default=None, help="batch (attention: 4, kv_attention: 16)")
     ap.add_argument("--H", type=int, default=None, help="heads (attention: 56, kv_attention: 96)")
