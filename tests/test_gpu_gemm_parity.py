@@ -150,6 +150,50 @@ def test_gemm_last_wave_k_split_is_exact(M, N, K):
     assert not big[4:33024].any(), "header and counters not handed back zero-filled"
 
 
+# Reductions too short for the K split whose tile count leaves a partly filled last wave: the tiles of that wave
+# are cut into 2 or 4 COLUMN parts (74 CTA pairs; 256 x 256 tiles).  100 tiles -> 26 left over -> halves;
+# 80 tiles -> 6 left over -> quarters (halves for INT8 output), here with ragged M and an N tail that leaves
+# the last tile's third quarter with 8 columns and its fourth with none.  Every epilogue, element by element.
+N_SPLIT_SHAPES = [(1200, 5120, 1152), (1000, 5000, 1152)]
+
+
+@pytest.mark.parametrize("epilogue", ["i32", "bf16", "f16_relu", "i8_requant_absmax", "bf16_residual"])
+@pytest.mark.parametrize("M,N,K", N_SPLIT_SHAPES)
+def test_gemm_last_wave_n_split_every_epilogue(ws, M, N, K, epilogue):
+    Xq, Wq = synth.int8_tensor(31, 1, (M, K)), synth.int8_tensor(31, 2, (N, K))
+    rng = synth.rng_for(31, 3)
+    xs = rng.uniform(0.01, 0.2, M).astype(np.float32)
+    wsc = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    acc = oracle.gemm_i32(Xq, Wq)
+    Xd, Wd = dev(Xq), dev(Wq)
+    if epilogue == "i32":
+        got = sq.sq_w8a8_gemm(Xd, Wd, None, None, ws, out_dtype=torch.int32)
+        assert np.array_equal(host(got), acc)
+    elif epilogue in ("bf16", "f16_relu"):
+        dtype, relu = ("bf16", False) if epilogue == "bf16" else ("f16", True)
+        bias = synth.bias(31, 4, N, dtype, std=0.5)
+        got = sq.sq_w8a8_gemm(Xd, Wd, dev(xs), dev(wsc), ws, bias=dev(bias, dtype), relu=relu,
+                              out_dtype=torch.bfloat16 if dtype == "bf16" else torch.float16)
+        assert np.array_equal(host(got), oracle.round_to(oracle.dequant(acc, xs, wsc, bias, relu=relu), dtype))
+    elif epilogue == "i8_requant_absmax":
+        bias = synth.bias(31, 4, N, "f16", std=0.5)
+        r = rng.uniform(0.5, 2.0, N).astype(np.float32)
+        rmax = torch.zeros(M, dtype=torch.float32, device="cuda")
+        got = sq.sq_w8a8_gemm(Xd, Wd, dev(xs), dev(wsc), ws, bias=dev(bias, "f16"), relu=True, requant_mul=dev(r),
+                              row_absmax_out=rmax, out_dtype=torch.int8)
+        y = oracle.dequant(acc, xs, wsc, bias, relu=True)
+        assert np.array_equal(host(got), oracle.requant(y, r))
+        assert np.array_equal(host(rmax), np.abs(y).max(1))
+    else:
+        bias = synth.bias(31, 4, N, "bf16", std=0.5)
+        res = synth.to_dtype_f32(rng.standard_normal((M, N)).astype(np.float32) * 4, "bf16")
+        y = oracle.round_to(oracle.dequant(acc, xs, wsc, bias), "bf16")
+        got = sq.sq_w8a8_gemm_residual(Xd, Wd, dev(xs), dev(wsc), ws, dev(res, "bf16"), bias=dev(bias, "bf16"),
+                                       out=torch.zeros((M, N), dtype=torch.bfloat16, device="cuda"))
+        assert np.array_equal(host(got), oracle.round_to(y + res, "bf16"))
+    assert sq.device_status(ws) == 0
+
+
 # the residual connection folded into the epilogue: bit for bit the unfused pair of calls.  Shapes: one
 # CTA pair tile with ragged M, single-CTA narrow and wide tiles, the weight-streaming kernel (shared
 # tiles), a K-split last wave (fix-up path), a strided residual and output
