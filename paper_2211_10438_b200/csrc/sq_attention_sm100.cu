@@ -11,8 +11,8 @@
 //
 // One CTA per (128-query tile, head, batch), two CTAs per SM.  Warps 0-7: softmax, two threads per
 // query row (warps 0-3 own key half 0 of every tile, warps 4-7 half 1; the row is the thread's TMEM
-// lane, so row reductions are thread-local per half and merged once after pass 1); warp 8: one
-// lane issues the TMA loads and the tcgen05 MMAs.  TMEM: 2 x 64 columns of scores + 128 of output.
+// lane, so row reductions are thread-local per half and merged once after pass 1); warp 8 walks the
+// steps converged and one elected lane of it issues the TMA loads and the tcgen05 MMAs.  TMEM: 2 x 64 columns of scores + 128 of output.
 // The score MMA is issued per key half with separate full / free barriers, so the tensor core
 // refills one half while the other is being read, and the next step's first half is issued as
 // soon as the current one is drained.  The softmax is kept lean: the row maximum is taken on the
@@ -175,8 +175,10 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
     pdl_launch_dependents();
 
     if (warp == CTRL_WARP) {
-        // ===================== control lane: TMA loads and MMA issue =====================
-        if (lane == 0) {
+        // ===================== control warp: TMA loads and MMA issue =====================
+        // The whole warp walks the steps and waits on the barriers, converged; one elected lane issues the
+        // loads, the MMAs and the commits (their operands are then warp-uniform values to the compiler).
+        {
             // The score MMA is issued per HALF of the key tile (64 keys, 64 TMEM columns), each half
             // with its own full / free barriers: while the softmax warps work on one half, the
             // tensor core already fills the other, and the next step's first half is issued as
@@ -184,11 +186,19 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
             // through pass 1 (t < n_kv) and pass 2; key tile of step t is t % n_kv.
             const uint32_t idesc_s = make_idesc(TILE, HALF, 0);   // Q (K-major) x K^T (K-major), 64 keys
             const uint32_t idesc_pv = make_idesc(TILE, TILE, 1);  // P (K-major) x V ([keys, d]: N contiguous)
+            const uint32_t q_lo = smem_desc_lo(smem_u32(s_q), 16), k_lo0 = smem_desc_lo(smem_u32(s_k), 16);
+            const uint32_t p_lo = smem_desc_lo(smem_u32(s_p), 16), v_lo0 = smem_desc_lo(smem_u32(s_v), 16384u);
+            const uint32_t bars0 = smem_u32(bars);
+            auto bar_addr = [&](uint64_t* b) { return bars0 + (uint32_t)(b - bars) * 8u; };
             const int T = 2 * n_kv;
             bool ok = true;
             uint32_t kph[2] = {0, 0}, vph[2] = {0, 0}, s_free_ph[2] = {0, 0};
             uint32_t p_full_ph = 0, pv_done_ph = 0;
+            auto wait = [&](uint64_t* b, uint32_t parity, uint32_t where) {
+                return mbar_wait_warp(b, bar_addr(b), parity, abort_flag, p.status, where);
+            };
             auto load_kv = [&](int t) {  // operands of step t into stage t & 1
+                if (!elect_one()) return;
                 const int st = t & 1, j = t % n_kv;
                 mbar_expect_tx(bar_k + st, TILE_BYTES);
                 tma_load_4d<1>(s_k + st * TILE_BYTES, &tmap_qkv, bar_k + st, xk, row_base + j * TILE, 0, 0);
@@ -198,19 +208,22 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
                 }
             };
             auto issue_qk = [&](int t, int hh) {  // scores of key half hh of step t
-                const uint32_t qa = smem_u32(s_q), ka = smem_u32(s_k + (t & 1) * TILE_BYTES) + hh * (HALF * 128);
+                if (!elect_one()) return;
+                const uint32_t k_lo = k_lo0 + (uint32_t)(((t & 1) * TILE_BYTES + hh * (HALF * 128)) >> 4);
+                umma_i8_lo<1>(tmem_s + hh * HALF, q_lo, k_lo, idesc_s, 0u);
 #pragma unroll
-                for (int k = 0; k < TILE / UMMA_K; ++k)
-                    umma_i8<1>(tmem_s + hh * HALF, make_smem_desc(qa + k * UMMA_K, 16), make_smem_desc(ka + k * UMMA_K, 16),
-                               idesc_s, k > 0 ? 1u : 0u);
-                umma_commit<1>(bar_s_full + hh);
+                for (int k = 1; k < TILE / UMMA_K; ++k)
+                    umma_i8_lo<1>(tmem_s + hh * HALF, q_lo + k * (UMMA_K >> 4), k_lo + k * (UMMA_K >> 4), idesc_s, 1u);
+                umma_commit_u32<1>(bar_addr(bar_s_full + hh));
             };
-            mbar_expect_tx(bar_q, TILE_BYTES);
-            tma_load_4d<1>(s_q, &tmap_qkv, bar_q, xq, row_base + qt * TILE, 0, 0);
+            if (elect_one()) {
+                mbar_expect_tx(bar_q, TILE_BYTES);
+                tma_load_4d<1>(s_q, &tmap_qkv, bar_q, xq, row_base + qt * TILE, 0, 0);
+            }
             load_kv(0);
             load_kv(1);  // T >= 2 always
-            ok = mbar_wait(bar_q, 0, abort_flag, p.status, 20);
-            if (ok) ok = mbar_wait(bar_k, kph[0], abort_flag, p.status, 21);
+            ok = wait(bar_q, 0, 20);
+            if (ok) ok = wait(bar_k, kph[0], 21);
             kph[0] ^= 1u;
             if (ok) {
                 tcgen05_fence_after();
@@ -221,35 +234,37 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
                 const int st = t & 1;
                 const bool more = t + 1 < T;
                 if (more) {  // (a) first half of the next step, once this step's first half is drained
-                    if (!(ok = mbar_wait(bar_k + (st ^ 1), kph[st ^ 1], abort_flag, p.status, 21))) break;
+                    if (!(ok = wait(bar_k + (st ^ 1), kph[st ^ 1], 21))) break;
                     kph[st ^ 1] ^= 1u;
-                    if (!(ok = mbar_wait(bar_s_free, s_free_ph[0], abort_flag, p.status, 22))) break;
+                    if (!(ok = wait(bar_s_free, s_free_ph[0], 22))) break;
                     s_free_ph[0] ^= 1u;
                     tcgen05_fence_after();
                     issue_qk(t + 1, 0);
                 }
                 if (t >= n_kv) {  // (b) out += P V once the softmax warps have written this step's P tile
-                    if (!(ok = mbar_wait(bar_p_full, p_full_ph, abort_flag, p.status, 24))) break;
+                    if (!(ok = wait(bar_p_full, p_full_ph, 24))) break;
                     p_full_ph ^= 1u;
-                    if (!(ok = mbar_wait(bar_v + st, vph[st], abort_flag, p.status, 25))) break;
+                    if (!(ok = wait(bar_v + st, vph[st], 25))) break;
                     vph[st] ^= 1u;
                     tcgen05_fence_after();
-                    const uint32_t pa = smem_u32(s_p), va = smem_u32(s_v + st * TILE_BYTES);
+                    if (elect_one()) {
+                        const uint32_t v_lo = v_lo0 + (uint32_t)((st * TILE_BYTES) >> 4);
 #pragma unroll
-                    for (int k = 0; k < TILE / UMMA_K; ++k)
-                        umma_i8<1>(tmem_o, make_smem_desc(pa + k * UMMA_K, 16),
-                                   make_smem_desc(va + k * (UMMA_K * 128), 16384u), idesc_pv, (t > n_kv || k > 0) ? 1u : 0u);
-                    umma_commit<1>(bar_pv_done);
+                        for (int k = 0; k < TILE / UMMA_K; ++k)
+                            umma_i8_lo<1>(tmem_o, p_lo + k * (UMMA_K >> 4), v_lo + k * ((UMMA_K * 128) >> 4), idesc_pv,
+                                          (t > n_kv || k > 0) ? 1u : 0u);
+                        umma_commit_u32<1>(bar_addr(bar_pv_done));
+                    }
                 }
                 if (more) {  // (c) second half of the next step
-                    if (!(ok = mbar_wait(bar_s_free + 1, s_free_ph[1], abort_flag, p.status, 23))) break;
+                    if (!(ok = wait(bar_s_free + 1, s_free_ph[1], 23))) break;
                     s_free_ph[1] ^= 1u;
                     tcgen05_fence_after();
                     issue_qk(t + 1, 1);
                 }
                 if (t + 2 < T) {  // (d) this step's stages are free once its MMAs are complete: refill them
                     if (t >= n_kv) {  // K(t): both halves drained above; V(t): wait for P.V
-                        if (!(ok = mbar_wait(bar_pv_done, pv_done_ph, abort_flag, p.status, 27))) break;
+                        if (!(ok = wait(bar_pv_done, pv_done_ph, 27))) break;
                         pv_done_ph ^= 1u;
                     }
                     load_kv(t + 2);
