@@ -32,6 +32,7 @@
 #include "sq_common.cuh"
 #include "sq_bulk.cuh"
 #include "sq_kernels.h"
+#include "sq_tcgen05.cuh"
 
 namespace sq {
 
@@ -131,12 +132,56 @@ __global__ void row_wait_selftest_kernel(uint32_t* status, uint32_t budget) {
     }
 }
 
+// Sixteen 32-bit words per thread to / from tensor memory (lane = thread of the warp's lane quarter).
+__device__ __forceinline__ void tm_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+__device__ __forceinline__ void tm_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tm_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tm_ld_wait8(uint32_t (&r)[8]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) asm volatile("" : "+r"(r[i]));
+}
+// The loaded words may be used only behind the wait: route them through an empty statement placed after it.
+__device__ __forceinline__ void tm_ld_wait16(uint32_t (&r)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) asm volatile("" : "+r"(r[i]));
+}
+
 // EXACT: the row has exactly GROUP * V vectors, so no per-vector bounds checks are needed.
+// TM (LayerNorm, EXACT): the folded parameters do not sit in shared memory as 16-bit values that every row
+// unpacks again (two integer instructions per element, a fifth of all the kernel issues) but in TENSOR
+// MEMORY as fp32, written once per CTA: a thread's 16 V words (gamma and beta of its V vectors) live in its
+// own lane, and the threads of all groups that hold the same columns share them (warps W and W + 4k of
+// a lane quarter hold the same columns unless the group has eight warps, which then take two column
+// ranges).  The values are the unpacked 16-bit parameters, so the arithmetic is unchanged bit for bit;
+// the 4 C bytes of shared memory go to more ring stages.
 // MUL (never together with LN): every element is first multiplied by a per-column fp32 factor --
 // s_j when weights are folded (Eq. 3), 1/s_j for an activation whose producer cannot absorb it.
 // The factors live in shared memory for the CTA's lifetime, in the space LayerNorm's parameters
 // would take (4 bytes per column either way).
-template <typename T, int GROUP, int V, bool LN, bool EXACT, bool MUL = false, int CTA = CTA_THREADS>
+template <typename T, int GROUP, int V, bool LN, bool EXACT, bool MUL = false, int CTA = CTA_THREADS, int TMW = 0>
 __global__ void __launch_bounds__(CTA, 1)
 row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__ gamma,
                 const T* __restrict__ beta, const float* __restrict__ col_mul, float eps, int mode, int stages,
@@ -145,13 +190,17 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                 int stats_are_input, uint32_t* __restrict__ status) {
     constexpr int G = CTA / GROUP;  // rows in flight per CTA
     constexpr int NW = GROUP / 32;
+    constexpr bool TM = TMW != 0;   // parameters in tensor memory, read TMW (8 or 16) words at a time
+    static_assert(TMW == 0 || TMW == 8 || TMW == 16, "tensor-memory read width");
     extern __shared__ __align__(128) uint8_t smem[];
     const int row_bytes = C * 2;
     const int nvec = C >> 3;
-    uint8_t* s_gamma = smem;                                   // [C] T   (LN only)
-    uint8_t* s_beta = smem + (LN ? row_bytes : 0);             // [C] T   (LN only)
+    static_assert(!TM || (LN && EXACT && !MUL && 16 * V * (NW == 8 ? 2 : 1) <= 512 && (NW == 1 || NW == 2 || NW == 4 || NW == 8)),
+                  "tensor-memory parameters: LayerNorm on exact rows, one or two column ranges of 16 V words");
+    uint8_t* s_gamma = smem;                                   // [C] T   (LN only, not TM)
+    uint8_t* s_beta = smem + (LN ? row_bytes : 0);             // [C] T   (LN only, not TM)
     const float* s_mul = reinterpret_cast<const float*>(smem); // [C] fp32 (MUL only)
-    uint8_t* s_rows = smem + ((LN || MUL) ? 2 * row_bytes : 0);  // [G][stages][C] T
+    uint8_t* s_rows = smem + (((LN && !TM) || MUL) ? 2 * row_bytes : 0);  // [G][stages][C] T
     uint64_t* full = reinterpret_cast<uint64_t*>(s_rows + (size_t)G * stages * row_bytes);  // [G][stages]
     constexpr int NWP = (NW + 3) & ~3;  // partial slots padded to whole 16-byte vectors
     float* s_red = reinterpret_cast<float*>(
@@ -167,6 +216,9 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     uint8_t* my_rows = s_rows + (size_t)g * stages * row_bytes;
     float* red = s_red + g * 3 * NWP;
     volatile uint32_t* my_flag = reinterpret_cast<volatile uint32_t*>(s_red + G * 3 * NWP) + g;
+    uint32_t* tmem_holder = const_cast<uint32_t*>(reinterpret_cast<volatile uint32_t*>(s_red + G * 3 * NWP) + G);
+    constexpr uint32_t kTmCols = 512;
+    if (TM && tid < 32) tc::tmem_alloc<1>(tmem_holder, kTmCols);  // warp 0; freed at the end of the kernel
 
     if (gt == 0) {
         for (int s = 0; s < stages; ++s) mbar_init(my_full + s, 1);
@@ -189,7 +241,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
         const float4* m4 = reinterpret_cast<const float4*>(col_mul);
         for (int v = tid; v < 2 * nvec; v += CTA) reinterpret_cast<float4*>(smem)[v] = __ldg(m4 + v);
     }
-    if (LN) {  // parameters: global -> shared once per CTA
+    if (LN && !TM) {  // parameters: global -> shared once per CTA
         const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
         const uint4* b4 = reinterpret_cast<const uint4*>(beta);
         for (int v = tid; v < nvec; v += CTA) {
@@ -197,7 +249,38 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
             reinterpret_cast<uint4*>(s_beta)[v] = beta ? __ldg(b4 + v) : make_uint4(0u, 0u, 0u, 0u);
         }
     }
+    uint32_t tm_addr = 0;
+    if (TM) {
+        tc::tcgen05_fence_before();
+        __syncthreads();  // the allocation's address is in shared memory
+        tc::tcgen05_fence_after();
+        const int warp = tid >> 5;
+        // this thread's lane quarter and, for eight-warp groups, the column range of its half of the group
+        tm_addr = *tmem_holder + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)((NW == 8 ? (gwarp >> 2) : 0) * 16 * V);
+        if (warp < (NW == 8 ? 8 : 4)) {  // one writer per lane quarter and column range
+            const uint4* g4 = reinterpret_cast<const uint4*>(gamma);
+            const uint4* b4 = reinterpret_cast<const uint4*>(beta);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const int v = gt + i * GROUP;
+                float2 ga[4], be[4];
+                unpack8_pairs<T>(__ldg(g4 + v), ga);
+                unpack8_pairs<T>(beta ? __ldg(b4 + v) : make_uint4(0u, 0u, 0u, 0u), be);
+                uint32_t w[16];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {  // words: gamma, beta of pairs 0, 1, then of pairs 2, 3 (eight words per half vector)
+                    const int o = 8 * (j >> 1) + 2 * (j & 1);
+                    w[o] = __float_as_uint(ga[j].x); w[o + 1] = __float_as_uint(ga[j].y);
+                    w[o + 4] = __float_as_uint(be[j].x); w[o + 5] = __float_as_uint(be[j].y);
+                }
+                tm_st16(tm_addr + 16 * i, w);
+            }
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+        tc::tcgen05_fence_before();
+    }
     __syncthreads();
+    if (TM) tc::tcgen05_fence_after();
 
     float tensor_delta = 0.0f;
     if (mode == ROW_GIVEN_SCALE) tensor_delta = __ldg(scale);
@@ -301,6 +384,36 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
             }
             const float shift = -__fmul_rn(mu, rstd);
             const float2 rstd2 = make_float2(rstd, rstd), shift2 = make_float2(shift, shift);
+            if constexpr (TM) {
+                // TMW words at a time (a vector's 16, or half a vector's 8 where registers are short), the next
+                // read on its way while this one is used; a half vector holds gamma, beta of two pairs
+                constexpr int NP = TMW / 4;  // pairs per read
+                uint32_t gb[2][TMW == 0 ? 8 : TMW];
+                auto ld = [&](int k, uint32_t (&r)[TMW == 0 ? 8 : TMW]) {
+                    if constexpr (TMW == 16) tm_ld16(tm_addr + 16 * k, r); else tm_ld8(tm_addr + 8 * k, r);
+                };
+                auto ld_wait = [&](uint32_t (&r)[TMW == 0 ? 8 : TMW]) {
+                    if constexpr (TMW == 16) tm_ld_wait16(r); else tm_ld_wait8(r);
+                };
+                constexpr int READS = 16 * V / (TMW == 0 ? 8 : TMW);
+                ld(0, gb[0]);
+#pragma unroll
+                for (int k = 0; k < READS; ++k) {
+                    uint32_t (&cur)[TMW == 0 ? 8 : TMW] = gb[k & 1];
+                    ld_wait(cur);
+                    if (k + 1 < READS) ld(k + 1, gb[(k + 1) & 1]);
+#pragma unroll
+                    for (int jj = 0; jj < NP; ++jj) {
+                        const int i = (k * NP + jj) >> 2, j = (k * NP + jj) & 3;
+                        const int o = 8 * (jj >> 1) + 2 * (jj & 1);  // word of this pair's gamma inside the read
+                        const float2 ga = make_float2(__uint_as_float(cur[o]), __uint_as_float(cur[o + 1]));
+                        const float2 be = make_float2(__uint_as_float(cur[o + 4]), __uint_as_float(cur[o + 5]));
+                        const float2 t = __ffma2_rn(__ffma2_rn(y[FP32_ROW ? i : 0][j], rstd2, shift2), ga, be);
+                        y[FP32_ROW ? i : 0][j] = t;
+                        m = fmaxf(m, fmaxf(fabsf(t.x), fabsf(t.y)));
+                    }
+                }
+            } else {
 #pragma unroll
             for (int i = 0; i < V; ++i) {
                 const int v = gt + i * GROUP;
@@ -316,6 +429,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
                         m = fmaxf(m, fmaxf(fabsf(t.x), fabsf(t.y)));
                     }
                 }
+            }
             }
         } else if (MUL) {
 #pragma unroll
@@ -393,22 +507,31 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     }
     if (mode == ROW_ABSMAX_ONLY && gt == 0) atomic_max_nonneg(absmax_word, group_max);
     (void)parity;
+    if (TM) {  // every group is done with the parameters (whether it finished or gave up)
+        tc::tcgen05_fence_before();
+        __syncthreads();
+        if (tid < 32) {
+            tc::tcgen05_fence_after();
+            tc::tmem_dealloc<1>(*tmem_holder, kTmCols);
+        }
+    }
 }
 
-template <typename T, int GROUP, int V, bool LN, bool EXACT = false, bool MUL = false, int CTA = CTA_THREADS>
+template <typename T, int GROUP, int V, bool LN, bool EXACT = false, bool MUL = false, int CTA = CTA_THREADS, int TMW = 0>
 sq_status launch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, const void* beta, const float* col_mul, float eps,
                       int mode, int8_t* Xq, float* scale, float* absmax_word, float* stats, int stats_are_input,
                       uint32_t* status, cudaStream_t st) {
     constexpr int G = CTA / GROUP;
+    constexpr bool TM = TMW != 0;
     const size_t row_bytes = (size_t)C * 2;
-    const size_t fixed = ((LN || MUL) ? 2 * row_bytes : 0) + 2048 /*barriers + reduction scratch*/;
+    const size_t fixed = (((LN && !TM) || MUL) ? 2 * row_bytes : 0) + 2048 /*barriers + reduction scratch*/;
     const size_t budget = 220 * 1024;
     if (budget < fixed + G * row_bytes) return SQ_ERR_UNSUPPORTED;
     int stages = (int)((budget - fixed) / (G * row_bytes));
     stages = std::min(stages, 8);
-    const size_t smem = ((LN || MUL) ? 2 * row_bytes : 0) + (size_t)G * stages * row_bytes + (size_t)G * stages * 8 +
-                        (size_t)G * 3 * ((GROUP / 32 + 3) & ~3) * 4 + (size_t)G * 4 + 144;
-    auto kern = row_pipe_kernel<T, GROUP, V, LN, EXACT, MUL, CTA>;
+    const size_t smem = (((LN && !TM) || MUL) ? 2 * row_bytes : 0) + (size_t)G * stages * row_bytes + (size_t)G * stages * 8 +
+                        (size_t)G * 3 * ((GROUP / 32 + 3) & ~3) * 4 + (size_t)G * 4 + 4 + 144;
+    auto kern = row_pipe_kernel<T, GROUP, V, LN, EXACT, MUL, CTA, TMW>;
     static bool attr_set[64] = {false};
     int dev = 0;
     SQ_CUDA_OK(cudaGetDevice(&dev));
@@ -443,12 +566,23 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
         if (nvec == (GROUP) * (V))                                                                               \
             return launch_pipe<T, GROUP, V, LN, true, false, 384>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, scale, \
                                                                   absmax_word, stats, stats_are_input, status, st)
-        SQ_PIPE_LN384(32, 16);   // 4096: one warp per row, no barrier in the reductions
-        SQ_PIPE_LN384(64, 14);   // 7168
+        // Parameters in tensor memory where it measured faster (fraction of the 6534 GB/s copy bandwidth, shared
+        // memory -> tensor memory): 32768 x 4096 0.84 -> 0.86 with whole-vector reads; with half-vector reads
+        // 16384 x 14336 0.85 -> 0.92, 16384 x 20480 0.83 -> 0.89-0.92 and 8192 x 7168 43.1 -> 37.2 us (65536 x 7168
+        // unchanged at 0.90); 5120 and 8192 lose 4-5 % and stay as they were; groups of three warps (9216, 12288)
+        // would need three column ranges, more than tensor memory has.
+#define SQ_PIPE_LN_TM(GROUP, V, CTA, TMW)                                                                        \
+        if (nvec == (GROUP) * (V))                                                                               \
+            return launch_pipe<T, GROUP, V, LN, true, false, CTA, LN ? TMW : 0>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, \
+                                                                                scale, absmax_word, stats, stats_are_input, status, st)
+        SQ_PIPE_LN_TM(32, 16, 384, 16);           // 4096
+        SQ_PIPE_LN_TM(64, 14, 384, 8);            // 7168
+        SQ_PIPE_LN_TM(128, 14, 384, 8);           // 14336
+        SQ_PIPE_LN_TM(256, 10, CTA_THREADS, 8);   // 20480
+#undef SQ_PIPE_LN_TM
         SQ_PIPE_LN384(64, 16);   // 8192
         SQ_PIPE_LN384(96, 12);   // 9216
         SQ_PIPE_LN384(96, 16);   // 12288
-        SQ_PIPE_LN384(128, 14);  // 14336
 #undef SQ_PIPE_LN384
     }
     SQ_PIPE_EXACT(64, 8);    // 4096
