@@ -569,19 +569,20 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
         // Parameters in tensor memory where it measured faster (fraction of the 6534 GB/s copy bandwidth, shared
         // memory -> tensor memory): 32768 x 4096 0.84 -> 0.86 with whole-vector reads; with half-vector reads
         // 16384 x 14336 0.85 -> 0.92, 16384 x 20480 0.83 -> 0.89-0.92 and 8192 x 7168 43.1 -> 37.2 us (65536 x 7168
-        // unchanged at 0.90); 5120 and 8192 lose 4-5 % and stay as they were; groups of three warps (9216, 12288)
-        // would need three column ranges, more than tensor memory has.
+        // unchanged at 0.90); 5120 and 8192 lose 4-5 % and stay as they were; groups of three warps (12288)
+        // would need three column ranges, more than tensor memory has, and 12288 as 128 x 12 gains 3 % at 16384 rows
+        // but loses 7 % at 4096.
 #define SQ_PIPE_LN_TM(GROUP, V, CTA, TMW)                                                                        \
         if (nvec == (GROUP) * (V))                                                                               \
             return launch_pipe<T, GROUP, V, LN, true, false, CTA, LN ? TMW : 0>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, \
                                                                                 scale, absmax_word, stats, stats_are_input, status, st)
         SQ_PIPE_LN_TM(32, 16, 384, 16);           // 4096
         SQ_PIPE_LN_TM(64, 14, 384, 8);            // 7168
+        SQ_PIPE_LN_TM(128, 9, 384, 16);           // 9216: four-warp groups (three-warp ones cannot share columns), 0.82 -> 0.90
         SQ_PIPE_LN_TM(128, 14, 384, 8);           // 14336
         SQ_PIPE_LN_TM(256, 10, CTA_THREADS, 8);   // 20480
 #undef SQ_PIPE_LN_TM
         SQ_PIPE_LN384(64, 16);   // 8192
-        SQ_PIPE_LN384(96, 12);   // 9216
         SQ_PIPE_LN384(96, 16);   // 12288
 #undef SQ_PIPE_LN384
     }
