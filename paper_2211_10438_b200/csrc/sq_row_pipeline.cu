@@ -9,9 +9,10 @@
 //   * rows arrive through a ring of shared-memory stages filled by cp.async.bulk (one bulk
 //     copy per row, completion on an mbarrier), so the next rows stream in from HBM while
 //     the current one is being reduced and quantised;
-//   * the folded LayerNorm parameters gamma_hat / beta_hat live in shared memory for the whole
-//     kernel; a row is unpacked once into registers, so HBM sees 2 bytes in + 1 byte out per
-//     element and nothing else;
+//   * the folded LayerNorm parameters gamma_hat / beta_hat live on the SM for the whole kernel -- in
+//     shared memory as 16-bit values, or (hidden sizes 4096, 7168, 9216, 14336, 20480) as fp32 in
+//     tensor memory, which saves unpacking them for every row; a row is unpacked once into
+//     registers, so HBM sees 2 bytes in + 1 byte out per element and nothing else;
 //   * reductions are warp shuffles + one named barrier each: one for the statistics (per-thread
 //     mean and squared deviations merged with the parallel-variance update; rows with a ragged
 //     tail take the sum first and the deviations second), one for the absolute maximum.
@@ -21,11 +22,11 @@
 // HBM traffic per element), hence the two-wide fp32 instructions (same rounding per half as the
 // scalar ones), the single-FMA rounding, byte-permute packing, vector loads of the reduction
 // partials and multiplications by 1/C in the statistics.
-// Tried and measured no faster: gamma_hat / beta_hat in each thread's own tensor-memory lane
-// (tcgen05.st once, tcgen05.ld one vector ahead), which frees their shared memory for a second
-// ring stage at hidden sizes 8192 to 20480 -- bit-identical output, 0.79 instead of 0.81 of the copy
-// bandwidth at 20480 and 0.82 instead of 0.87 at 12288, so the bytes in flight are not what
-// limits those shapes; 256- and 320-thread CTAs with 128 to 160 values per thread at 20480 (too
+// Tried and measured no faster: gamma_hat / beta_hat as 16-BIT values in each thread's own
+// tensor-memory lane, which frees their shared memory for a second ring stage at hidden sizes 8192
+// to 20480 -- bit-identical output, 0.79 instead of 0.81 of the copy bandwidth at 20480 and 0.82
+// instead of 0.87 at 12288, so the bytes in flight are not what limits those shapes (the
+// instructions are: the fp32 form above removes two of them per element); 256- and 320-thread CTAs with 128 to 160 values per thread at 20480 (too
 // few warps to cover the reductions); 640 threads with 64 values per thread; fp32 copies of
 // gamma_hat / beta_hat in shared memory, which take the two unpacks per element out of the inner
 // loop but double the bytes every row reads back from shared memory (65536 x 7168: 0.96 -> 0.71).
