@@ -71,32 +71,49 @@ __device__ __forceinline__ float ex2_approx(float x) {
 // INT32 -> fp32 for |a| < 2^22 without the conversion unit (which shares its pipe with ex2): adding
 // the integer to the bit pattern of 1.5 * 2^23 gives the float 1.5 * 2^23 + a exactly (one unit in
 // the last place is 1 there), and the subtraction is exact.  Scores obey |q . k| <= 127^2 * 128 < 2^21.
-__device__ __forceinline__ float score_to_float(uint32_t a) {
-    return __int_as_float((int)a + 0x4B400000) - 12582912.0f;
-}
+// (Done on pairs in score_pair_x below.)
 
 // Pass 1 on one chunk of 32 scores: running maximum (exp2 domain) and sum.  NVIS = 32 for chunks
 // that lie entirely below the diagonal (no per-element visibility test), otherwise the count of
 // visible keys is passed in.  Four partial sums keep the adds independent of one another.
 // Invisible keys of a diagonal chunk are handled without branches: their exponent argument is
 // replaced by -inf (ex2 gives 0, the P code rounds to 0) and their score by INT_MIN in the maximum.
+// The softmax warps are bound by instruction issue, so the per-score work is done on PAIRS with the
+// two-wide fp32 instructions (each half rounds exactly like the scalar instruction; one issue slot for
+// two values) and the integer maximum with the three-input form: bit for bit the scalar sequence --
+// magic-number conversion, x = fma(s, c1, -m2), ex2, four partial sums over the scores c = 0..3 mod 4.
+__device__ __forceinline__ float2 score_pair_x(uint32_t a0, uint32_t a1, float2 c1v, float2 neg_m2) {
+    const float2 s = __fadd2_rn(make_float2(__int_as_float((int)a0 + 0x4B400000), __int_as_float((int)a1 + 0x4B400000)),
+                                make_float2(-12582912.0f, -12582912.0f));
+    return __ffma2_rn(s, c1v, neg_m2);
+}
+
 template <bool FULL>
 __device__ __forceinline__ void pass1_chunk(const uint32_t (&acc)[32], int nvis, float c1, float& m2, float& l) {
     int cmax = INT_MIN;
+    if (FULL) {
+        cmax = max((int)acc[0], (int)acc[1]);
 #pragma unroll
-    for (int c = 0; c < 32; ++c) cmax = max(cmax, (FULL || c < nvis) ? (int)acc[c] : INT_MIN);
+        for (int c = 2; c < 32; c += 2) cmax = __vimax3_s32(cmax, (int)acc[c], (int)acc[c + 1]);
+    } else {
+#pragma unroll
+        for (int c = 0; c < 32; ++c) cmax = max(cmax, c < nvis ? (int)acc[c] : INT_MIN);
+    }
     const float cm2 = c1 * __int2float_rn(cmax);
     if (cm2 > m2) {  // rescale the running sum to the new maximum
         l *= ex2_approx(m2 - cm2);
         m2 = cm2;
     }
-    float s[4] = {0.0f, 0.0f, 0.0f, 0.0f};  // four partial sums keep the adds independent
+    const float2 c1v = make_float2(c1, c1), neg_m2 = make_float2(-m2, -m2);
+    float2 s[2] = {make_float2(0.0f, 0.0f), make_float2(0.0f, 0.0f)};  // four partial sums keep the adds independent
 #pragma unroll
-    for (int c = 0; c < 32; ++c) {
-        const float x = fmaf(score_to_float(acc[c]), c1, -m2);
-        s[c & 3] += ex2_approx((FULL || c < nvis) ? x : -INFINITY);
+    for (int c = 0; c < 32; c += 2) {
+        const float2 x = score_pair_x(acc[c], acc[c + 1], c1v, neg_m2);
+        const float2 e = make_float2(ex2_approx((FULL || c < nvis) ? x.x : -INFINITY),
+                                     ex2_approx((FULL || c + 1 < nvis) ? x.y : -INFINITY));
+        s[(c >> 1) & 1] = __fadd2_rn(s[(c >> 1) & 1], e);
     }
-    l += (s[0] + s[1]) + (s[2] + s[3]);
+    l += (s[0].x + s[0].y) + (s[1].x + s[1].y);
 }
 
 // Pass 2 on one chunk: P = round(127 * e / l) as INT8 codes, 32 keys = two 16-byte pieces of this
@@ -104,15 +121,21 @@ __device__ __forceinline__ void pass1_chunk(const uint32_t (&acc)[32], int nvis,
 template <bool FULL>
 __device__ __forceinline__ void pass2_chunk(const uint32_t (&acc)[32], int nvis, float c1, float m2, float k127,
                                             uint8_t* prow, int r, int cc) {
+    const float2 c1v = make_float2(c1, c1), neg_m2 = make_float2(-m2, -m2);
+    const float2 k2 = make_float2(k127, k127), magic2 = make_float2(kRoundMagic, kRoundMagic);
     uint32_t w[8];
 #pragma unroll
     for (int v = 0; v < 8; ++v) {
         uint32_t q[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int c = 4 * v + e;
-            const float x = fmaf(score_to_float(acc[c]), c1, -m2);
-            q[e] = quant_code<false>(ex2_approx((FULL || c < nvis) ? x : -INFINITY), k127);  // e <= l: code <= 127
+        for (int h2 = 0; h2 < 2; ++h2) {
+            const int c = 4 * v + 2 * h2;
+            const float2 x = score_pair_x(acc[c], acc[c + 1], c1v, neg_m2);
+            const float2 e = make_float2(ex2_approx((FULL || c < nvis) ? x.x : -INFINITY),
+                                         ex2_approx((FULL || c + 1 < nvis) ? x.y : -INFINITY));
+            const float2 rr = __ffma2_rn(e, k2, magic2);  // e <= l: the code cannot exceed 127, no clamp
+            q[2 * h2] = __float_as_uint(rr.x);
+            q[2 * h2 + 1] = __float_as_uint(rr.y);
         }
         w[v] = pack4(q[0], q[1], q[2], q[3]);
     }
