@@ -218,7 +218,7 @@ row_pipe_kernel(const T* __restrict__ X, int64_t M, int C, const T* __restrict__
     float* red = s_red + g * 3 * NWP;
     volatile uint32_t* my_flag = reinterpret_cast<volatile uint32_t*>(s_red + G * 3 * NWP) + g;
     uint32_t* tmem_holder = const_cast<uint32_t*>(reinterpret_cast<volatile uint32_t*>(s_red + G * 3 * NWP) + G);
-    constexpr uint32_t kTmCols = 512;
+    constexpr uint32_t kTmCols = 16 * V * (NW == 8 ? 2 : 1) <= 256 ? 256 : 512;  // a power of two that holds the column ranges
     if (TM && tid < 32) tc::tmem_alloc<1>(tmem_holder, kTmCols);  // warp 0; freed at the end of the kernel
 
     if (gt == 0) {
