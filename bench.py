@@ -363,11 +363,11 @@ def generation_rows(lin, steps, prompt_blk, B, S, H, d, hid, dt, ch, fac, seed, 
         gen.ctx.fill_(ctx)
         gen.lens.fill_(ctx + 1)
         for _ in range(3):
-            gen.step(x, advance=False)
+            gen.step(x, max_len=ctx + 1, advance=False)  # the host knows how far every sequence has got
         torch.cuda.synchronize()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            gen.step(x, advance=False)
+            gen.step(x, max_len=ctx + 1, advance=False)  # the host knows how far every sequence has got
         time.sleep(0.2)
         for _ in range(3):
             g.replay()

@@ -36,7 +36,7 @@ constexpr int KV_TILE = 32;                  // keys per ring stage
 constexpr int KV_TILE_BYTES = KV_TILE * KV_D;
 constexpr int KV_WARPS = 4;
 constexpr int KV_THREADS = KV_WARPS * 32;
-constexpr int KV_STAGES = 4;                 // ring stages per warp
+constexpr int KV_STAGES = 2;                 // ring stages per warp (two: five CTAs fit an SM; deeper rings with fewer CTAs measured slower)
 constexpr int KV_MAX_CLUSTER = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -124,6 +124,19 @@ kv_decode_attention_kernel(const KvParams p) {
     }
     pdl_wait();  // q, the cache and the lengths may come from the preceding launch
     pdl_launch_dependents();
+    // Everything this CTA reads besides the cache is requested here, at once: the sequence length, the new
+    // token's key and value rows, the re-quantisation factor.  Read where they are used, each of them is a
+    // dependent trip to L2 or HBM (about a microsecond) on a path that is nothing but latency at short contexts.
+    const size_t new_off = (size_t)b * p.ld_new + (size_t)h * KV_D;
+    uint4 k_new_row = make_uint4(0u, 0u, 0u, 0u);
+    uint32_t v_new_word = 0u;
+    int8_t v_new_byte = 0;
+    if (p.k_new != nullptr) {
+        if (w == 0 && lane < KV_D / 16) k_new_row = __ldg(reinterpret_cast<const uint4*>(p.k_new + new_off) + lane);
+        if (w == 0) v_new_word = __ldg(reinterpret_cast<const uint32_t*>(p.v_new + new_off) + lane);
+        v_new_byte = __ldg(p.v_new + new_off + tid);
+    }
+    const float requant = (p.out_dt == SQ_I8 && crank == 0) ? __ldg(p.requant_mul) : 1.0f;
     int len = __ldg(p.lens + b);
     const bool truncated = len > p.max_len;
     if (truncated) {  // the caller's bound was wrong: say so, and stay inside what was sized
@@ -207,11 +220,10 @@ kv_decode_attention_kernel(const KvParams p) {
         __syncwarp();
         if (lane == 0 && u + KV_STAGES < total) issue(u + KV_STAGES);
     }
-    const size_t new_off = (size_t)b * p.ld_new + (size_t)h * KV_D;
     if (owns_new && w == 0) {  // score of the newest position from its own key row
         int acc = 0;
         if (lane < KV_D / 16) {
-            const uint4 kv = __ldg(reinterpret_cast<const uint4*>(p.k_new + new_off) + lane);
+            const uint4 kv = k_new_row;
             const uint4 qv = *reinterpret_cast<const uint4*>(q_s + lane * 16);
             acc = __dp4a((int)kv.x, (int)qv.x, acc);
             acc = __dp4a((int)kv.y, (int)qv.y, acc);
@@ -292,13 +304,13 @@ kv_decode_attention_kernel(const KvParams p) {
     if (owns_new) {
         const int pos = len - 1;
         if (w == 0) {  // the newest position's share of the output, from its own value row
-            const uint32_t vw = __ldg(reinterpret_cast<const uint32_t*>(p.v_new + new_off) + lane);
+            const uint32_t vw = v_new_word;
 #pragma unroll
             for (int k = 0; k < 4; ++k) o[k] += p_new * (int)(int8_t)((vw >> (8 * k)) & 0xffu);
         }
         // value row -> cache: channel tid, byte (pos % 4) of its 4-position word
         p.vc[(((size_t)b * p.H + h) * (size_t)p.lmax + (size_t)(pos & ~3)) * KV_D + (size_t)tid * 4 + (pos & 3)] =
-            __ldg(p.v_new + new_off + tid);
+            v_new_byte;
     }
     *reinterpret_cast<int4*>(wpart + w * KV_D + 4 * lane) = make_int4(o[0], o[1], o[2], o[3]);
     __syncthreads();
@@ -314,7 +326,7 @@ kv_decode_attention_kernel(const KvParams p) {
         for (int r = 0; r < C; ++r) tot += (int)ld_cluster_u32(x_part + tid, (uint32_t)r);
         const float y = __fmul_rn(__int2float_rn(tot), p.alpha_pv);
         if (p.out_dt == SQ_I8)
-            reinterpret_cast<int8_t*>(p.out)[out_off] = (int8_t)(quant_code(y, __ldg(p.requant_mul)) & 0xffu);
+            reinterpret_cast<int8_t*>(p.out)[out_off] = (int8_t)(quant_code(y, requant) & 0xffu);
         else if (p.out_dt == SQ_F16)
             reinterpret_cast<__half*>(p.out)[out_off] = __float2half_rn(y);
         else
@@ -375,10 +387,13 @@ kv_cache_write_kernel(const int8_t* __restrict__ qkv, int64_t ld, int B, int T, 
 
 }  // namespace
 
-// Cluster width: enough CTAs to fill the machine a few times over, each keeping a worthwhile
-// number of keys, and a score buffer that fits in shared memory.
+// Cluster width: enough CTAs to put two on every SM, each keeping a worthwhile number of keys, and a
+// score buffer that fits in shared memory.  Splitting a sequence costs three cluster-wide meetings, so
+// it is done only when (sequence, head) pairs alone leave SMs idle: measured on B200, 56 heads, context
+// 2047, wanting 2 / 4 / 8 CTAs per SM: batch 2: 11.3 / 15.1 / 15.2 us, batch 4: 25.1 / 28.2 / 33.4,
+// batch 8: 37.4 / 47.6 / 47.0 (batch 12: 63.8 / 64.0 / 58.9).
 int kv_choose_cluster(int64_t B, int64_t H, int64_t max_len) {
-    const int64_t want = 4LL * sm_count();
+    const int64_t want = 2LL * sm_count();
     int c = 1;
     while (c < KV_MAX_CLUSTER && B * H * c < want && max_len / (2 * c) >= 256) c *= 2;
     while (c < KV_MAX_CLUSTER && kv_smem_bytes((int)(((max_len + c - 1) / c + KV_TILE - 1) / KV_TILE * KV_TILE)) > 200 * 1024) c *= 2;

@@ -148,7 +148,7 @@ def generation_block(args):
     blk.ctx.fill_(args.S)
     blk.lens.fill_(args.S + 1)
     x = torch.randn((B, hid), device="cuda", dtype=dt, generator=g)
-    us = _time(lambda: blk.step(x, advance=False), args.calls)
+    us = _time(lambda: blk.step(x, max_len=args.S + 1, advance=False), args.calls)
     byts = blk.bytes_per_step(args.S * B)
     print("generation_block B=%d ctx=%d, %d launches per step: %.1f us per step (stream, no graph), %.0f GB/s of weights + cache"
           % (B, args.S, blk.launches_per_step, us, byts / us / 1e3))
