@@ -33,7 +33,7 @@ SAMPLE_ROWS_BASELINE = 2048  # the whole config-2 problem
 SAMPLE_ROWS_REFERENCE = 64
 # dram__bytes_read.sum + dram__bytes_write.sum per gemm_i8_kernel launch, mean over the four GEMMs of one step,
 # from the ncu capture summarised in profiles/gemm_i8_kernel__opt13b_prefill.md
-GEMM_DRAM_BYTES_PER_LAUNCH = 141.5e6
+GEMM_DRAM_BYTES_PER_LAUNCH = 128.3e6
 
 
 def measured_peaks():

@@ -149,6 +149,26 @@ __device__ __forceinline__ void tma_load_4d_policy(void* dst, const CUtensorMap*
         : "memory");
 }
 
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// tma_load_4d<CG> with an L2 cache policy
+template <int CG>
+__device__ __forceinline__ void tma_load_4d_hint(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1,
+                                                 int c2, int c3, uint64_t policy) {
+    if (CG == 1) {
+        tma_load_4d_policy(dst, map, bar, c0, c1, c2, c3, policy);
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+            "[%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+            ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar) & kPeerBitMask), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+            : "memory");
+    }
+}
+
 // Pulls one box of a tensor map into L2 without a shared-memory destination.
 __device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
     asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global [%0, {%1, %2, %3, %4}];"
