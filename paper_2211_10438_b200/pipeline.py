@@ -261,9 +261,9 @@ class DecoderBlockDecode:
     `fused=True` moves both LayerNorm+quantise steps into the prologues of the GEMMs that consume
     them (five launches).  Measured on B200 (OPT-30B shapes, batch 16, one CUDA graph per step): inside
     a chain of dependent launches the separate quantiser kernel overlaps the GEMM's own start-up and
-    the seven-launch form is the faster one (158 against 164 us per layer); for a GEMM called on its
+    the seven-launch form is the faster one (152 against 158 us per layer); for a GEMM called on its
     own the fused form wins.  `fuse_residual=False` keeps the residual adds as kernels of their own
-    (nine launches with `fused=False`: 161 us).  Same `lin` / `steps` as the prompt block.  `ctx`
+    (nine launches with `fused=False`: about 3 us more).  Same `lin` / `steps` as the prompt block.  `ctx`
     (int32 device tensor [B]) counts the positions each sequence has cached.  `keep_codes` also
     writes the LayerNorm codes of the fused form to x1q / x2q so that a checker can look at them."""
 
