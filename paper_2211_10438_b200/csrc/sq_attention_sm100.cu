@@ -304,6 +304,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
         const int qi = qt * TILE + r;                // query position
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t s_full_ph = 0, pv_done_ph = 0;
+        const float rq = __ldg(p.requant_mul);  // requested now: read in the epilogue it would be a dependent trip to L2
         const float c1 = p.alpha_qk * kLog2e;  // exp(alpha * acc - max) = exp2(c1 * acc - m2)
         float m2 = -INFINITY, l = 0.0f;        // running maximum (in the exp2 domain) and sum of this half
         bool ok = true;
@@ -364,7 +365,6 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
         // ---- epilogue: out = round(((P V) * alpha_pv) * requant); each half takes 64 output channels ----
         if (ok && (ok = warp_wait(bar_pv_done, pv_done_ph, abort_flag, p.status, 29))) {
             tcgen05_fence_after();
-            const float rq = __ldg(p.requant_mul);
             int8_t* orow = p.out + ((int64_t)(row_base + qi)) * p.hid + h * TILE;
 #pragma unroll 1
             for (int cc = 2 * g; cc < 2 * g + 2; ++cc) {

@@ -180,7 +180,7 @@ __device__ __forceinline__ int tile_num_kb(const Params& p, int mi, int tile_m) 
 template <int BLOCK_N, bool FIX = false, bool EW8 = false, bool PLAIN16 = false>
 __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap* tmap_c, uint8_t* stg,
                                               uint32_t taddr, int64_t row, int row0_warp, int64_t col0, int b,
-                                              int h, int64_t c_off, const float* s_wscale,
+                                              int h, int64_t c_off, float xs, const float* s_wscale,
                                               const float* s_bias, const float* s_requant, int lane,
                                               int cc_begin, int cc_end, const int32_t* fix_base = nullptr,
                                               int fix_count = 0, int fix_mine = 0, size_t fix_stride = 0) {
@@ -193,8 +193,6 @@ __device__ __forceinline__ void epilogue_slot(const Params& p, const CUtensorMap
     const void* const residual = PLAIN16 ? nullptr : p.residual;
     float* const row_absmax_out = PLAIN16 ? nullptr : p.row_absmax_out;
     const bool row_ok = row < p.M;
-    float xs = p.alpha;
-    if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row_ok) ? row : 0));
     float row_max = 0.0f;
     // 32-column chunks per 128-byte staging row: 1 (int32), 2 (fp16/bf16), 4 (int8)
     const int chunks_per_store = out_dt == SQ_I32 ? 1 : (out_dt == SQ_I8 ? 4 : 2);
@@ -663,6 +661,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + off));
                 }
             }
+            // this thread's row and its activation step: requested while the tile's MMAs still run (read behind the
+            // wait, the load is a dependent trip to L2 in every tile's epilogue)
+            const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
+            float xs = p.alpha;
+            if (p.x_scale) xs = __ldg(p.x_scale + ((p.x_per_row && row < p.M) ? row : 0));
             if (et == 0)
                 *epi_go = mbar_wait(tmem_full + slot, slot_phase, abort_flag, p.status, 4) ? 1u : 0u;
             epi_bar_sync<C::EPI_THREADS>();  // constants staged; outcome of the wait visible to all epilogue threads
@@ -672,7 +675,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             trace_go = clock64();
 #endif
 
-            const int64_t row = ((int64_t)mi * CG + rank) * BLOCK_M + quarter * 32 + lane;
             const int64_t c_off = (int64_t)b * p.c_stride_batch + (int64_t)h * p.c_stride_head +
                                   row * p.c_stride_row + col0;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS);
@@ -686,7 +688,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int cc_end = half == 0 ? min(g_split * cps, width / 32) : width / 32;
             if (EW == 8 || piece < 0) {  // (the eight-warp configuration serves short reductions: never split)
                 epilogue_slot<BLOCK_N, false, EW == 8, PLAIN16>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b, h,
-                                       c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
+                                       c_off, xs, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end);
             } else {
                 // K piece of a split tile: park the accumulators, then see who is last
                 constexpr size_t kTileInts = (size_t)BLOCK_M * BLOCK_N;
@@ -712,7 +714,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 if (*epi_last != 0u) {
                     __threadfence();
                     epilogue_slot<BLOCK_N, true, false, PLAIN16>(p, &tmap_c, staging + warp * (32 * 128), taddr, row, row0_warp, col0, b,
-                                                 h, c_off, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end,
+                                                 h, c_off, xs, s_wscale, s_bias, s_requant, lane, cc_begin, cc_end,
                                                  tile_slots, p.split, piece, (size_t)CG * kTileInts);
                     if (et == 0) p.counters[rem * CG + rank] = 0u;  // hand the counter back zeroed
                 }
