@@ -116,14 +116,13 @@ __device__ __forceinline__ void pass1_chunk(const uint32_t (&acc)[32], int nvis,
     l += (s[0].x + s[0].y) + (s[1].x + s[1].y);
 }
 
-// Pass 2 on one chunk: P = round(127 * e / l) as INT8 codes, 32 keys = two 16-byte pieces of this
-// row of the K-major, 128B-swizzled P tile.
+// Pass 2 on one chunk: P = round(127 * e / l) as INT8 codes, 32 keys = eight packed words (two 16-byte
+// pieces of this row of the K-major, 128B-swizzled P tile, stored by the caller once the tile is free).
 template <bool FULL>
 __device__ __forceinline__ void pass2_chunk(const uint32_t (&acc)[32], int nvis, float c1, float m2, float k127,
-                                            uint8_t* prow, int r, int cc) {
+                                            uint32_t (&w)[8]) {
     const float2 c1v = make_float2(c1, c1), neg_m2 = make_float2(-m2, -m2);
     const float2 k2 = make_float2(k127, k127), magic2 = make_float2(kRoundMagic, kRoundMagic);
-    uint32_t w[8];
 #pragma unroll
     for (int v = 0; v < 8; ++v) {
         uint32_t q[4];
@@ -139,9 +138,6 @@ __device__ __forceinline__ void pass2_chunk(const uint32_t (&acc)[32], int nvis,
         }
         w[v] = pack4(q[0], q[1], q[2], q[3]);
     }
-    const int piece = cc * 2;
-    *reinterpret_cast<uint4*>(prow + (((piece) ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-    *reinterpret_cast<uint4*>(prow + (((piece + 1) ^ (r & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
 }
 
 __global__ void __launch_bounds__(ATT_THREADS, 2)
@@ -344,21 +340,32 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const AttParams p
             uint8_t* prow = s_p + r * 128;
             if (!(ok = warp_wait(bar_s_full + g, s_full_ph, abort_flag, p.status, 27))) break;
             s_full_ph ^= 1u;
+            tcgen05_fence_after();
+            // The codes of this step are computed into registers while the previous step's P.V may still be
+            // reading the P tile; only the stores wait for it.  The score half is handed back as soon as it
+            // has been read, so the next step's score MMA overlaps the rest of this one.
+            uint32_t w[2][8];
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                const int cc = 2 * g + ci;
+                uint32_t acc[32];
+                tmem_ld32(tmem_s + lane_addr + cc * 32, acc);
+                tmem_ld_wait();
+                if (!diag) pass2_chunk<true>(acc, 32, c1, m2, k127, w[ci]);
+                else pass2_chunk<false>(acc, min(32, r - cc * 32 + 1), c1, m2, k127, w[ci]);
+            }
+            tcgen05_fence_before();
+            mbar_arrive(bar_s_free + g);
             if (j > 0) {  // the previous step's P.V has finished reading the P tile
                 if (!(ok = warp_wait(bar_pv_done, pv_done_ph, abort_flag, p.status, 28))) break;
                 pv_done_ph ^= 1u;
             }
-            tcgen05_fence_after();
-#pragma unroll 1
-            for (int cc = 2 * g; cc < 2 * g + 2; ++cc) {
-                uint32_t acc[32];
-                tmem_ld32(tmem_s + lane_addr + cc * 32, acc);
-                tmem_ld_wait();
-                if (!diag) pass2_chunk<true>(acc, 32, c1, m2, k127, prow, r, cc);
-                else pass2_chunk<false>(acc, min(32, r - cc * 32 + 1), c1, m2, k127, prow, r, cc);
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                const int piece = (2 * g + ci) * 2;
+                *reinterpret_cast<uint4*>(prow + (((piece) ^ (r & 7)) << 4)) = make_uint4(w[ci][0], w[ci][1], w[ci][2], w[ci][3]);
+                *reinterpret_cast<uint4*>(prow + (((piece + 1) ^ (r & 7)) << 4)) = make_uint4(w[ci][4], w[ci][5], w[ci][6], w[ci][7]);
             }
-            tcgen05_fence_before();
-            mbar_arrive(bar_s_free + g);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P tile: generic writes -> MMA reads
             mbar_arrive(bar_p_full);
         }
