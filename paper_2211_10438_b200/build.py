@@ -47,6 +47,15 @@ def build_issue_only() -> str:
     return out
 
 
+def build_no_nsplit() -> str:
+    """Tuning build: libsq_no_nsplit.so, in which the prefill GEMM never cuts the tiles of a partly filled last
+    wave into column parts (-DSQ_GEMM_NO_NSPLIT): the "without" arm of that split's A/B timings."""
+    out = os.path.join(HERE, "libsq_no_nsplit.so")
+    subprocess.run([_nvcc(), *NVCC_FLAGS, "-DSQ_GEMM_NO_NSPLIT", "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out],
+                   check=True)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "sq.h"))
@@ -81,5 +90,7 @@ if __name__ == "__main__":
         print(build_trace())
     elif "--issue-only" in sys.argv:
         print(build_issue_only())
+    elif "--no-nsplit" in sys.argv:
+        print(build_no_nsplit())
     else:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

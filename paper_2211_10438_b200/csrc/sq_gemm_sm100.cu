@@ -908,7 +908,12 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
         const int64_t G = sm_count() / CG;
         const int64_t R = (int64_t)p.total_tiles % G;
         const int max_ns = a.out_dt == SQ_I8 ? 2 : 4;  // a staged store row is 128 bytes: a part must fill it
+#ifdef SQ_GEMM_NO_NSPLIT  // tuning build (python -m paper_2211_10438_b200.build --no-nsplit): the split withheld, for A/B timing
+        const int ns = 1;
+        (void)max_ns;
+#else
         const int ns = (p.total_tiles > G && R > 0) ? ((4 * R <= G && max_ns >= 4) ? 4 : (2 * R <= G ? 2 : 1)) : 1;
+#endif
         if (ns > 1) {
             if (!make_map(&mbp, a.B, 1, a.K, a.N, a.heads, a.batch, a.strideB[2], a.strideB[1], a.strideB[0], BLOCK_K,
                           C::B_ROWS / ns, &p.b_slot_row, &p.b_slot_head, &p.b_slot_batch))
