@@ -56,6 +56,17 @@ def build_no_nsplit() -> str:
     return out
 
 
+def build_variant(name: str, defines) -> str:
+    """Tuning build: libsq_<name>.so, the library compiled with extra -D flags.  The kernels read a few of their
+    constants through such macros so that the A/B timings quoted in their comments can be repeated: SQ_KV_STAGES
+    (ring stages per warp of the KV-cache attention, default 2), SQ_DEC_STAGES (ring stages of the decode GEMM,
+    default 10), SQ_LN_NO_TM (LayerNorm parameters in shared instead of tensor memory), SQ_GEMM_NO_L2_HINTS,
+    SQ_GEMM_NO_NSPLIT.  Used through `workloads ... --lib`."""
+    out = os.path.join(HERE, "libsq_%s.so" % name)
+    subprocess.run([_nvcc(), *NVCC_FLAGS, *defines, "-shared", *[os.path.join(CSRC, s) for s in SOURCES], "-o", out], check=True)
+    return out
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
     headers.append(os.path.join(os.path.dirname(HERE), "include", "sq.h"))
@@ -92,5 +103,7 @@ if __name__ == "__main__":
         print(build_issue_only())
     elif "--no-nsplit" in sys.argv:
         print(build_no_nsplit())
+    elif "--variant" in sys.argv:  # --variant NAME -DFLAG[=VALUE] ...
+        print(build_variant(sys.argv[sys.argv.index("--variant") + 1], [a for a in sys.argv if a.startswith("-D")]))
     else:
         print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

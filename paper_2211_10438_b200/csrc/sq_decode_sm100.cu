@@ -46,7 +46,10 @@ template <int DN>
 struct DecCfg {
     static constexpr int X_BYTES = DN * BLOCK_K;
     static constexpr int STAGE = W_BYTES + X_BYTES;
-    static constexpr int STAGES = 10;
+#ifndef SQ_DEC_STAGES  // tuning builds may override it (-DSQ_DEC_STAGES=5)
+#define SQ_DEC_STAGES 10
+#endif
+    static constexpr int STAGES = SQ_DEC_STAGES;
     static constexpr int TMEM_COLS = 2 * DN < 32 ? 32 : 2 * DN;  // two accumulator slots
     static constexpr int SMEM = 1024 + STAGES * STAGE + (2 * STAGES + 7) * 8 + 64 + DN * 4 + 64;
 };

@@ -926,6 +926,10 @@ sq_status launch_ew(const GemmArgs& a, cudaStream_t st) {
     // A single band of m-tiles (A is then re-read by every wave, B streamed exactly once), A well inside the 126 MB L2,
     // and a second wave to find it there.  Measured on B200: 2048 x 5120 x 20480 147.1 -> 143.8 us, DRAM reads 217 -> 183 MB
     // (147 MB of operands); with several bands (8192 x 20480 x 20480) the weights come round once per band and the hints cost 1 %.
+#ifdef SQ_GEMM_NO_L2_HINTS  // tuning build (-DSQ_GEMM_NO_L2_HINTS)
+    p.l2_hints = 0;
+    if (false)
+#endif
     p.l2_hints = (a.batch == 1 && a.heads == 1 && !a.causal && !a.b_is_kn && a.K >= 8192 && a.M <= 8 * BLOCK_M * CG &&
                   a.M * a.K <= (48LL << 20) && (int64_t)p.total_tiles > sm_count() / CG)
                      ? 1 : 0;

@@ -36,7 +36,10 @@ constexpr int KV_TILE = 32;                  // keys per ring stage
 constexpr int KV_TILE_BYTES = KV_TILE * KV_D;
 constexpr int KV_WARPS = 4;
 constexpr int KV_THREADS = KV_WARPS * 32;
-constexpr int KV_STAGES = 2;                 // ring stages per warp (two: four to six CTAs fit an SM, by the score buffer; deeper rings with fewer CTAs measured slower)
+#ifndef SQ_KV_STAGES  // tuning builds may override it: python -m paper_2211_10438_b200.build --variant NAME -DSQ_KV_STAGES=4
+#define SQ_KV_STAGES 2
+#endif
+constexpr int KV_STAGES = SQ_KV_STAGES;                 // ring stages per warp (two: four to six CTAs fit an SM, by the score buffer; deeper rings with fewer CTAs measured slower)
 constexpr int KV_MAX_CLUSTER = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 

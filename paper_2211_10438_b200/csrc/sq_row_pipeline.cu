@@ -40,6 +40,11 @@ namespace sq {
 namespace {
 
 constexpr int CTA_THREADS = 512;
+#ifdef SQ_LN_NO_TM  // tuning build (-DSQ_LN_NO_TM): LayerNorm parameters stay in shared memory at every hidden size
+constexpr bool kLnTensorMemory = false;
+#else
+constexpr bool kLnTensorMemory = true;
+#endif
 
 using namespace bulk;
 template <int GROUP, int CTA = CTA_THREADS>
@@ -575,7 +580,7 @@ sq_status dispatch_pipe(const void* X, int64_t M, int64_t C, const void* gamma, 
         // but loses 7 % at 4096.
 #define SQ_PIPE_LN_TM(GROUP, V, CTA, TMW)                                                                        \
         if (nvec == (GROUP) * (V))                                                                               \
-            return launch_pipe<T, GROUP, V, LN, true, false, CTA, LN ? TMW : 0>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, \
+            return launch_pipe<T, GROUP, V, LN, true, false, CTA, (LN && kLnTensorMemory) ? TMW : 0>(X, M, C, gamma, beta, nullptr, eps, mode, Xq, \
                                                                                 scale, absmax_word, stats, stats_are_input, status, st)
         SQ_PIPE_LN_TM(32, 16, 384, 16);           // 4096
         SQ_PIPE_LN_TM(64, 14, 384, 8);            // 7168
